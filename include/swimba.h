@@ -1,0 +1,163 @@
+/*
+ * swimba.h -- C ABI of the Swimba (Switch Mamba) token-mixer forward for NVIDIA B200.
+ *
+ * The layer (paper, Section "MoE-parameterized SSM" and Theorem 1):
+ *   router    g_t = W_r u_t, pi_t = softmax(g_t) over all E experts; the k largest entries
+ *             are kept with their softmax values, NOT renormalised (Background, "Mixture of
+ *             Experts and Switching Dynamics", router softmax equation and the text after it);
+ *   streams   every active expert maps the same token features to candidate streams
+ *             [B_t^(e) ; C_t^(e)] = W_e[e] u_t (Section "MoE-parameterized SSM");
+ *   mix       Btilde_t = sum_{e in K_t} pi_{t,e} B_t^(e), Ctilde_t likewise (Theorem 1);
+ *   SSM       ONE recurrence with the transition shared by all experts (shared-A equation):
+ *             Delta = softplus(dt + dt_bias), a = exp(Delta * A_h),
+ *             h_t = a h_{t-1} + Delta Btilde_t x_t^T,   y_t = Ctilde_t^T h_t + D_h x_t
+ *             (selective-SSM equation, channelwise convention), evaluated chunk-wise in the
+ *             SSD form (Background, "Mamba-2 and SSD").
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer unless its name ends in _host.  All tensors are
+ *     row-major with the last index contiguous and must be 16-byte aligned.
+ *   - The caller owns every tensor and the workspace; the library owns only the handle (a few
+ *     bytes of device memory for a status word).  Nothing is allocated or freed after create.
+ *   - Calls enqueue work on the given CUDA stream and return without synchronising.
+ *   - Return value: SWIMBA_OK or a negative SWIMBA_ERR_* code.  When an error is detected on
+ *     the host nothing is enqueued and no output is touched.  Nothing throws or aborts.
+ *   - "dtype" below means: float for SWIMBA_DTYPE_FP32, bfloat16 for SWIMBA_DTYPE_BF16.
+ *     A, dt, dt_bias, D, the SSM state and the router weights returned are always float.
+ *   - Notation: T = B*L tokens, F = d_model, H heads, P head_dim, N d_state, G groups,
+ *     S = 2*G*N (mixed stream width: G*N entries of Btilde then G*N of Ctilde), E experts,
+ *     k = top_k.  Head h reads group h / (H/G).
+ */
+#ifndef SWIMBA_H_
+#define SWIMBA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SWIMBA_OK 0
+#define SWIMBA_ERR_NULL_ARG (-1)           /* a required pointer is NULL                      */
+#define SWIMBA_ERR_BAD_CONFIG (-2)         /* a configuration field is out of range           */
+#define SWIMBA_ERR_UNSUPPORTED_SHAPE (-3)  /* B, L or a size combination the kernels lack     */
+#define SWIMBA_ERR_MISALIGNED (-4)         /* a tensor or the workspace is not 16-B aligned   */
+#define SWIMBA_ERR_WORKSPACE_TOO_SMALL (-5)
+#define SWIMBA_ERR_CUDA (-6)               /* a CUDA runtime/driver call failed               */
+#define SWIMBA_ERR_DEVICE_TIMEOUT (-7)     /* a bounded device-side wait ran out              */
+#define SWIMBA_ERR_DEVICE_BOUNDS (-8)      /* a device-side index check failed                */
+
+#define SWIMBA_DTYPE_FP32 0
+#define SWIMBA_DTYPE_BF16 1
+
+#define SWIMBA_MAX_EXPERTS 64
+#define SWIMBA_MAX_TOPK 8
+
+typedef struct swimba_handle swimba_handle; /* opaque, library-owned */
+
+typedef struct {
+    int32_t d_model;   /* F: width of the token features the router and experts read          */
+    int32_t n_heads;   /* H                                                                    */
+    int32_t head_dim;  /* P                                                                    */
+    int32_t d_state;   /* N                                                                    */
+    int32_t n_groups;  /* G, H % G == 0                                                        */
+    int32_t n_experts; /* E, 1..SWIMBA_MAX_EXPERTS                                             */
+    int32_t top_k;     /* k, 1..min(E, SWIMBA_MAX_TOPK); k == E is dense routing               */
+    int32_t chunk;     /* Q in {64,128,256}: SSD chunk length (results do not depend on it)    */
+    int32_t dtype;     /* SWIMBA_DTYPE_*                                                       */
+    int32_t flags;     /* reserved, must be 0                                                  */
+} swimba_config;
+
+typedef struct {
+    const void *W_router;  /* [E, F]        dtype; may be NULL when E == 1                     */
+    const void *W_expert;  /* [E, S, F]     dtype; rows [0,GN) give B, rows [GN,2GN) give C    */
+    const float *A;        /* [H]  negative reals                                              */
+    const float *dt_bias;  /* [H]                                                              */
+    const float *D;        /* [H]  skip weight, may be NULL (no skip term)                     */
+} swimba_weights;
+
+/* Create a layer handle.  Validates the configuration (Section "MoE-parameterized SSM":
+ * E experts, k active, one shared transition) against what the kernels support:
+ * F % 8 == 0, N % 16 == 0 and N <= 256, P <= 256, (N/16 rounded up to a power of two) * P <= 1024.
+ * Uses the current CUDA device.  *out is set only on success. */
+int swimba_create(const swimba_config *cfg, swimba_handle **out);
+
+/* Bytes of device workspace swimba_forward / swimba_route_mix / swimba_ssd need for B
+ * sequences of L tokens (0 if B or L is not positive). */
+size_t swimba_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+
+/* Whole token-mixer forward: router -> top-k -> expert projection -> parameter-space mix ->
+ * one chunked SSD evaluation (Section "MoE-parameterized SSM", state and output equations;
+ * Theorem 1).
+ *   u        [B,L,F]   dtype  token features read by the router and the experts
+ *   x        [B,L,H,P] dtype  SSM input stream (shared by all experts)
+ *   dt       [B,L,H]   float  raw (pre-softplus) step sizes, or NULL meaning dt == 0
+ *   h0       [B,H,P,N] float  initial state, or NULL meaning zeros
+ *   y        [B,L,H,P] dtype  out
+ *   h_final  [B,H,P,N] float  out, may be NULL
+ *   topk_idx [B,L,k]   int32  out, may be NULL: active experts, largest weight first, ties
+ *                             to the lower expert index
+ *   topk_w   [B,L,k]   float  out, may be NULL: their softmax values
+ * L need not be a multiple of the chunk length.  B == 0 or L == 0 is a no-op returning OK. */
+int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                   const float *dt, const float *h0, int32_t B, int32_t L, void *y,
+                   float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,
+                   size_t workspace_bytes, void *cuda_stream);
+
+/* First half of the forward only (router softmax equation, top-k rule, Theorem 1's mixed
+ * streams): u[T,F] -> BC[T,S] dtype (Btilde then Ctilde), topk_idx[T,k], topk_w[T,k]
+ * (either may be NULL).  The workspace is the one sized by swimba_workspace_bytes(h, 1, T). */
+int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
+                     void *BC, int32_t *topk_idx, float *topk_w, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream);
+
+/* Second half only: the single selective-SSM evaluation (selective-SSM equation; Background,
+ * "Mamba-2 and SSD") on given mixed streams BC[B,L,S] dtype.  Other arguments as in
+ * swimba_forward; w->W_router and w->W_expert are not read. */
+int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const void *BC,
+               const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
+               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* Bytes of device workspace swimba_decode_step needs for B sequences. */
+size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B);
+
+/* One autoregressive step (the recurrence of Theorem 1 advanced by one token per sequence,
+ * the O(T) inference mode of Background "Mamba-2 and SSD"): routes and mixes the B tokens,
+ * then state <- a*state + Delta x Btilde^T in place and y = state Ctilde + D x.
+ *   u [B,F] dtype, x [B,H,P] dtype, dt [B,H] float or NULL, state [B,H,P,N] float in/out,
+ *   y [B,H,P] dtype out, topk_idx [B,k] / topk_w [B,k] out or NULL. */
+int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                       const float *dt, float *state, int32_t B, void *y, int32_t *topk_idx,
+                       float *topk_w, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/* End-to-end variant of swimba_forward for callers whose activations live in HOST memory
+ * (pinned memory makes the copies asynchronous): copies u_host, x_host, dt_host (may be NULL)
+ * to device staging, runs the forward of Theorem 1, copies y (and h_final / topk outputs when
+ * given) back, all on the given stream; the caller synchronises the stream before reading.
+ * Weights stay device pointers.  The workspace holds the staging buffers as well and is sized
+ * by swimba_host_workspace_bytes. */
+size_t swimba_host_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u_host,
+                        const void *x_host, const float *dt_host, int32_t B, int32_t L,
+                        void *y_host, float *h_final_host, int32_t *topk_idx_host,
+                        float *topk_w_host, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream);
+
+/* Number of kernels the most recent forward/route_mix/ssd/decode call on this handle enqueued. */
+int swimba_last_launch_count(const swimba_handle *h);
+
+/* Synchronises the stream of the most recent call, then returns SWIMBA_OK or the error code the
+ * device recorded (bounded waits that ran out, failed index checks) and clears it. */
+int swimba_status(swimba_handle *h);
+
+/* Human-readable description of the most recent error on this handle ("" if none). */
+const char *swimba_last_error(const swimba_handle *h);
+
+/* Frees the handle and its device status word.  NULL is allowed. */
+void swimba_destroy(swimba_handle *h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWIMBA_H_ */

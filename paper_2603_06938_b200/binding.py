@@ -1,0 +1,236 @@
+"""ctypes binding over libswimba.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (see include/swimba.h).  Tensors are
+torch CUDA tensors used purely as device memory; every step of the path runs inside the library's
+kernels.  There is no fallback: if the library is missing, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libswimba.so")
+
+OK = 0
+ERR_NULL_ARG = -1
+ERR_BAD_CONFIG = -2
+ERR_UNSUPPORTED_SHAPE = -3
+ERR_MISALIGNED = -4
+ERR_WORKSPACE_TOO_SMALL = -5
+ERR_CUDA = -6
+ERR_DEVICE_TIMEOUT = -7
+ERR_DEVICE_BOUNDS = -8
+DTYPE_FP32 = 0
+DTYPE_BF16 = 1
+
+EXPORTS = [
+    "swimba_create", "swimba_workspace_bytes", "swimba_forward", "swimba_route_mix", "swimba_ssd",
+    "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
+    "swimba_forward_host", "swimba_last_launch_count", "swimba_status", "swimba_last_error",
+    "swimba_destroy",
+]
+
+
+class SwimbaError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"swimba error {code}: {msg}")
+        self.code = code
+
+
+class swimba_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "d_model", "n_heads", "head_dim", "d_state", "n_groups", "n_experts", "top_k", "chunk",
+        "dtype", "flags")]
+
+
+class swimba_weights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("W_router", "W_expert", "A", "dt_bias", "D")]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libswimba.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2603_06938_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        L.swimba_create.argtypes = [ctypes.POINTER(swimba_config), ctypes.POINTER(vp)]
+        L.swimba_create.restype = ctypes.c_int
+        L.swimba_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_workspace_bytes.restype = sz
+        L.swimba_decode_workspace_bytes.argtypes = [vp, i32]
+        L.swimba_decode_workspace_bytes.restype = sz
+        L.swimba_host_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_host_workspace_bytes.restype = sz
+        L.swimba_forward.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32,
+                                     vp, vp, vp, vp, vp, sz, vp]
+        L.swimba_forward.restype = ctypes.c_int
+        L.swimba_route_mix.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, i64, vp, vp, vp, vp,
+                                       sz, vp]
+        L.swimba_route_mix.restype = ctypes.c_int
+        L.swimba_ssd.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32, vp,
+                                 vp, vp, sz, vp]
+        L.swimba_ssd.restype = ctypes.c_int
+        L.swimba_decode_step.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32,
+                                         vp, vp, vp, vp, sz, vp]
+        L.swimba_decode_step.restype = ctypes.c_int
+        L.swimba_forward_host.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, i32, i32,
+                                          vp, vp, vp, vp, vp, sz, vp]
+        L.swimba_forward_host.restype = ctypes.c_int
+        L.swimba_last_launch_count.argtypes = [vp]
+        L.swimba_last_launch_count.restype = ctypes.c_int
+        L.swimba_status.argtypes = [vp]
+        L.swimba_status.restype = ctypes.c_int
+        L.swimba_last_error.argtypes = [vp]
+        L.swimba_last_error.restype = ctypes.c_char_p
+        L.swimba_destroy.argtypes = [vp]
+        L.swimba_destroy.restype = None
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors must be contiguous"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Handle:
+    """Owns one swimba_handle*; `cfg` mirrors the C configuration."""
+
+    def __init__(self, ptr: ctypes.c_void_p, cfg: swimba_config):
+        self.ptr = ptr
+        self.cfg = cfg
+
+    def _raise(self, code: int):
+        msg = lib().swimba_last_error(self.ptr)
+        raise SwimbaError(code, msg.decode() if msg else "")
+
+
+def swimba_create(d_model: int, n_heads: int, head_dim: int, d_state: int, n_groups: int,
+                  n_experts: int, top_k: int, chunk: int, dtype: int, flags: int = 0) -> Handle:
+    cfg = swimba_config(d_model, n_heads, head_dim, d_state, n_groups, n_experts, top_k, chunk,
+                        dtype, flags)
+    out = ctypes.c_void_p()
+    rc = lib().swimba_create(ctypes.byref(cfg), ctypes.byref(out))
+    if rc != OK:
+        raise SwimbaError(rc, "swimba_create rejected the configuration")
+    return Handle(out, cfg)
+
+
+def swimba_destroy(h: Handle) -> None:
+    if h.ptr:
+        lib().swimba_destroy(h.ptr)
+        h.ptr = None
+
+
+def make_weights(W_router, W_expert, A, dt_bias, D) -> swimba_weights:
+    w = swimba_weights()
+    w.W_router = W_router.data_ptr() if W_router is not None else None
+    w.W_expert = W_expert.data_ptr() if W_expert is not None else None
+    w.A = A.data_ptr() if A is not None else None
+    w.dt_bias = dt_bias.data_ptr() if dt_bias is not None else None
+    w.D = D.data_ptr() if D is not None else None
+    w._keep = (W_router, W_expert, A, dt_bias, D)   # keep the tensors alive
+    return w
+
+
+def swimba_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_decode_workspace_bytes(h: Handle, B: int) -> int:
+    return int(lib().swimba_decode_workspace_bytes(h.ptr, B))
+
+
+def swimba_host_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_host_workspace_bytes(h.ptr, B, L))
+
+
+def _ws(workspace: Optional[torch.Tensor]):
+    if workspace is None:
+        return None, 0
+    return ctypes.c_void_p(workspace.data_ptr()), workspace.numel() * workspace.element_size()
+
+
+def swimba_forward(h: Handle, w: swimba_weights, u, x, dt, h0, B: int, L: int, y, h_final,
+                   topk_idx, topk_w, workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_forward(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), B, L,
+                              _ptr(y), _ptr(h_final), _ptr(topk_idx), _ptr(topk_w), wp, wb,
+                              _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_route_mix(h: Handle, w: swimba_weights, u, T: int, BC, topk_idx, topk_w, workspace,
+                     stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_route_mix(h.ptr, ctypes.byref(w), _ptr(u), T, _ptr(BC), _ptr(topk_idx),
+                                _ptr(topk_w), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_ssd(h: Handle, w: swimba_weights, x, BC, dt, h0, B: int, L: int, y, h_final, workspace,
+               stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_ssd(h.ptr, ctypes.byref(w), _ptr(x), _ptr(BC), _ptr(dt), _ptr(h0), B, L,
+                          _ptr(y), _ptr(h_final), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_decode_step(h: Handle, w: swimba_weights, u, x, dt, state, B: int, y, topk_idx, topk_w,
+                       workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_decode_step(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(state),
+                                  B, _ptr(y), _ptr(topk_idx), _ptr(topk_w), wp, wb,
+                                  _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B: int, L: int,
+                        y_host, h_final_host, topk_idx_host, topk_w_host, workspace, stream=None,
+                        check: bool = True) -> int:
+    """Host tensors (ideally pinned) in and out; the caller synchronises the stream."""
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_forward_host(h.ptr, ctypes.byref(w), _ptr(u_host), _ptr(x_host),
+                                   _ptr(dt_host), B, L, _ptr(y_host), _ptr(h_final_host),
+                                   _ptr(topk_idx_host), _ptr(topk_w_host), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_last_launch_count(h: Handle) -> int:
+    return int(lib().swimba_last_launch_count(h.ptr))
+
+
+def swimba_status(h: Handle) -> int:
+    return int(lib().swimba_status(h.ptr))
+
+
+def swimba_last_error(h: Handle) -> str:
+    msg = lib().swimba_last_error(h.ptr)
+    return msg.decode() if msg else ""

@@ -1,0 +1,385 @@
+// Host side of the C ABI: handle, argument validation, workspace layout and kernel sequencing.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace swimba;
+
+struct swimba_handle {
+    swimba_config cfg;
+    int device;
+    int sm_count;
+    int *d_status;          // device status word
+    cudaStream_t last_stream;
+    int last_launches;
+    char err[256];
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t elt_size(int dtype) { return dtype == SWIMBA_DTYPE_FP32 ? 4 : 2; }
+
+int fail(swimba_handle *h, int code, const char *msg)
+{
+    if (h) snprintf(h->err, sizeof(h->err), "%s", msg);
+    return code;
+}
+
+// Workspace of the forward: [BC | idx | w], each 256-byte aligned.
+struct FwdLayout {
+    size_t bc, idx, w, total;
+};
+FwdLayout fwd_layout(const swimba_config &c, int64_t T)
+{
+    FwdLayout l;
+    const size_t S = 2u * c.n_groups * c.d_state;
+    size_t off = 0;
+    l.bc = off;  off += align_up((size_t)T * S * elt_size(c.dtype));
+    l.idx = off; off += align_up((size_t)T * c.top_k * sizeof(int32_t));
+    l.w = off;   off += align_up((size_t)T * c.top_k * sizeof(float));
+    l.total = off;
+    return l;
+}
+
+// Workspace of a decode step: [BC fp32 | idx | w].
+struct DecLayout {
+    size_t bc, idx, w, total;
+};
+DecLayout dec_layout(const swimba_config &c, int B)
+{
+    DecLayout l;
+    const size_t S = 2u * c.n_groups * c.d_state;
+    size_t off = 0;
+    l.bc = off;  off += align_up((size_t)B * S * sizeof(float));
+    l.idx = off; off += align_up((size_t)B * c.top_k * sizeof(int32_t));
+    l.w = off;   off += align_up((size_t)B * c.top_k * sizeof(float));
+    l.total = off;
+    return l;
+}
+
+// Host-variant staging: [u | x | dt | y | h_final | idx | w] in front of the forward workspace.
+struct HostLayout {
+    size_t u, x, dt, y, hf, idx, w, fwd, total;
+};
+HostLayout host_layout(const swimba_config &c, int B, int L)
+{
+    HostLayout l;
+    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const size_t HP = (size_t)c.n_heads * c.head_dim;
+    size_t off = 0;
+    l.u = off;   off += align_up(T * c.d_model * es);
+    l.x = off;   off += align_up(T * HP * es);
+    l.dt = off;  off += align_up(T * c.n_heads * sizeof(float));
+    l.y = off;   off += align_up(T * HP * es);
+    l.hf = off;  off += align_up((size_t)B * HP * c.d_state * sizeof(float));
+    l.idx = off; off += align_up(T * c.top_k * sizeof(int32_t));
+    l.w = off;   off += align_up(T * c.top_k * sizeof(float));
+    l.fwd = off; off += fwd_layout(c, (int64_t)T).total;
+    l.total = off;
+    return l;
+}
+
+int check_weights(swimba_handle *h, const swimba_weights *w, bool need_experts)
+{
+    if (!w) return fail(h, SWIMBA_ERR_NULL_ARG, "weights struct is NULL");
+    if (!w->A || !w->dt_bias) return fail(h, SWIMBA_ERR_NULL_ARG, "A or dt_bias is NULL");
+    if (need_experts) {
+        if (!w->W_expert) return fail(h, SWIMBA_ERR_NULL_ARG, "W_expert is NULL");
+        if (!w->W_router && h->cfg.n_experts > 1)
+            return fail(h, SWIMBA_ERR_NULL_ARG, "W_router is NULL with more than one expert");
+        if (!aligned16(w->W_expert) || !aligned16(w->W_router))
+            return fail(h, SWIMBA_ERR_MISALIGNED, "weights must be 16-byte aligned");
+    }
+    if (!aligned16(w->A) || !aligned16(w->dt_bias) || !aligned16(w->D))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "A/dt_bias/D must be 16-byte aligned");
+    return SWIMBA_OK;
+}
+
+int set_device(swimba_handle *h)
+{
+    int cur = -1;
+    if (cudaGetDevice(&cur) != cudaSuccess) return fail(h, SWIMBA_ERR_CUDA, "cudaGetDevice failed");
+    if (cur != h->device) return fail(h, SWIMBA_ERR_CUDA, "handle used on a different device than it was created on");
+    return SWIMBA_OK;
+}
+
+// Router + projection + mix into BC (dtype, or fp32 when bc_fp32).
+int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *u,
+                  int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt)
+{
+    const swimba_config &c = h->cfg;
+    const int S = 2 * c.n_groups * c.d_state;
+    // With one expert the softmax is identically 1; the router kernel handles it without W_router
+    // being dereferenced only if it is given, so substitute the expert matrix as a dummy operand.
+    const void *Wr = w->W_router ? w->W_router : w->W_expert;
+    int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt);
+    if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
+    rc = launch_project_mix_simt(ctx, c.dtype, u, w->W_expert, idx, wt, T, c.d_model, S,
+                                 c.n_experts, c.top_k, BC, bc_fp32);
+    if (rc != SWIMBA_OK) return fail(h, rc, "projection launch failed");
+    return SWIMBA_OK;
+}
+
+int run_ssd(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *x,
+            const void *BC, const float *dt, const float *h0, int B, int L, void *y,
+            float *h_final)
+{
+    const swimba_config &c = h->cfg;
+    int rc = launch_ssd_sequential(ctx, c.dtype, x, BC, false, dt, w->A, w->dt_bias, w->D, h0, B, L,
+                                   c.n_heads, c.head_dim, c.d_state, c.n_groups, y, h_final);
+    if (rc != SWIMBA_OK) return fail(h, rc, "SSD launch failed");
+    return SWIMBA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int swimba_create(const swimba_config *cfg, swimba_handle **out)
+{
+    if (!cfg || !out) return SWIMBA_ERR_NULL_ARG;
+    const swimba_config &c = *cfg;
+    if (c.d_model <= 0 || c.n_heads <= 0 || c.head_dim <= 0 || c.d_state <= 0 || c.n_groups <= 0 ||
+        c.n_experts <= 0 || c.top_k <= 0)
+        return SWIMBA_ERR_BAD_CONFIG;
+    if (c.n_heads % c.n_groups != 0) return SWIMBA_ERR_BAD_CONFIG;
+    if (c.n_experts > SWIMBA_MAX_EXPERTS || c.top_k > c.n_experts || c.top_k > SWIMBA_MAX_TOPK)
+        return SWIMBA_ERR_BAD_CONFIG;
+    if (c.chunk != 64 && c.chunk != 128 && c.chunk != 256) return SWIMBA_ERR_BAD_CONFIG;
+    if (c.dtype != SWIMBA_DTYPE_FP32 && c.dtype != SWIMBA_DTYPE_BF16) return SWIMBA_ERR_BAD_CONFIG;
+    if (c.flags != 0) return SWIMBA_ERR_BAD_CONFIG;
+    if (c.d_model % 8 != 0 || c.d_state % 16 != 0 || c.d_state > 256 || c.head_dim > 256)
+        return SWIMBA_ERR_UNSUPPORTED_SHAPE;
+    int ns = 1;
+    while (ns * 16 < c.d_state) ns <<= 1;
+    if (ns * c.head_dim > 1024) return SWIMBA_ERR_UNSUPPORTED_SHAPE;
+
+    swimba_handle *h = new (std::nothrow) swimba_handle;
+    if (!h) return SWIMBA_ERR_CUDA;
+    memset(h, 0, sizeof(*h));
+    h->cfg = c;
+    if (cudaGetDevice(&h->device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess ||
+        cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
+        if (h->d_status) cudaFree(h->d_status);
+        delete h;
+        cudaGetLastError();
+        return SWIMBA_ERR_CUDA;
+    }
+    *out = h;
+    return SWIMBA_OK;
+}
+
+size_t swimba_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    return fwd_layout(h->cfg, (int64_t)B * L).total;
+}
+
+size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B)
+{
+    if (!h || B <= 0) return 0;
+    return dec_layout(h->cfg, B).total;
+}
+
+size_t swimba_host_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    return host_layout(h->cfg, B, L).total;
+}
+
+int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
+                     void *BC, int32_t *topk_idx, float *topk_w, void *workspace,
+                     size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (T < 0 || T > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !BC || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC or workspace is NULL");
+    if (!aligned16(u) || !aligned16(BC) || !aligned16(workspace) || !aligned16(topk_idx) || !aligned16(topk_w))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const FwdLayout l = fwd_layout(h->cfg, T);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt);
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const void *BC,
+               const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
+               void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    int rc = check_weights(h, w, false);
+    if (rc != SWIMBA_OK) return rc;
+    if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!x || !BC || !y) return fail(h, SWIMBA_ERR_NULL_ARG, "x, BC or y is NULL");
+    if (!aligned16(x) || !aligned16(BC) || !aligned16(y) || !aligned16(dt) || !aligned16(h0) ||
+        !aligned16(h_final) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    (void)workspace_bytes;
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                   const float *dt, const float *h0, int32_t B, int32_t L, void *y,
+                   float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,
+                   size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    if ((int64_t)B * L > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !x || !y || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, x, y or workspace is NULL");
+    if (!aligned16(u) || !aligned16(x) || !aligned16(y) || !aligned16(dt) || !aligned16(h0) ||
+        !aligned16(h_final) || !aligned16(topk_idx) || !aligned16(topk_w) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const int64_t T = (int64_t)B * L;
+    const FwdLayout l = fwd_layout(h->cfg, T);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    void *BC = ws + l.bc;
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt);
+    if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                       const float *dt, float *state, int32_t B, void *y, int32_t *topk_idx,
+                       float *topk_w, void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (B == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !x || !y || !state || !workspace)
+        return fail(h, SWIMBA_ERR_NULL_ARG, "u, x, y, state or workspace is NULL");
+    if (!aligned16(u) || !aligned16(x) || !aligned16(y) || !aligned16(dt) || !aligned16(state) ||
+        !aligned16(topk_idx) || !aligned16(topk_w) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const DecLayout l = dec_layout(h->cfg, B);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    const swimba_config &c = h->cfg;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    float *BC = (float *)(ws + l.bc);
+    rc = run_route_mix(h, ctx, w, u, B, BC, true, idx, wt);
+    if (rc == SWIMBA_OK) {
+        rc = launch_decode_update(ctx, c.dtype, x, BC, dt, w->A, w->dt_bias, w->D, state, B,
+                                  c.n_heads, c.head_dim, c.d_state, c.n_groups, y);
+        if (rc != SWIMBA_OK) fail(h, rc, "decode launch failed");
+    }
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u_host,
+                        const void *x_host, const float *dt_host, int32_t B, int32_t L,
+                        void *y_host, float *h_final_host, int32_t *topk_idx_host,
+                        float *topk_w_host, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u_host || !x_host || !y_host || !workspace)
+        return fail(h, SWIMBA_ERR_NULL_ARG, "u_host, x_host, y_host or workspace is NULL");
+    if (!aligned16(workspace)) return fail(h, SWIMBA_ERR_MISALIGNED, "workspace must be 16-byte aligned");
+    const swimba_config &c = h->cfg;
+    const HostLayout l = host_layout(c, B, L);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    char *ws = (char *)workspace;
+    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const size_t HP = (size_t)c.n_heads * c.head_dim;
+    bool ok = cudaMemcpyAsync(ws + l.u, u_host, T * c.d_model * es, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(ws + l.x, x_host, T * HP * es, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (dt_host)
+        ok = ok && cudaMemcpyAsync(ws + l.dt, dt_host, T * c.n_heads * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "host-to-device copy failed"); }
+    rc = swimba_forward(h, w, ws + l.u, ws + l.x, dt_host ? (const float *)(ws + l.dt) : nullptr,
+                        nullptr, B, L, ws + l.y, h_final_host ? (float *)(ws + l.hf) : nullptr,
+                        (int32_t *)(ws + l.idx), (float *)(ws + l.w), ws + l.fwd,
+                        workspace_bytes - l.fwd, cuda_stream);
+    if (rc != SWIMBA_OK) return rc;
+    ok = cudaMemcpyAsync(y_host, ws + l.y, T * HP * es, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (h_final_host)
+        ok = ok && cudaMemcpyAsync(h_final_host, ws + l.hf, (size_t)B * HP * c.d_state * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (topk_idx_host)
+        ok = ok && cudaMemcpyAsync(topk_idx_host, ws + l.idx, T * c.top_k * sizeof(int32_t), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (topk_w_host)
+        ok = ok && cudaMemcpyAsync(topk_w_host, ws + l.w, T * c.top_k * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "device-to-host copy failed"); }
+    return SWIMBA_OK;
+}
+
+int swimba_last_launch_count(const swimba_handle *h) { return h ? h->last_launches : 0; }
+
+int swimba_status(swimba_handle *h)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) {
+        snprintf(h->err, sizeof(h->err), "stream synchronisation failed: %s",
+                 cudaGetErrorString(cudaGetLastError()));
+        return SWIMBA_ERR_CUDA;
+    }
+    int code = 0;
+    if (cudaMemcpy(&code, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(h, SWIMBA_ERR_CUDA, "reading the device status word failed");
+    if (code != 0) {
+        cudaMemset(h->d_status, 0, 64);
+        snprintf(h->err, sizeof(h->err), "device reported error %d", code);
+    }
+    return code;
+}
+
+const char *swimba_last_error(const swimba_handle *h) { return h ? h->err : ""; }
+
+void swimba_destroy(swimba_handle *h)
+{
+    if (!h) return;
+    if (h->d_status) cudaFree(h->d_status);
+    delete h;
+}
+
+}  // extern "C"

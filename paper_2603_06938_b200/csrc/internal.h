@@ -1,0 +1,28 @@
+// Launchers shared between the API translation unit and the kernel files.
+#pragma once
+#include "common.cuh"
+
+namespace swimba {
+
+// K1a: router logits, softmax over all E, top-k (indices + un-renormalised weights).
+int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
+                  int E, int k, int32_t *idx, float *w);
+
+// K1b (SIMT): project the k selected experts and mix.  BC is written in `dtype`, or as float
+// per slot-sum when bc_fp32 is set.
+int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void *W_e,
+                            const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
+                            int k, void *BC, bool bc_fp32);
+
+// Per-timestep SIMT evaluation of the recurrence (fp32 state in registers).
+int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
+                          const float *dt, const float *A, const float *dt_bias, const float *D,
+                          const float *h0, int B, int L, int H, int P, int N, int G, void *y,
+                          float *h_final);
+
+// K4: one-token state update, state[B,H,P,N] in place.
+int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const float *BC,
+                         const float *dt, const float *A, const float *dt_bias, const float *D,
+                         float *state, int B, int H, int P, int N, int G, void *y);
+
+}  // namespace swimba

@@ -1,0 +1,126 @@
+"""Shared test plumbing: run one layer through the CUDA library and through the CPU oracle on the
+same seeded host arrays, and compare under the routing protocol.
+
+Routing protocol.  The library computes router logits from the same (bf16 or fp32) inputs in fp32,
+the oracle in fp64.  A token is *certified* when the smallest gap among its k+1 largest oracle
+logits exceeds twice the worst-case fp32 summation error F * 2^-24 * sum_f |W_r[e,f] u[t,f]|; for
+those tokens indices must match bit for bit, order included.  The few remaining near-tied tokens
+may differ; the oracle is then re-run with the library's routing forced so that every token's
+float outputs are still compared.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2603_06938_b200 import binding as sb
+from paper_2603_06938_b200 import synth
+
+
+def dtype_code(cfg: synth.LayerConfig) -> int:
+    return sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
+
+
+def create_handle(cfg: synth.LayerConfig, chunk=None) -> sb.Handle:
+    return sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k,
+                            chunk if chunk is not None else cfg.Q, dtype_code(cfg))
+
+
+def dev(t):
+    return None if t is None else t.cuda().contiguous()
+
+
+def device_weights(inp):
+    keep = {n: dev(inp[n]) for n in ("W_r", "W_e", "A", "dt_bias", "D")}
+    return sb.make_weights(keep["W_r"], keep["W_e"], keep["A"], keep["dt_bias"], keep["D"]), keep
+
+
+def gpu_forward(cfg: synth.LayerConfig, inp, chunk=None, h0=None, want_topk=True):
+    """Runs swimba_forward; returns host tensors dict(y, h_final, idx, w)."""
+    h = create_handle(cfg, chunk)
+    try:
+        B, L = inp["u"].shape[0], inp["u"].shape[1]
+        w, keep = device_weights(inp)
+        u, x, dt = dev(inp["u"]), dev(inp["x"]), dev(inp["dt"])
+        h0d = dev(h0 if h0 is not None else inp.get("h0"))
+        y = torch.full_like(x, float("nan"))
+        hf = torch.full((B, cfg.H, cfg.P, cfg.N), float("nan"), device="cuda")
+        idx = torch.full((B, L, cfg.k), -1, dtype=torch.int32, device="cuda") if want_topk else None
+        wt = torch.full((B, L, cfg.k), float("nan"), device="cuda") if want_topk else None
+        ws = torch.empty(max(sb.swimba_workspace_bytes(h, B, L), 16), dtype=torch.uint8, device="cuda")
+        sb.swimba_forward(h, w, u, x, dt, h0d, B, L, y, hf, idx, wt, ws)
+        rc = sb.swimba_status(h)
+        assert rc == 0, sb.swimba_last_error(h)
+        launches = sb.swimba_last_launch_count(h)
+        return dict(y=y.cpu(), h_final=hf.cpu(), idx=None if idx is None else idx.cpu(),
+                    w=None if wt is None else wt.cpu(), launches=launches)
+    finally:
+        sb.swimba_destroy(h)
+
+
+def oracle_forward(cfg: synth.LayerConfig, inp, h0=None, forced_idx=None, forced_w=None):
+    h0 = h0 if h0 is not None else inp.get("h0")
+    return oracle.swimba_forward(
+        synth.f64(inp["u"]), synth.f64(inp["x"]), synth.f64(inp["dt"]), synth.f64(inp["W_r"]),
+        synth.f64(inp["W_e"]), synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), synth.f64(inp["D"]),
+        k=cfg.k, G=cfg.G, h0=synth.f64(h0), forced_idx=forced_idx, forced_w=forced_w)
+
+
+def max_rel(got, ref) -> float:
+    """max |got - ref| / max |ref| over the whole tensor."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    den = np.max(np.abs(ref))
+    return float(np.max(np.abs(got - ref)) / (den if den > 0 else 1.0))
+
+
+def check_routing(cfg: synth.LayerConfig, inp, idx_gpu, w_gpu, require_all_certified=False):
+    """Certified tokens must match exactly; returns (#ambiguous tokens, oracle router output)."""
+    F = cfg.F
+    u2 = synth.f64(inp["u"]).reshape(-1, F)
+    r = oracle.router(u2, synth.f64(inp["W_r"]), cfg.k)
+    idx_gpu = idx_gpu.numpy().reshape(-1, cfg.k)
+    w_gpu = w_gpu.numpy().reshape(-1, cfg.k)
+    bound = 2.0 * F * 2.0 ** -24 * r["absdot"]
+    certified = r["margin"] > bound
+    if cfg.E == cfg.k == 1:
+        certified[:] = True
+    assert np.array_equal(idx_gpu[certified], r["idx"][certified]), "certified routing differs"
+    n_amb = int((~certified).sum())
+    if require_all_certified:
+        assert n_amb == 0
+    # ambiguous tokens must still pick k distinct valid experts
+    assert idx_gpu.min() >= 0 and idx_gpu.max() < cfg.E
+    if cfg.k > 1:
+        srt = np.sort(idx_gpu, axis=-1)
+        assert np.all(srt[:, 1:] != srt[:, :-1])
+    # weights: softmax values of the chosen experts (no renormalisation)
+    chosen = np.take_along_axis(r["pi"], idx_gpu.astype(np.int64), axis=-1)
+    np.testing.assert_allclose(w_gpu, chosen, rtol=2e-5, atol=1e-7)
+    return n_amb, r
+
+
+def compare_forward(cfg: synth.LayerConfig, inp, got, tol_y, tol_h, h0=None,
+                    require_all_certified=False):
+    n_amb, _ = check_routing(cfg, inp, got["idx"], got["w"], require_all_certified)
+    B, L = inp["u"].shape[:2]
+    forced_idx = got["idx"].numpy().reshape(B, L, cfg.k)
+    forced_w = None
+    if n_amb:
+        # weights for the library's routing, in fp64, from the oracle's own softmax
+        r = oracle.router(synth.f64(inp["u"]).reshape(-1, cfg.F), synth.f64(inp["W_r"]), cfg.k)
+        forced_w = np.take_along_axis(r["pi"], forced_idx.reshape(-1, cfg.k).astype(np.int64), -1)
+        ref = oracle_forward(cfg, inp, h0=h0, forced_idx=forced_idx, forced_w=forced_w)
+    else:
+        ref = oracle_forward(cfg, inp, h0=h0)
+    ey = max_rel(got["y"].double().numpy(), ref["y"])
+    eh = max_rel(got["h_final"].double().numpy(), ref["h_final"])
+    assert ey <= tol_y, f"y max-rel error {ey:.3e} > {tol_y}"
+    assert eh <= tol_h, f"h_final max-rel error {eh:.3e} > {tol_h}"
+    return dict(err_y=ey, err_h=eh, ambiguous=n_amb, ref=ref)
+
+
+def tolerances(cfg: synth.LayerConfig):
+    """fp32 path: 1e-4 on everything; bf16 inputs with fp32 accumulation: 2e-2 on y, 1e-2 on state."""
+    return (1e-4, 1e-4) if cfg.dtype == "fp32" else (2e-2, 1e-2)

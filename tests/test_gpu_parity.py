@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: routing indices bit-exact (see helpers.check_routing for
+near-ties); fp32 path 1e-4 max relative error; bf16 inputs with fp32 accumulation 2e-2 on y and
+1e-2 on the final state, both as max|got-ref| / max|ref|.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2603_06938_b200 import binding as sb
+from paper_2603_06938_b200 import synth
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def cfg_of(dtype="bf16", **kw):
+    base = dict(name="case", dtype=dtype, B=2, L=300, F=64, H=4, P=64, N=128, G=1, E=4, k=2, Q=128)
+    base.update(kw)
+    return synth.LayerConfig(**base)
+
+
+# ------------------------------------------------------------------ config 0, whole tensor
+def test_tiny_fp32_config_full_parity():
+    cfg = synth.CONFIGS["tiny_fp32"]
+    inp = synth.make_inputs(cfg, seed=0)
+    got = hp.gpu_forward(cfg, inp)
+    res = hp.compare_forward(cfg, inp, got, 1e-4, 1e-4, require_all_certified=True)
+    assert got["launches"] > 0
+    assert res["ambiguous"] == 0
+
+
+# ------------------------------------------------------------ small, odd and ragged shapes
+CASES = [
+    cfg_of("bf16"),                                        # several tiles + ragged tail
+    cfg_of("bf16", L=77, B=3),                             # shorter than one tile
+    cfg_of("bf16", L=128, B=1),                            # exactly one tile
+    cfg_of("bf16", L=1, B=2),                              # single token
+    cfg_of("bf16", L=513, k=4, E=4),                       # dense routing (k == E)
+    cfg_of("bf16", L=260, k=1, E=8),                       # switch routing
+    cfg_of("bf16", L=260, k=1, E=1),                       # plain Mamba-2 (router skipped)
+    cfg_of("bf16", L=200, H=4, G=2),                       # two B/C groups
+    cfg_of("bf16", L=300, H=3, P=32, N=64, F=40),          # other head/state sizes
+    cfg_of("bf16", L=700, H=2, E=16, k=3, F=136),
+    cfg_of("fp32", L=150, N=16, P=64, H=3, F=48),
+    cfg_of("fp32", L=97, N=32, P=16, H=2, G=2, E=3, k=2, F=24),
+    cfg_of("fp32", L=64, N=128, P=64, H=2, E=5, k=5, F=72),
+]
+
+
+@pytest.mark.parametrize("i", range(len(CASES)))
+def test_small_shapes_full_parity(i):
+    cfg = CASES[i]
+    inp = synth.make_inputs(cfg, seed=100 + i)
+    got = hp.gpu_forward(cfg, inp)
+    hp.compare_forward(cfg, inp, got, *hp.tolerances(cfg))
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_optional_arguments_and_initial_state(dtype):
+    cfg = cfg_of(dtype, L=210, h0_std=0.5, N=64 if dtype == "fp32" else 128)
+    inp = synth.make_inputs(cfg, seed=7, with_dt=False)     # dt == NULL: time-invariant transition
+    inp["D"] = None                                         # no skip term
+    got = hp.gpu_forward(cfg, inp, want_topk=False)
+    ref = hp.oracle_forward(cfg, inp)
+    ty, th = hp.tolerances(cfg)
+    assert hp.max_rel(got["y"].double().numpy(), ref["y"]) <= ty
+    assert hp.max_rel(got["h_final"].double().numpy(), ref["h_final"]) <= th
+
+
+def test_empty_inputs_are_a_no_op():
+    cfg = cfg_of("bf16")
+    h = hp.create_handle(cfg)
+    inp = synth.make_inputs(dataclasses.replace(cfg, L=4), seed=1)
+    w, keep = hp.device_weights(inp)
+    assert sb.swimba_workspace_bytes(h, 0, 10) == 0
+    assert sb.swimba_forward(h, w, None, None, None, None, 0, 5, None, None, None, None, None) == 0
+    assert sb.swimba_forward(h, w, None, None, None, None, 3, 0, None, None, None, None, None) == 0
+    assert sb.swimba_status(h) == 0
+    sb.swimba_destroy(h)
+
+
+# ------------------------------------------------------------------------------ properties
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_result_does_not_depend_on_chunk_length(dtype):
+    cfg = cfg_of(dtype, L=600, N=64 if dtype == "fp32" else 128)
+    inp = synth.make_inputs(cfg, seed=11)
+    ref = hp.oracle_forward(cfg, inp)
+    ty, th = hp.tolerances(cfg)
+    for Q in (64, 128, 256):
+        got = hp.gpu_forward(cfg, inp, chunk=Q)
+        assert hp.max_rel(got["y"].double().numpy(), ref["y"]) <= ty
+        assert hp.max_rel(got["h_final"].double().numpy(), ref["h_final"]) <= th
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_two_calls_with_carried_state_equal_one_call(dtype):
+    cfg = cfg_of(dtype, L=500, B=2, N=64 if dtype == "fp32" else 128)
+    inp = synth.make_inputs(cfg, seed=12)
+    whole = hp.gpu_forward(cfg, inp)
+    cut = 207
+    first = {k: (v[:, :cut] if k in ("u", "x", "dt") else v) for k, v in inp.items()}
+    second = {k: (v[:, cut:] if k in ("u", "x", "dt") else v) for k, v in inp.items()}
+    g1 = hp.gpu_forward(dataclasses.replace(cfg, L=cut), {k: (v.contiguous() if torch.is_tensor(v) else v) for k, v in first.items()})
+    g2 = hp.gpu_forward(dataclasses.replace(cfg, L=cfg.L - cut), {k: (v.contiguous() if torch.is_tensor(v) else v) for k, v in second.items()}, h0=g1["h_final"])
+    y12 = torch.cat([g1["y"], g2["y"]], 1)
+    ty, th = hp.tolerances(cfg)
+    assert hp.max_rel(y12.double().numpy(), whole["y"].double().numpy()) <= ty
+    assert hp.max_rel(g2["h_final"].numpy(), whole["h_final"].numpy()) <= th
+    ref = hp.oracle_forward(cfg, inp)
+    assert hp.max_rel(y12.double().numpy(), ref["y"]) <= ty
+    assert hp.max_rel(g2["h_final"].double().numpy(), ref["h_final"]) <= th
+
+
+def test_forward_is_bitwise_reproducible():
+    cfg = cfg_of("bf16", L=400)
+    inp = synth.make_inputs(cfg, seed=13)
+    a = hp.gpu_forward(cfg, inp)
+    b = hp.gpu_forward(cfg, inp)
+    assert torch.equal(a["y"].view(torch.int16), b["y"].view(torch.int16))
+    assert torch.equal(a["h_final"], b["h_final"])
+    assert torch.equal(a["idx"], b["idx"])
+
+
+def test_theorem3_state_bound_holds_on_device():
+    # ||h_T|| <= rho^T ||h_0|| + (1-rho^T)/(1-rho) U, per (head, channel), with the mixed streams
+    cfg = cfg_of("fp32", L=256, B=1, N=32, P=16, H=2, h0_std=1.0)
+    inp = synth.make_inputs(cfg, seed=14)
+    got = hp.gpu_forward(cfg, inp)
+    ref = hp.oracle_forward(cfg, inp)
+    dlt = np.logaddexp(0.0, synth.f64(inp["dt"]) + synth.f64(inp["dt_bias"]))
+    a = np.exp(dlt * synth.f64(inp["A"]))
+    Bt = ref["BC"][0, :, :cfg.N]
+    x = synth.f64(inp["x"])
+    for h in range(cfg.H):
+        rho = a[0, :, h].max()
+        for p in range(cfg.P):
+            U = np.linalg.norm(dlt[0, :, h, None] * x[0, :, h, p, None] * Bt, axis=-1).max()
+            bound = rho ** cfg.L * np.linalg.norm(synth.f64(inp["h0"])[0, h, p]) + \
+                (1 - rho ** cfg.L) / (1 - rho) * U
+            assert np.linalg.norm(got["h_final"][0, h, p].double().numpy()) <= bound * (1 + 1e-4)
+
+
+# ------------------------------------------------------------------------- split entry points
+def test_route_mix_and_ssd_entry_points():
+    cfg = cfg_of("bf16", L=300)
+    inp = synth.make_inputs(cfg, seed=15)
+    B, L = cfg.B, cfg.L
+    h = hp.create_handle(cfg)
+    w, keep = hp.device_weights(inp)
+    u, x, dt = hp.dev(inp["u"]), hp.dev(inp["x"]), hp.dev(inp["dt"])
+    ws = torch.empty(sb.swimba_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    BC = torch.empty(B, L, cfg.S, dtype=torch.bfloat16, device="cuda")
+    idx = torch.empty(B, L, cfg.k, dtype=torch.int32, device="cuda")
+    wt = torch.empty(B, L, cfg.k, device="cuda")
+    sb.swimba_route_mix(h, w, u, B * L, BC, idx, wt, ws)
+    assert sb.swimba_status(h) == 0
+    hp.check_routing(cfg, inp, idx.cpu(), wt.cpu())
+    ref_bc = oracle.mix_topk(synth.f64(inp["u"]).reshape(B * L, -1), synth.f64(inp["W_e"]),
+                             idx.cpu().numpy().reshape(B * L, -1), wt.cpu().double().numpy().reshape(B * L, -1))
+    assert hp.max_rel(BC.cpu().double().numpy().reshape(B * L, -1), ref_bc) <= 1e-2
+    # SSD on the library's own (bf16-rounded) mixed streams against the oracle recurrence on them
+    y = torch.empty_like(x)
+    hf = torch.empty(B, cfg.H, cfg.P, cfg.N, device="cuda")
+    sb.swimba_ssd(h, w, x, BC, dt, None, B, L, y, hf, ws)
+    assert sb.swimba_status(h) == 0
+    yr, hr = oracle.ssm_recurrence(synth.f64(inp["x"]), BC.cpu().double().numpy(), synth.f64(inp["dt"]),
+                                   synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), synth.f64(inp["D"]))
+    assert hp.max_rel(y.cpu().double().numpy(), yr) <= 2e-2
+    assert hp.max_rel(hf.cpu().double().numpy(), hr) <= 1e-2
+    sb.swimba_destroy(h)
+
+
+# -------------------------------------------------------------------------------- decode
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_decode_steps_match_oracle_and_forward(dtype):
+    cfg = cfg_of(dtype, B=5, L=40, H=4, P=64, N=128 if dtype == "bf16" else 32, E=8, k=2, F=128,
+                 h0_std=0.1)
+    inp = synth.make_inputs(cfg, seed=21)
+    B, L = cfg.B, cfg.L
+    h = hp.create_handle(cfg)
+    w, keep = hp.device_weights(inp)
+    state = hp.dev(inp["h0"]).clone()
+    ws = torch.empty(sb.swimba_decode_workspace_bytes(h, B), dtype=torch.uint8, device="cuda")
+    ys, idxs = [], []
+    for t in range(L):
+        u = hp.dev(inp["u"][:, t])
+        x = hp.dev(inp["x"][:, t])
+        dt = hp.dev(inp["dt"][:, t])
+        y = torch.empty_like(x)
+        idx = torch.empty(B, cfg.k, dtype=torch.int32, device="cuda")
+        wt = torch.empty(B, cfg.k, device="cuda")
+        sb.swimba_decode_step(h, w, u, x, dt, state, B, y, idx, wt, ws)
+        ys.append(y.cpu())
+        idxs.append(idx.cpu())
+    assert sb.swimba_status(h) == 0
+    y_dec = torch.stack(ys, 1)
+    idx_dec = torch.stack(idxs, 1)
+    ty, th = hp.tolerances(cfg)
+    # (a) against the oracle's decode loop == oracle forward (pinned on the CPU side)
+    fwd = hp.gpu_forward(cfg, inp)
+    res = hp.compare_forward(cfg, inp, dict(y=y_dec, h_final=state.cpu(), idx=idx_dec, w=fwd["w"]),
+                             ty, th)
+    # (b) against the library's own forward over the same L tokens
+    assert torch.equal(idx_dec, fwd["idx"])
+    assert hp.max_rel(y_dec.double().numpy(), fwd["y"].double().numpy()) <= ty
+    assert hp.max_rel(state.cpu().numpy(), fwd["h_final"].numpy()) <= th
+    sb.swimba_destroy(h)
+
+
+# ------------------------------------------------------------------- host-detected errors
+def test_host_side_errors_leave_outputs_untouched():
+    cfg = cfg_of("bf16", L=64)
+    inp = synth.make_inputs(cfg, seed=31)
+    B, L = cfg.B, cfg.L
+    h = hp.create_handle(cfg)
+    w, keep = hp.device_weights(inp)
+    u, x, dt = hp.dev(inp["u"]), hp.dev(inp["x"]), hp.dev(inp["dt"])
+    y = torch.full_like(x, 7.0)
+    ws = torch.empty(sb.swimba_workspace_bytes(h, B, L) + 64, dtype=torch.uint8, device="cuda")
+
+    def call(**kw):
+        a = dict(u=u, x=x, dt=dt, y=y, ws=ws, B=B, L=L)
+        a.update(kw)
+        return sb.swimba_forward(h, w, a["u"], a["x"], a["dt"], None, a["B"], a["L"], a["y"], None,
+                                 None, None, a["ws"], check=False)
+
+    assert call(u=None) == sb.ERR_NULL_ARG
+    assert call(y=None) == sb.ERR_NULL_ARG
+    assert call(ws=ws[:128]) == sb.ERR_WORKSPACE_TOO_SMALL
+    assert call(ws=ws[8:]) == sb.ERR_MISALIGNED
+    assert call(B=-1) == sb.ERR_UNSUPPORTED_SHAPE
+    assert "workspace" in sb.swimba_last_error(h) or sb.swimba_last_error(h) != ""
+    torch.cuda.synchronize()
+    assert torch.all(y == 7.0)
+    assert call() == 0 and sb.swimba_status(h) == 0
+    assert not torch.any(y == 7.0)
+    sb.swimba_destroy(h)
+    for bad in (dict(top_k=5), dict(chunk=100), dict(n_groups=3), dict(dtype=3), dict(n_experts=0),
+                dict(n_experts=65, top_k=1)):
+        args = dict(d_model=64, n_heads=4, head_dim=64, d_state=128, n_groups=1, n_experts=4,
+                    top_k=2, chunk=128, dtype=1)
+        args.update(bad)
+        with pytest.raises(sb.SwimbaError) as e:
+            sb.swimba_create(**args)
+        assert e.value.code == sb.ERR_BAD_CONFIG
+    with pytest.raises(sb.SwimbaError) as e:
+        sb.swimba_create(d_model=60, n_heads=4, head_dim=64, d_state=128, n_groups=1, n_experts=4,
+                         top_k=2, chunk=128, dtype=1)
+    assert e.value.code == sb.ERR_UNSUPPORTED_SHAPE
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    cfg = cfg_of("bf16", L=300)
+    inp = synth.make_inputs(cfg, seed=41)
+    B, L = cfg.B, cfg.L
+    dev_out = hp.gpu_forward(cfg, inp)
+    h = hp.create_handle(cfg)
+    w, keep = hp.device_weights(inp)
+    ws = torch.empty(sb.swimba_host_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    u, x, dt = inp["u"].pin_memory(), inp["x"].pin_memory(), inp["dt"].pin_memory()
+    y = torch.empty_like(x).pin_memory()
+    hf = torch.empty(B, cfg.H, cfg.P, cfg.N).pin_memory()
+    idx = torch.empty(B, L, cfg.k, dtype=torch.int32).pin_memory()
+    sb.swimba_forward_host(h, w, u, x, dt, B, L, y, hf, idx, None, ws)
+    assert sb.swimba_status(h) == 0
+    assert torch.equal(y.view(torch.int16), dev_out["y"].view(torch.int16))
+    assert torch.equal(hf, dev_out["h_final"])
+    assert torch.equal(idx, dev_out["idx"])
+    sb.swimba_destroy(h)
