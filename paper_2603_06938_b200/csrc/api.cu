@@ -32,8 +32,12 @@ int fail(swimba_handle *h, int code, const char *msg)
 
 // Workspace of the forward: [BC | idx | w], each 256-byte aligned.
 struct FwdLayout {
-    size_t bc, idx, w, total;
+    size_t bc, idx, w, gemm, total;
 };
+bool use_tensor_k1(const swimba_config &c)
+{
+    return c.dtype == SWIMBA_DTYPE_BF16 && expert_gemm_supported(c.d_model, 2 * c.n_groups * c.d_state);
+}
 FwdLayout fwd_layout(const swimba_config &c, int64_t T)
 {
     FwdLayout l;
@@ -42,6 +46,8 @@ FwdLayout fwd_layout(const swimba_config &c, int64_t T)
     l.bc = off;  off += align_up((size_t)T * S * elt_size(c.dtype));
     l.idx = off; off += align_up((size_t)T * c.top_k * sizeof(int32_t));
     l.w = off;   off += align_up((size_t)T * c.top_k * sizeof(float));
+    l.gemm = off;
+    if (use_tensor_k1(c)) off += align_up(expert_gemm_workspace_bytes(T, (int)S, c.n_experts, c.top_k));
     l.total = off;
     return l;
 }
@@ -110,15 +116,28 @@ int set_device(swimba_handle *h)
 
 // Router + projection + mix into BC (dtype, or fp32 when bc_fp32).
 int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *u,
-                  int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt)
+                  int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt, void *gemm_ws)
 {
     const swimba_config &c = h->cfg;
     const int S = 2 * c.n_groups * c.d_state;
     // With one expert the softmax is identically 1; the router kernel handles it without W_router
     // being dereferenced only if it is given, so substitute the expert matrix as a dummy operand.
     const void *Wr = w->W_router ? w->W_router : w->W_expert;
-    int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt);
+    const bool tensor = gemm_ws && !bc_fp32 && use_tensor_k1(c);
+    int *counts = nullptr;
+    if (tensor) {
+        counts = expert_gemm_counts(gemm_ws);
+        if (cudaMemsetAsync(counts, 0, sizeof(int) * SWIMBA_MAX_EXPERTS, ctx.stream) != cudaSuccess)
+            return fail(h, SWIMBA_ERR_CUDA, "clearing the expert histogram failed");
+    }
+    int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts);
     if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
+    if (tensor) {
+        rc = launch_expert_gemm(ctx, u, w->W_expert, idx, wt, T, c.d_model, S, c.n_experts, c.top_k,
+                                BC, gemm_ws);
+        if (rc != SWIMBA_OK) return fail(h, rc, "expert GEMM launch failed");
+        return SWIMBA_OK;
+    }
     rc = launch_project_mix_simt(ctx, c.dtype, u, w->W_expert, idx, wt, T, c.d_model, S,
                                  c.n_experts, c.top_k, BC, bc_fp32);
     if (rc != SWIMBA_OK) return fail(h, rc, "projection launch failed");
@@ -213,7 +232,7 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
     LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
-    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt);
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
     return rc;
@@ -267,7 +286,7 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
-    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt);
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
     if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
@@ -298,7 +317,7 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     float *BC = (float *)(ws + l.bc);
-    rc = run_route_mix(h, ctx, w, u, B, BC, true, idx, wt);
+    rc = run_route_mix(h, ctx, w, u, B, BC, true, idx, wt, nullptr);
     if (rc == SWIMBA_OK) {
         rc = launch_decode_update(ctx, c.dtype, x, BC, dt, w->A, w->dt_bias, w->D, state, B,
                                   c.n_heads, c.head_dim, c.d_state, c.n_groups, y);

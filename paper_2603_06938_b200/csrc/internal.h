@@ -6,7 +6,17 @@ namespace swimba {
 
 // K1a: router logits, softmax over all E, top-k (indices + un-renormalised weights).
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
-                  int E, int k, int32_t *idx, float *w);
+                  int E, int k, int32_t *idx, float *w, int *counts /* [E] histogram of selected experts, or NULL */);
+
+// K1b (tensor cores): grouped GEMM over tokens sorted by expert + slot sum.  `workspace` is sized by
+// expert_gemm_workspace_bytes; its first SWIMBA_MAX_EXPERTS ints are the histogram the router
+// fills (zeroed by the caller beforehand).
+size_t expert_gemm_workspace_bytes(int64_t T, int S, int E, int k);
+bool expert_gemm_supported(int F, int S);
+int *expert_gemm_counts(void *workspace);
+int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int32_t *idx,
+                       const float *w, int64_t T, int F, int S, int E, int k, void *BC,
+                       void *workspace);
 
 // K1b (SIMT): project the k selected experts and mix.  BC is written in `dtype`, or as float
 // per slot-sum when bc_fp32 is set.

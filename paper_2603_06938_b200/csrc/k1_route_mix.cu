@@ -11,7 +11,7 @@ namespace swimba {
 template <typename T, int EP>
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
-                   int k, int32_t *__restrict__ idx, float *__restrict__ w)
+                   int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts)
 {
     const int lane = threadIdx.x & 31;
     const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -61,18 +61,19 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
         if (lane == 0) {
             idx[t * k + j] = best;
             w[t * k + j] = bestp / z;
+            if (counts) atomicAdd(&counts[best], 1);
         }
     }
 }
 
 template <typename T>
 static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Ttok, int F, int E,
-                           int k, int32_t *idx, float *w)
+                           int k, int32_t *idx, float *w, int *counts)
 {
     const int warps = 8;
     dim3 grid((unsigned)ceil_div64(Ttok, warps)), block(warps * 32);
 #define SWIMBA_ROUTER_CASE(EPV)                                                              \
-    router_topk_kernel<T, EPV><<<grid, block, 0, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w)
+    router_topk_kernel<T, EPV><<<grid, block, 0, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, counts)
     if (E <= 1) SWIMBA_ROUTER_CASE(1);
     else if (E <= 2) SWIMBA_ROUTER_CASE(2);
     else if (E <= 4) SWIMBA_ROUTER_CASE(4);
@@ -86,13 +87,13 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
 }
 
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
-                  int E, int k, int32_t *idx, float *w)
+                  int E, int k, int32_t *idx, float *w, int *counts)
 {
     if (T <= 0) return SWIMBA_OK;
     if (dtype == SWIMBA_DTYPE_FP32)
-        return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w);
+        return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w, counts);
     return launch_router_t<__nv_bfloat16>(ctx, (const __nv_bfloat16 *)u,
-                                          (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w);
+                                          (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w, counts);
 }
 
 // One warp per (token, block of RW stream rows): BC[t, r] = sum_j w_j <W_e[e_j, r, :], u_t>.
