@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the Swimba token-mixer forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config small_lm] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path (router, top-k, expert projection, mix, SSD) over one
+batch of synthetic layer-shaped input.  Prints ONE JSON line on rank 0.  With N > 1 (torchrun)
+every rank runs an independent replica on its own batch: the path has no exchange step, so there
+is no collective on the data path (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch
+
+from paper_2603_06938_b200 import synth
+
+METRIC = "swimba_layer_fwd_tokens_per_s"
+UNIT = "tokens/s"
+NSETS = 4   # rotating input sets: together several times the 126 MB L2
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel from the ncu
+# captures summarised under profiles/; None until a capture of that kernel exists.
+NCU_TRAFFIC_BYTES = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return dict(sm_mhz=statistics.median(sm) if sm else None,
+                    sm_max_mhz=max(mx) if mx else None, reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+def algorithmic_work(cfg: synth.LayerConfig):
+    """Per-launch algorithmic work of each kernel for B x L tokens ('Roofline')."""
+    T, F, S, E, k = cfg.tokens, cfg.F, cfg.S, cfg.E, cfg.k
+    H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.Q
+    es = 2 if cfg.dtype == "bf16" else 4
+    w = {}
+    w["router_topk"] = dict(bound="hbm", work=T * F * es + E * F * es + T * k * 8)
+    w["expert_gemm"] = dict(bound="tensor", work=2.0 * T * k * F * S)
+    w["mix_slots"] = dict(bound="hbm", work=T * k * S * es + T * S * es)
+    w["project_mix_simt"] = dict(bound="alu", work=2.0 * T * k * F * S)
+    ssd_flops = float(T) * (Q * N * G + H * (Q * P + 4 * N * P))
+    ssd_bytes = T * (2 * H * P * es + S * es + H * 4) + cfg.B * H * P * N * 4
+    w["ssd_tiles"] = dict(bound="tensor", work=ssd_flops, bytes=ssd_bytes)
+    w["ssd_sequential"] = dict(bound="alu", work=4.0 * T * H * P * N, bytes=ssd_bytes)
+    w["scatter_rows"] = dict(bound="hbm", work=T * k * 8)
+    w["tile_table"] = dict(bound="hbm", work=E * 16)
+    w["segment_scan"] = dict(bound="hbm", work=0)
+    return w
+
+
+def roofline_entry(name, avg_ms, work, pk):
+    info = work.get(name)
+    if info is None or avg_ms <= 0:
+        return None
+    if info["bound"] == "hbm":
+        ach = info["work"] / (avg_ms * 1e-3) / 1e9
+        peak, unit = pk["hbm_gbs"], "GB/s"
+    elif info["bound"] == "tensor":
+        ach = info["work"] / (avg_ms * 1e-3) / 1e12
+        peak, unit = pk["bf16_tflops"], "TFLOP/s"
+    else:
+        # plain FP32 ALU work: 148 SMs x 128 FMA lanes x 2 flop x 1.965 GHz
+        ach = info["work"] / (avg_ms * 1e-3) / 1e12
+        peak, unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
+    return dict(kernel=name, bound=info["bound"], achieved=ach, peak=peak, unit=unit,
+                frac=ach / peak, traffic=NCU_TRAFFIC_BYTES.get(name),
+                peak_source=pk["source"], avg_ms=avg_ms)
+
+
+def time_oracle_sample(cfg: synth.LayerConfig, n_seq: int, seed: int = 0):
+    """The CPU oracle, as it stands, on n_seq whole sequences of the workload."""
+    import dataclasses
+    import oracle
+    sub = dataclasses.replace(cfg, B=n_seq)
+    inp = synth.make_inputs(sub, seed=seed)
+    args = [synth.f64(inp[n]) for n in ("u", "x", "dt", "W_r", "W_e", "A", "dt_bias", "D")]
+    t0 = time.perf_counter()
+    oracle.swimba_forward(*args, k=cfg.k, G=cfg.G)
+    dt = time.perf_counter() - t0
+    return dict(value=sub.tokens / dt, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
+                sample=f"{n_seq} of {cfg.B} sequences x {cfg.L} tokens of {cfg.name}, fp64, "
+                       f"{dt:.2f} s"), dt
+
+
+def run_reference(args, cfg, rank, world):
+    if rank != 0:
+        return
+    n_seq = 1
+    vals, times = [], []
+    for i in range(args.warmup + args.steps):
+        r, dt = time_oracle_sample(cfg, n_seq, seed=i)
+        if i >= args.warmup:
+            vals.append(r)
+            times.append(dt)
+    tok = n_seq * cfg.L
+    ms = 1e3 * sum(times) / len(times)
+    value = tok / (ms * 1e-3)
+    cb = dict(vals[-1])
+    cb["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(cfg, sample=f"{n_seq} sequence(s) per step"),
+        "cpu_baseline": cb,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def config_dict(cfg, **extra):
+    d = {"workload": f"{cfg.name}: B={cfg.B} L={cfg.L} d_model={cfg.F} H={cfg.H} P={cfg.P} "
+                     f"N={cfg.N} G={cfg.G} E={cfg.E} top_k={cfg.k} chunk={cfg.Q} {cfg.dtype}",
+         "tokens_per_step_per_gpu": cfg.tokens,
+         "l2_policy": f"inputs rotate over {NSETS} distinct sets (> L2) between timed steps"}
+    d.update(extra)
+    return d
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="small_lm", choices=[c for c in synth.CONFIG_ORDER if c != "decode"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = synth.CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+
+    from paper_2603_06938_b200 import binding as sb
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    pk = peaks()
+    dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
+    sets = [synth.make_inputs(cfg, seed=1000 * rank + i) for i in range(NSETS)]
+    wts = {n: sets[0][n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    dev_sets = [dict(u=s["u"].cuda(), x=s["x"].cuda(), dt=s["dt"].cuda()) for s in sets]
+    B, L = cfg.B, cfg.L
+    y = torch.empty_like(dev_sets[0]["x"])
+    hf = torch.empty(B, cfg.H, cfg.P, cfg.N, device="cuda")
+    ws = torch.empty(sb.swimba_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        s = dev_sets[i % NSETS]
+        sb.swimba_forward(h, w, s["u"], s["x"], s["dt"], None, B, L, y, hf, None, None, ws)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    launches_per_step = sb.swimba_last_launch_count(h)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.2)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    ms_step = ms_total / args.steps
+    value = world * cfg.tokens / (ms_step * 1e-3)
+
+    # per-kernel durations, live, same launch configuration (CUDA events around every kernel)
+    sb.swimba_profile(h, True)
+    per = {}
+    for i in range(args.steps):
+        step(i)
+        for name, ms in sb.swimba_profile_read(h):
+            per.setdefault(name, []).append(ms)
+    sb.swimba_profile(h, False)
+    clocks = sampler.stop() if rank == 0 else None
+
+    work = algorithmic_work(cfg)
+    tot = sum(sum(v) for v in per.values())
+    kernels = []
+    for name, v in per.items():
+        n_per_step = len(v) / args.steps
+        avg = sum(v) / len(v)
+        ent = roofline_entry(name, avg, work, pk) or dict(kernel=name, avg_ms=avg)
+        ent["share"] = sum(v) / tot if tot > 0 else 0.0
+        ent["launches_per_step"] = n_per_step
+        kernels.append(ent)
+    kernels.sort(key=lambda e: -e["share"])
+    dom = kernels[0] if kernels else None
+    roofline = None
+    if dom and "bound" in dom:
+        roofline = {k_: dom[k_] for k_ in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
+        roofline["kernel"] = dom["kernel"]
+        roofline["peak_source"] = "of " + pk["source"]
+
+    # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H in the timed region
+    hws = torch.empty(sb.swimba_host_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    host_sets = [dict(u=s["u"].pin_memory(), x=s["x"].pin_memory(), dt=s["dt"].pin_memory())
+                 for s in sets[:2]]
+    y_host = torch.empty_like(sets[0]["x"]).pin_memory()
+    for i in range(2):
+        s = host_sets[i % 2]
+        sb.swimba_forward_host(h, w, s["u"], s["x"], s["dt"], B, L, y_host, None, None, None, hws)
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        s = host_sets[i % 2]
+        sb.swimba_forward_host(h, w, s["u"], s["x"], s["dt"], B, L, y_host, None, None, None, hws)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    es = 2 if cfg.dtype == "bf16" else 4
+    h2d = cfg.tokens * (cfg.F * es + cfg.H * cfg.P * es + cfg.H * 4)
+    d2h = cfg.tokens * cfg.H * cfg.P * es
+    e2e = {"value": world * cfg.tokens / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    sb.swimba_destroy(h)
+    del dev_sets, hws, ws, y, hf
+
+    decode = None
+    if rank == 0 and world == 1 and not args.no_decode:
+        decode = bench_decode(sb, pk)
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu, _ = time_oracle_sample(cfg, min(cfg.B, 4))
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
+            "data": "synthetic", "config": config_dict(cfg), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
+            "kernels": kernels, "decode": decode, "cpu_baseline": cpu,
+        }
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
+    """Decode configuration: us/step over `steps` consecutive steps, against the HBM bytes of the
+    fp32 state read-modify-write."""
+    cfg = synth.CONFIGS["decode"]
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(4)
+    wt = synth.make_weights(cfg, gen)
+    wts = {n: v.cuda() for n, v in wt.items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    state = (0.1 * torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, generator=gen)).cuda()
+    toks = [{n: v.cuda() for n, v in synth.make_decode_step_inputs(cfg, gen).items()} for _ in range(8)]
+    y = torch.empty_like(toks[0]["x"])
+    ws = torch.empty(sb.swimba_decode_workspace_bytes(h, cfg.B), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        t = toks[i % len(toks)]
+        sb.swimba_decode_step(h, w, t["u"], t["x"], t["dt"], state, cfg.B, y, None, None, ws)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / steps
+    launches = sb.swimba_last_launch_count(h)
+    sb.swimba_profile(h, True)
+    per = {}
+    for i in range(32):
+        step(i)
+        for name, ms in sb.swimba_profile_read(h):
+            per.setdefault(name, []).append(ms)
+    sb.swimba_profile(h, False)
+    assert sb.swimba_status(h) == 0
+    state_bytes = 2 * cfg.B * cfg.H * cfg.P * cfg.N * 4
+    upd_us = 1e3 * sum(per.get("decode_update", [0])) / max(1, len(per.get("decode_update", [])))
+    out = {
+        "workload": f"decode: B={cfg.B} d_model={cfg.F} H={cfg.H} P={cfg.P} N={cfg.N} E={cfg.E} "
+                    f"top_k={cfg.k}, fp32 state {state_bytes // 2 / 1e6:.0f} MB (> L2)",
+        "us_per_step": us, "steps": steps, "launches_per_step": launches,
+        "tokens_per_s": cfg.B / (us * 1e-6),
+        "kernel_us": {n: 1e3 * sum(v) / len(v) for n, v in per.items()},
+        "roofline": {"kernel": "decode_update", "bound": "hbm",
+                     "achieved": state_bytes / (upd_us * 1e-6) / 1e9 if upd_us > 0 else None,
+                     "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": state_bytes / (upd_us * 1e-6) / 1e9 / pk["hbm_gbs"] if upd_us > 0 else None,
+                     "traffic": NCU_TRAFFIC_BYTES.get("decode_update"),
+                     "whole_step_frac": state_bytes / (us * 1e-6) / 1e9 / pk["hbm_gbs"]},
+    }
+    sb.swimba_destroy(h)
+    return out
+
+
+if __name__ == "__main__":
+    main()

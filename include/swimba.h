@@ -144,6 +144,16 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
                         float *topk_w_host, void *workspace, size_t workspace_bytes,
                         void *cuda_stream);
 
+/* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
+ * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
+ * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
+ * launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router, 2 tile table, 3 scatter,
+ * 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD tile
+ * kernel, 10 segment scan, 11 decode projection) and ms[i] its duration in milliseconds.
+ * Both arrays are HOST arrays. */
+int swimba_profile(swimba_handle *h, int enable);
+int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);
+
 /* Number of kernels the most recent forward/route_mix/ssd/decode call on this handle enqueued. */
 int swimba_last_launch_count(const swimba_handle *h);
 

@@ -30,7 +30,8 @@ DTYPE_BF16 = 1
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
-    "swimba_forward_host", "swimba_last_launch_count", "swimba_status", "swimba_last_error",
+    "swimba_forward_host", "swimba_profile", "swimba_profile_read",
+    "swimba_last_launch_count", "swimba_status", "swimba_last_error",
     "swimba_destroy",
 ]
 
@@ -86,6 +87,10 @@ def lib() -> ctypes.CDLL:
         L.swimba_forward_host.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, i32, i32,
                                           vp, vp, vp, vp, vp, sz, vp]
         L.swimba_forward_host.restype = ctypes.c_int
+        L.swimba_profile.argtypes = [vp, ctypes.c_int]
+        L.swimba_profile.restype = ctypes.c_int
+        L.swimba_profile_read.argtypes = [vp, vp, vp, i32]
+        L.swimba_profile_read.restype = ctypes.c_int
         L.swimba_last_launch_count.argtypes = [vp]
         L.swimba_last_launch_count.restype = ctypes.c_int
         L.swimba_status.argtypes = [vp]
@@ -221,6 +226,28 @@ def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B
     if check and rc != OK:
         h._raise(rc)
     return rc
+
+
+KERNEL_NAMES = {1: "router_topk", 2: "tile_table", 3: "scatter_rows", 4: "expert_gemm",
+                5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
+                9: "ssd_tiles", 10: "segment_scan", 11: "decode_project"}
+
+
+def swimba_profile(h: Handle, enable: bool) -> None:
+    rc = lib().swimba_profile(h.ptr, 1 if enable else 0)
+    if rc != OK:
+        h._raise(rc)
+
+
+def swimba_profile_read(h: Handle):
+    """[(kernel name, milliseconds)] of the kernels the most recent call launched."""
+    ids = (ctypes.c_int32 * 64)()
+    ms = (ctypes.c_float * 64)()
+    n = lib().swimba_profile_read(h.ptr, ctypes.cast(ids, ctypes.c_void_p),
+                                  ctypes.cast(ms, ctypes.c_void_p), 64)
+    if n < 0:
+        h._raise(n)
+    return [(KERNEL_NAMES.get(ids[i], str(ids[i])), float(ms[i])) for i in range(n)]
 
 
 def swimba_last_launch_count(h: Handle) -> int:

@@ -14,6 +14,7 @@ struct swimba_handle {
     int *d_status;          // device status word
     cudaStream_t last_stream;
     int last_launches;
+    Profiler prof;
     char err[256];
 };
 
@@ -229,7 +230,8 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
     if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
@@ -254,7 +256,8 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
         return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
     (void)workspace_bytes;
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    h->prof.n = 0;
     rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
@@ -282,7 +285,8 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
@@ -313,7 +317,8 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     const swimba_config &c = h->cfg;
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     float *BC = (float *)(ws + l.bc);
@@ -372,6 +377,32 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
     return SWIMBA_OK;
 }
 
+int swimba_profile(swimba_handle *h, int enable)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    if (enable && !h->prof.ev[0]) {
+        for (int i = 0; i < 2 * PROF_MAX; ++i)
+            if (cudaEventCreate(&h->prof.ev[i]) != cudaSuccess) return fail(h, SWIMBA_ERR_CUDA, "event creation failed");
+    }
+    h->prof.on = enable != 0;
+    h->prof.n = 0;
+    return SWIMBA_OK;
+}
+
+int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries)
+{
+    if (!h || !kernel_ids || !ms) return SWIMBA_ERR_NULL_ARG;
+    if (!h->prof.on) return 0;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return fail(h, SWIMBA_ERR_CUDA, "stream synchronisation failed");
+    int n = h->prof.n < max_entries ? h->prof.n : max_entries;
+    for (int i = 0; i < n; ++i) {
+        kernel_ids[i] = h->prof.stage[i];
+        if (cudaEventElapsedTime(&ms[i], h->prof.ev[2 * i], h->prof.ev[2 * i + 1]) != cudaSuccess)
+            return fail(h, SWIMBA_ERR_CUDA, "cudaEventElapsedTime failed");
+    }
+    return n;
+}
+
 int swimba_last_launch_count(const swimba_handle *h) { return h ? h->last_launches : 0; }
 
 int swimba_status(swimba_handle *h)
@@ -398,6 +429,8 @@ void swimba_destroy(swimba_handle *h)
 {
     if (!h) return;
     if (h->d_status) cudaFree(h->d_status);
+    if (h->prof.ev[0])
+        for (int i = 0; i < 2 * PROF_MAX; ++i) if (h->prof.ev[i]) cudaEventDestroy(h->prof.ev[i]);
     delete h;
 }
 

@@ -8,10 +8,39 @@
 
 namespace swimba {
 
+// Kernel ids reported by the optional per-kernel timing (swimba_profile_read).
+enum Stage {
+    STAGE_ROUTER = 1, STAGE_TILE_TABLE = 2, STAGE_SCATTER = 3, STAGE_EXPERT_GEMM = 4,
+    STAGE_MIX_SLOTS = 5, STAGE_PROJECT_SIMT = 6, STAGE_SSD_SEQUENTIAL = 7, STAGE_DECODE_UPDATE = 8,
+    STAGE_SSD_TILES = 9, STAGE_SEGMENT_SCAN = 10, STAGE_DECODE_PROJECT = 11,
+};
+
+constexpr int PROF_MAX = 64;
+struct Profiler {
+    bool on;
+    int n;
+    cudaEvent_t ev[2 * PROF_MAX];
+    int stage[PROF_MAX];
+};
+
 struct LaunchCtx {
     cudaStream_t stream;
     int *d_status;   // device status word (0 = ok, else a SWIMBA_ERR_* code)
     int launches;    // kernels enqueued through this context
+    Profiler *prof;  // optional CUDA-event bracket around every kernel
+    void begin(int stage) {
+        if (prof && prof->on && prof->n < PROF_MAX) {
+            prof->stage[prof->n] = stage;
+            cudaEventRecord(prof->ev[2 * prof->n], stream);
+        }
+    }
+    void end() {
+        if (prof && prof->on && prof->n < PROF_MAX) {
+            cudaEventRecord(prof->ev[2 * prof->n + 1], stream);
+            prof->n++;
+        }
+        launches++;
+    }
 };
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

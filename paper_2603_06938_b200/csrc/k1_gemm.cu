@@ -297,13 +297,15 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int
     const uint32_t box[3] = {(uint32_t)GM_BK, (uint32_t)BN, 1};
     if (!encode_tmap_bf16(&tmap, W_e, 3, dims, strides, box)) return SWIMBA_ERR_CUDA;
 
+    ctx.begin(STAGE_TILE_TABLE);
     tile_table_kernel<<<1, SWIMBA_MAX_EXPERTS, 0, ctx.stream>>>(counts, E, offsets, cursor, num_tiles,
                                                                tile_expert, tile_row0, tile_rows);
-    ctx.launches++;
+    ctx.end();
     const int64_t n_entries = T * k;
+    ctx.begin(STAGE_SCATTER);
     scatter_rows_kernel<<<(unsigned)ceil_div64(n_entries, 256), 256, 0, ctx.stream>>>(
         idx, n_entries, offsets, cursor, perm);
-    ctx.launches++;
+    ctx.end();
 
     const size_t smem = gemm_smem_bytes(BN);
     dim3 grid((unsigned)max_tiles, (unsigned)(S / BN));
@@ -317,19 +319,21 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int
                                                      num_tiles, tile_expert, tile_row0,         \
                                                      tile_rows, F, S, k, slots, ctx.d_status);  \
     } while (0)
+    ctx.begin(STAGE_EXPERT_GEMM);
     if (BN == 256) SWIMBA_GEMM_CASE(256);
     else if (BN == 128) SWIMBA_GEMM_CASE(128);
     else if (BN == 64) SWIMBA_GEMM_CASE(64);
     else SWIMBA_GEMM_CASE(32);
 #undef SWIMBA_GEMM_CASE
-    ctx.launches++;
+    ctx.end();
     if (k > 1) {
         const int64_t nvec = T * (S / 8);
         int64_t blocks = ceil_div64(nvec, 256);
         if (blocks > 148 * 16) blocks = 148 * 16;
+        ctx.begin(STAGE_MIX_SLOTS);
         mix_slots_kernel<<<(unsigned)blocks, 256, 0, ctx.stream>>>(slots, T, S, k,
                                                                   (__nv_bfloat16 *)BC);
-        ctx.launches++;
+        ctx.end();
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }

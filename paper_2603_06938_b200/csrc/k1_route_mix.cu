@@ -72,6 +72,7 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
 {
     const int warps = 8;
     dim3 grid((unsigned)ceil_div64(Ttok, warps)), block(warps * 32);
+    ctx.begin(STAGE_ROUTER);
 #define SWIMBA_ROUTER_CASE(EPV)                                                              \
     router_topk_kernel<T, EPV><<<grid, block, 0, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, counts)
     if (E <= 1) SWIMBA_ROUTER_CASE(1);
@@ -82,7 +83,7 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
     else if (E <= 32) SWIMBA_ROUTER_CASE(32);
     else SWIMBA_ROUTER_CASE(64);
 #undef SWIMBA_ROUTER_CASE
-    ctx.launches++;
+    ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
@@ -160,9 +161,10 @@ static int launch_pm(LaunchCtx &ctx, const void *u, const void *W_e, const int32
     const int warps = 8;
     const int64_t nw = T_ * ceil_div(S, RW);
     dim3 grid((unsigned)ceil_div64(nw, warps)), block(warps * 32);
+    ctx.begin(STAGE_PROJECT_SIMT);
     project_mix_simt_kernel<T, TO, RW><<<grid, block, 0, ctx.stream>>>(
         (const T *)u, (const T *)W_e, idx, w, T_, F, S, k, (TO *)BC);
-    ctx.launches++;
+    ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 

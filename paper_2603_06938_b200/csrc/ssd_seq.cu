@@ -109,9 +109,10 @@ static int launch_seq_t(LaunchCtx &ctx, const void *x, const void *BC, const flo
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
         return SWIMBA_ERR_CUDA;
+    ctx.begin(STAGE_SSD_SEQUENTIAL);
     kern<<<B * H, P * NS, smem, ctx.stream>>>((const T *)x, (const TBC *)BC, dt, A, dt_bias, D, h0,
                                              L, H, P, N, G, NS, (T *)y, h_final);
-    ctx.launches++;
+    ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
@@ -215,6 +216,7 @@ int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const float *
     int64_t blocks = ceil_div64(nwork, warps);
     const int64_t cap = (int64_t)sms * 8;
     if (blocks > cap) blocks = cap;
+    ctx.begin(STAGE_DECODE_UPDATE);
     if (dtype == SWIMBA_DTYPE_FP32)
         decode_update_kernel<float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
             (const float *)x, BC, dt, A, dt_bias, D, state, B, H, P, N, G, (float *)y);
@@ -222,7 +224,7 @@ int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const float *
         decode_update_kernel<__nv_bfloat16><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
             (const __nv_bfloat16 *)x, BC, dt, A, dt_bias, D, state, B, H, P, N, G,
             (__nv_bfloat16 *)y);
-    ctx.launches++;
+    ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
