@@ -107,7 +107,8 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
 
 /* First half of the forward only (router softmax equation, top-k rule, Theorem 1's mixed
  * streams): u[T,F] -> BC[T,S] dtype (Btilde then Ctilde), topk_idx[T,k], topk_w[T,k]
- * (either may be NULL).  The workspace is the one sized by swimba_workspace_bytes(h, 1, T). */
+ * (either may be NULL).  A workspace sized by swimba_workspace_bytes(h, B, L) for any B*L == T
+ * is large enough. */
 int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
                      void *BC, int32_t *topk_idx, float *topk_w, void *workspace,
                      size_t workspace_bytes, void *cuda_stream);

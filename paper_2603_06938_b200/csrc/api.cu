@@ -33,15 +33,16 @@ int fail(swimba_handle *h, int code, const char *msg)
 
 // Workspace of the forward: [BC | idx | w], each 256-byte aligned.
 struct FwdLayout {
-    size_t bc, idx, w, gemm, total;
+    size_t bc, idx, w, gemm, ssd, total;
 };
 bool use_tensor_k1(const swimba_config &c)
 {
     return c.dtype == SWIMBA_DTYPE_BF16 && expert_gemm_supported(c.d_model, 2 * c.n_groups * c.d_state);
 }
-FwdLayout fwd_layout(const swimba_config &c, int64_t T)
+FwdLayout fwd_layout(const swimba_config &c, int B, int L, int sm_count)
 {
     FwdLayout l;
+    const int64_t T = (int64_t)B * L;
     const size_t S = 2u * c.n_groups * c.d_state;
     size_t off = 0;
     l.bc = off;  off += align_up((size_t)T * S * elt_size(c.dtype));
@@ -49,6 +50,9 @@ FwdLayout fwd_layout(const swimba_config &c, int64_t T)
     l.w = off;   off += align_up((size_t)T * c.top_k * sizeof(float));
     l.gemm = off;
     if (use_tensor_k1(c)) off += align_up(expert_gemm_workspace_bytes(T, (int)S, c.n_experts, c.top_k));
+    l.ssd = off;
+    if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+        off += align_up(ssd_workspace_bytes(B, L, c.n_heads, c.chunk, sm_count));
     l.total = off;
     return l;
 }
@@ -73,7 +77,7 @@ DecLayout dec_layout(const swimba_config &c, int B)
 struct HostLayout {
     size_t u, x, dt, y, hf, idx, w, fwd, total;
 };
-HostLayout host_layout(const swimba_config &c, int B, int L)
+HostLayout host_layout(const swimba_config &c, int B, int L, int sm_count)
 {
     HostLayout l;
     const size_t T = (size_t)B * L, es = elt_size(c.dtype);
@@ -86,7 +90,7 @@ HostLayout host_layout(const swimba_config &c, int B, int L)
     l.hf = off;  off += align_up((size_t)B * HP * c.d_state * sizeof(float));
     l.idx = off; off += align_up(T * c.top_k * sizeof(int32_t));
     l.w = off;   off += align_up(T * c.top_k * sizeof(float));
-    l.fwd = off; off += fwd_layout(c, (int64_t)T).total;
+    l.fwd = off; off += fwd_layout(c, B, L, sm_count).total;
     l.total = off;
     return l;
 }
@@ -147,9 +151,15 @@ int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, con
 
 int run_ssd(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *x,
             const void *BC, const float *dt, const float *h0, int B, int L, void *y,
-            float *h_final)
+            float *h_final, void *ssd_ws)
 {
     const swimba_config &c = h->cfg;
+    if (ssd_ws && ssd_tiles_supported(c.dtype, c.head_dim, c.d_state)) {
+        int rc = launch_ssd_tiles(ctx, x, BC, dt, w->A, w->dt_bias, w->D, h0, B, L, c.n_heads,
+                                  c.n_groups, c.chunk, h->sm_count, y, h_final, ssd_ws);
+        if (rc != SWIMBA_OK) return fail(h, rc, "SSD tile kernel launch failed");
+        return SWIMBA_OK;
+    }
     int rc = launch_ssd_sequential(ctx, c.dtype, x, BC, false, dt, w->A, w->dt_bias, w->D, h0, B, L,
                                    c.n_heads, c.head_dim, c.d_state, c.n_groups, y, h_final);
     if (rc != SWIMBA_OK) return fail(h, rc, "SSD launch failed");
@@ -198,7 +208,7 @@ int swimba_create(const swimba_config *cfg, swimba_handle **out)
 size_t swimba_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
 {
     if (!h || B <= 0 || L <= 0) return 0;
-    return fwd_layout(h->cfg, (int64_t)B * L).total;
+    return fwd_layout(h->cfg, B, L, h->sm_count).total;
 }
 
 size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B)
@@ -210,7 +220,7 @@ size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B)
 size_t swimba_host_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
 {
     if (!h || B <= 0 || L <= 0) return 0;
-    return host_layout(h->cfg, B, L).total;
+    return host_layout(h->cfg, B, L, h->sm_count).total;
 }
 
 int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
@@ -226,8 +236,8 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
     if (!u || !BC || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC or workspace is NULL");
     if (!aligned16(u) || !aligned16(BC) || !aligned16(workspace) || !aligned16(topk_idx) || !aligned16(topk_w))
         return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
-    const FwdLayout l = fwd_layout(h->cfg, T);
-    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    const FwdLayout l = fwd_layout(h->cfg, 1, (int)T, h->sm_count);
+    if (workspace_bytes < l.ssd) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     char *ws = (char *)workspace;
     LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
@@ -254,11 +264,12 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
     if (!aligned16(x) || !aligned16(BC) || !aligned16(y) || !aligned16(dt) || !aligned16(h0) ||
         !aligned16(h_final) || !aligned16(workspace))
         return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
-    (void)workspace_bytes;
+    const FwdLayout l = fwd_layout(h->cfg, B, L, h->sm_count);
+    if (!workspace || workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
     h->prof.n = 0;
-    rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
+    rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final, (char *)workspace + l.ssd);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
     return rc;
@@ -281,7 +292,7 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
         !aligned16(h_final) || !aligned16(topk_idx) || !aligned16(topk_w) || !aligned16(workspace))
         return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
     const int64_t T = (int64_t)B * L;
-    const FwdLayout l = fwd_layout(h->cfg, T);
+    const FwdLayout l = fwd_layout(h->cfg, B, L, h->sm_count);
     if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     char *ws = (char *)workspace;
@@ -291,7 +302,7 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
     rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
-    if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final);
+    if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final, ws + l.ssd);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
     return rc;
@@ -347,7 +358,7 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
         return fail(h, SWIMBA_ERR_NULL_ARG, "u_host, x_host, y_host or workspace is NULL");
     if (!aligned16(workspace)) return fail(h, SWIMBA_ERR_MISALIGNED, "workspace must be 16-byte aligned");
     const swimba_config &c = h->cfg;
-    const HostLayout l = host_layout(c, B, L);
+    const HostLayout l = host_layout(c, B, L, h->sm_count);
     if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     int rc = check_weights(h, w, true);
     if (rc != SWIMBA_OK) return rc;

@@ -24,6 +24,13 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
                             const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
                             int k, void *BC, bool bc_fp32);
 
+// K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
+bool ssd_tiles_supported(int dtype, int P, int N);
+size_t ssd_workspace_bytes(int B, int L, int H, int chunk, int sm_count);
+int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                     const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
+                     int chunk, int sm_count, void *y, float *h_final, void *workspace);
+
 // Per-timestep SIMT evaluation of the recurrence (fp32 state in registers).
 int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
                           const float *dt, const float *A, const float *dt_bias, const float *D,
