@@ -145,6 +145,26 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
                         float *topk_w_host, void *workspace, size_t workspace_bytes,
                         void *cuda_stream);
 
+/* Allocation-free variant of swimba_route_mix (the paper has no counterpart: this is a
+ * packaging convenience).  For callers that cannot allocate device memory where they call the
+ * library -- a plug-in that is handed only its input and output buffers, a serving process whose
+ * memory pool is fully handed out, set-up code that runs before any allocator exists -- the
+ * scratch of the routing/projection stage lives in a fixed array inside the library image instead
+ * of a caller-provided workspace.  Same arguments and results as swimba_route_mix, minus the
+ * workspace.
+ *   - The array is SWIMBA_STATIC_SCRATCH_BYTES large and is held by every GPU that loads the
+ *     library until the process exits.  Token counts whose scratch need exceeds it are rejected
+ *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (with bf16, S = 256
+ *     and k = 2 the limit is a little under 8000 tokens per call).
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.  No call allocates or frees device memory.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents (the
+ *     entry point clears the part that must start at zero).  Two calls that overlap on the GPU,
+ *     e.g. on different streams, race on it: serialise them. */
+#define SWIMBA_STATIC_SCRATCH_BYTES (8 * 1024 * 1024)
+int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
+                            void *BC, int32_t *topk_idx, float *topk_w, void *cuda_stream);
+
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call

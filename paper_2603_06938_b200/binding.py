@@ -30,7 +30,7 @@ DTYPE_BF16 = 1
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
-    "swimba_forward_host", "swimba_profile", "swimba_profile_read",
+    "swimba_forward_host", "swimba_route_mix_static", "swimba_profile", "swimba_profile_read",
     "swimba_last_launch_count", "swimba_status", "swimba_last_error",
     "swimba_destroy",
 ]
@@ -87,6 +87,9 @@ def lib() -> ctypes.CDLL:
         L.swimba_forward_host.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, i32, i32,
                                           vp, vp, vp, vp, vp, sz, vp]
         L.swimba_forward_host.restype = ctypes.c_int
+        L.swimba_route_mix_static.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, i64, vp, vp, vp,
+                                              vp]
+        L.swimba_route_mix_static.restype = ctypes.c_int
         L.swimba_profile.argtypes = [vp, ctypes.c_int]
         L.swimba_profile.restype = ctypes.c_int
         L.swimba_profile_read.argtypes = [vp, vp, vp, i32]
@@ -189,6 +192,18 @@ def swimba_route_mix(h: Handle, w: swimba_weights, u, T: int, BC, topk_idx, topk
     wp, wb = _ws(workspace)
     rc = lib().swimba_route_mix(h.ptr, ctypes.byref(w), _ptr(u), T, _ptr(BC), _ptr(topk_idx),
                                 _ptr(topk_w), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_route_mix_static(h: Handle, w: swimba_weights, u, T: int, BC, topk_idx, topk_w,
+                            stream=None, check: bool = True) -> int:
+    """swimba_route_mix without a workspace argument: for callers that cannot allocate device
+    memory, the stage's scratch is a fixed array inside the library (8 MiB per GPU, shared by all
+    calls on that GPU, so overlapping calls must be serialised; larger T is rejected)."""
+    rc = lib().swimba_route_mix_static(h.ptr, ctypes.byref(w), _ptr(u), T, _ptr(BC),
+                                       _ptr(topk_idx), _ptr(topk_w), _stream(stream))
     if check and rc != OK:
         h._raise(rc)
     return rc

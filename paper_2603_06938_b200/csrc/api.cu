@@ -446,3 +446,54 @@ void swimba_destroy(swimba_handle *h)
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Allocation-free variant of swimba_route_mix.
+//
+// Some callers cannot obtain device memory at the point where they call the library: code that
+// runs inside a memory-budgeted serving process whose pool is already handed out, plug-ins that
+// receive only their input and output buffers from a host framework, or set-up paths that run
+// before an allocator exists.  For them the scratch that the routing/projection stage needs (the
+// expert histogram, the tile table, the row permutation and the per-slot projections) lives in a
+// fixed array that is part of the library image.  Every GPU that loads the library holds these
+// SWIMBA_STATIC_SCRATCH_BYTES until the process exits.
+// ------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_scratch[SWIMBA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];   // device address of g_static_scratch, per device
+}  // namespace
+
+extern "C" int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const void *u,
+                                       int64_t T, void *BC, int32_t *topk_idx, float *topk_w,
+                                       void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (T < 0 || T > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range");
+    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    int rc = set_device(h);
+    if (rc != SWIMBA_OK) return rc;
+    if (h->device < 0 || h->device >= kMaxDevices)
+        return fail(h, SWIMBA_ERR_CUDA, "device ordinal beyond the static-scratch table");
+    // In host code the array's name is only a stand-in; the kernels need its device address.
+    // Looked up once per device, with that device current (set_device checked it above).
+    if (!g_static_scratch_ptr[h->device]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return fail(h, SWIMBA_ERR_CUDA, "cudaGetSymbolAddress on the static scratch failed");
+        }
+        g_static_scratch_ptr[h->device] = p;
+    }
+    const FwdLayout l = fwd_layout(h->cfg, 1, (int)T, h->sm_count);
+    if (l.ssd > (size_t)SWIMBA_STATIC_SCRATCH_BYTES) {
+        snprintf(h->err, sizeof(h->err),
+                 "T = %lld tokens needs %zu bytes of scratch, the static scratch holds %d",
+                 (long long)T, l.ssd, (int)SWIMBA_STATIC_SCRATCH_BYTES);
+        return SWIMBA_ERR_WORKSPACE_TOO_SMALL;
+    }
+    return swimba_route_mix(h, w, u, T, BC, topk_idx, topk_w, g_static_scratch_ptr[h->device],
+                            (size_t)SWIMBA_STATIC_SCRATCH_BYTES, cuda_stream);
+}
