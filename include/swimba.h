@@ -154,8 +154,8 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
  * workspace.
  *   - The array is SWIMBA_STATIC_SCRATCH_BYTES large and is held by every GPU that loads the
  *     library until the process exits.  Token counts whose scratch need exceeds it are rejected
- *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (with bf16, S = 256
- *     and k = 2 the limit is a little under 8000 tokens per call).
+ *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (with bf16, S = 256,
+ *     E = 8 and k = 2 the limit is about 5000 tokens per call).
  *   - The first call on each device looks up the array's device address; make that first call
  *     outside any stream capture.  No call allocates or frees device memory.
  *   - All calls on a device share the one array, and it keeps the previous call's contents (the
@@ -168,9 +168,9 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router, 2 tile table, 3 scatter,
- * 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD tile
- * kernel, 10 segment scan, 11 decode projection) and ms[i] its duration in milliseconds.
+ * launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router + grouping by
+ * expert, 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
+ * tile kernel, 10 segment scan; 2, 3 and 11 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);

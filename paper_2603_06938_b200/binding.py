@@ -243,9 +243,9 @@ def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B
     return rc
 
 
-KERNEL_NAMES = {1: "router_topk", 2: "tile_table", 3: "scatter_rows", 4: "expert_gemm",
+KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
-                9: "ssd_tiles", 10: "segment_scan", 11: "decode_project"}
+                9: "ssd_tiles", 10: "segment_scan"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

@@ -57,9 +57,9 @@ FwdLayout fwd_layout(const swimba_config &c, int B, int L, int sm_count)
     return l;
 }
 
-// Workspace of a decode step: [BC fp32 | idx | w].
+// Workspace of a decode step: [BC (bf16 on the tensor-core path, else fp32) | idx | w | GEMM scratch].
 struct DecLayout {
-    size_t bc, idx, w, total;
+    size_t bc, idx, w, gemm, total;
 };
 DecLayout dec_layout(const swimba_config &c, int B)
 {
@@ -69,6 +69,8 @@ DecLayout dec_layout(const swimba_config &c, int B)
     l.bc = off;  off += align_up((size_t)B * S * sizeof(float));
     l.idx = off; off += align_up((size_t)B * c.top_k * sizeof(int32_t));
     l.w = off;   off += align_up((size_t)B * c.top_k * sizeof(float));
+    l.gemm = off;
+    if (use_tensor_k1(c)) off += align_up(expert_gemm_workspace_bytes(B, (int)S, c.n_experts, c.top_k));
     l.total = off;
     return l;
 }
@@ -129,17 +131,19 @@ int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, con
     // being dereferenced only if it is given, so substitute the expert matrix as a dummy operand.
     const void *Wr = w->W_router ? w->W_router : w->W_expert;
     const bool tensor = gemm_ws && !bc_fp32 && use_tensor_k1(c);
-    int *counts = nullptr;
+    int *counts = nullptr, *perm = nullptr;
     if (tensor) {
         counts = expert_gemm_counts(gemm_ws);
+        perm = expert_gemm_perm(gemm_ws);
         if (cudaMemsetAsync(counts, 0, sizeof(int) * SWIMBA_MAX_EXPERTS, ctx.stream) != cudaSuccess)
             return fail(h, SWIMBA_ERR_CUDA, "clearing the expert histogram failed");
     }
-    int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts);
+    int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts,
+                           perm, T, h->sm_count);
     if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
     if (tensor) {
-        rc = launch_expert_gemm(ctx, u, w->W_expert, idx, wt, T, c.d_model, S, c.n_experts, c.top_k,
-                                BC, gemm_ws);
+        rc = launch_expert_gemm(ctx, u, w->W_expert, wt, T, c.d_model, S, c.n_experts, c.top_k,
+                                h->sm_count, BC, gemm_ws);
         if (rc != SWIMBA_OK) return fail(h, rc, "expert GEMM launch failed");
         return SWIMBA_OK;
     }
@@ -332,11 +336,12 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
     h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
-    float *BC = (float *)(ws + l.bc);
-    rc = run_route_mix(h, ctx, w, u, B, BC, true, idx, wt, nullptr);
+    void *BC = ws + l.bc;
+    const bool tensor = use_tensor_k1(c);   // bf16 streams from the grouped GEMM, else fp32 from SIMT
+    rc = run_route_mix(h, ctx, w, u, B, BC, !tensor, idx, wt, tensor ? ws + l.gemm : nullptr);
     if (rc == SWIMBA_OK) {
-        rc = launch_decode_update(ctx, c.dtype, x, BC, dt, w->A, w->dt_bias, w->D, state, B,
-                                  c.n_heads, c.head_dim, c.d_state, c.n_groups, y);
+        rc = launch_decode_update(ctx, c.dtype, x, BC, !tensor, dt, w->A, w->dt_bias, w->D, state, B,
+                                  c.n_heads, c.head_dim, c.d_state, c.n_groups, h->sm_count, y);
         if (rc != SWIMBA_OK) fail(h, rc, "decode launch failed");
     }
     h->last_stream = ctx.stream;

@@ -5,18 +5,21 @@
 namespace swimba {
 
 // K1a: router logits, softmax over all E, top-k (indices + un-renormalised weights).
+// When counts is given (zeroed beforehand) the (token, slot) pairs are also grouped by expert:
+// perm[e * cap + i], i < counts[e], lists the entries t*k + j routed to expert e.
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
-                  int E, int k, int32_t *idx, float *w, int *counts /* [E] histogram of selected experts, or NULL */);
+                  int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
+                  int sm_count);
 
-// K1b (tensor cores): grouped GEMM over tokens sorted by expert + slot sum.  `workspace` is sized by
-// expert_gemm_workspace_bytes; its first SWIMBA_MAX_EXPERTS ints are the histogram the router
-// fills (zeroed by the caller beforehand).
+// K1b (tensor cores): grouped GEMM over the per-expert lists + slot sum.  `workspace` is sized
+// by expert_gemm_workspace_bytes and holds the histogram (zeroed by the caller before the
+// router runs), the per-expert lists (capacity T each) and the per-slot projections.
 size_t expert_gemm_workspace_bytes(int64_t T, int S, int E, int k);
 bool expert_gemm_supported(int F, int S);
 int *expert_gemm_counts(void *workspace);
-int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int32_t *idx,
-                       const float *w, int64_t T, int F, int S, int E, int k, void *BC,
-                       void *workspace);
+int *expert_gemm_perm(void *workspace);
+int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const float *w, int64_t T,
+                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace);
 
 // K1b (SIMT): project the k selected experts and mix.  BC is written in `dtype`, or as float
 // per slot-sum when bc_fp32 is set.
@@ -38,8 +41,9 @@ int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *
                           float *h_final);
 
 // K4: one-token state update, state[B,H,P,N] in place.
-int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const float *BC,
+// BC [B,S] is fp32 when bc_fp32, else bf16.
+int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
                          const float *dt, const float *A, const float *dt_bias, const float *D,
-                         float *state, int B, int H, int P, int N, int G, void *y);
+                         float *state, int B, int H, int P, int N, int G, int sm_count, void *y);
 
 }  // namespace swimba

@@ -20,68 +20,28 @@ constexpr int GM_THREADS = 192;
 }  // namespace
 
 // ------------------------------------------------------------------------------------------
-// Grouping: counts[e] were accumulated by the router kernel.
-// ------------------------------------------------------------------------------------------
-__global__ void tile_table_kernel(const int *__restrict__ counts, int E, int *__restrict__ offsets,
-                                  int *__restrict__ cursor, int *__restrict__ num_tiles,
-                                  int *__restrict__ tile_expert, int *__restrict__ tile_row0,
-                                  int *__restrict__ tile_rows)
-{
-    __shared__ int s_cnt[SWIMBA_MAX_EXPERTS], s_off[SWIMBA_MAX_EXPERTS], s_tb[SWIMBA_MAX_EXPERTS];
-    const int e = threadIdx.x;
-    s_cnt[e] = (e < E) ? counts[e] : 0;
-    __syncthreads();
-    if (e == 0) {
-        int off = 0, tb = 0;
-        for (int i = 0; i < E; ++i) {
-            s_off[i] = off;
-            s_tb[i] = tb;
-            off += s_cnt[i];
-            tb += ceil_div(s_cnt[i], GM_BM);
-        }
-        *num_tiles = tb;
-    }
-    __syncthreads();
-    if (e < E) {
-        offsets[e] = s_off[e];
-        cursor[e] = 0;
-        const int nt = ceil_div(s_cnt[e], GM_BM);
-        for (int i = 0; i < nt; ++i) {
-            tile_expert[s_tb[e] + i] = e;
-            tile_row0[s_tb[e] + i] = s_off[e] + i * GM_BM;
-            tile_rows[s_tb[e] + i] = min(GM_BM, s_cnt[e] - i * GM_BM);
-        }
-    }
-}
-
-// perm[offsets[e] + position] = t*k + j for every (token, slot) routed to expert e.  The order
-// inside an expert's segment is arbitrary; every output row is computed independently of its
-// position, so results do not depend on it.
-__global__ void scatter_rows_kernel(const int32_t *__restrict__ idx, int64_t n_entries,
-                                    const int *__restrict__ offsets, int *__restrict__ cursor,
-                                    int *__restrict__ perm)
-{
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n_entries) return;
-    const int e = idx[i];
-    const int pos = atomicAdd(&cursor[e], 1);
-    perm[offsets[e] + pos] = (int)i;
-}
-
-// ------------------------------------------------------------------------------------------
 // Grouped GEMM.  Warps 0-3: gather the A rows with cp.async, later the epilogue; warp 4: TMA
 // loads of the weight tile; warp 5: TMEM allocation and MMA issue.
 // ------------------------------------------------------------------------------------------
 template <int BN>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat16 *__restrict__ u,
-                   const int *__restrict__ perm, const float *__restrict__ w_slot,
-                   const int *__restrict__ num_tiles, const int *__restrict__ tile_expert,
-                   const int *__restrict__ tile_row0, const int *__restrict__ tile_rows, int F,
-                   int S, int k, __nv_bfloat16 *__restrict__ out, int *d_status)
+                   const int *__restrict__ perm, int64_t cap, const float *__restrict__ w_slot,
+                   const int *__restrict__ counts, int E, int F, int S, int k,
+                   __nv_bfloat16 *__restrict__ out, int *d_status)
 {
-    const int tile = blockIdx.x;
-    if (tile >= *num_tiles) return;
+    // Tile -> (expert, rows): tiles are numbered expert by expert, ceil(counts[e] / 128) each.
+    int e = 0, row0 = (int)blockIdx.x, cnt = 0;
+    for (; e < E; ++e) {
+        cnt = counts[e];
+        const int nt = (cnt + GM_BM - 1) / GM_BM;
+        if (row0 < nt) break;
+        row0 -= nt;
+    }
+    if (e == E) return;
+    row0 *= GM_BM;
+    const int nrows = min(GM_BM, cnt - row0);
+    perm += (int64_t)e * cap;
     const int n0 = blockIdx.y * BN;
     constexpr uint32_t A_BYTES = GM_BM * 128, B_BYTES = BN * 128;
     constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
@@ -100,7 +60,6 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     float *row_w = (float *)(row_dst + GM_BM);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int e = tile_expert[tile], row0 = tile_row0[tile], nrows = tile_rows[tile];
 
     if (tid == 0) {
         for (int s = 0; s < GM_STAGES; ++s) {
@@ -250,17 +209,21 @@ static size_t gemm_smem_bytes(int BN)
            GM_BM * 12 + 64;
 }
 
+// Workspace: [counts: 64 ints] [perm: E lists of capacity T] [slot outputs T*k*S bf16 when k > 1].
+static size_t gemm_ws_up(size_t v) { return (v + 255) / 256 * 256; }
+
 size_t expert_gemm_workspace_bytes(int64_t T, int S, int E, int k)
 {
-    const size_t a = 256;
-    auto up = [&](size_t v) { return (v + a - 1) / a * a; };
-    const size_t max_tiles = (size_t)ceil_div64(T * k, GM_BM) + E;
-    size_t tot = 0;
-    tot += up(4 * SWIMBA_MAX_EXPERTS * sizeof(int));        // counts, cursor, offsets, num_tiles
-    tot += 3 * up(max_tiles * sizeof(int));                 // tile table
-    tot += up((size_t)T * k * sizeof(int));                 // perm
-    if (k > 1) tot += up((size_t)T * k * S * sizeof(__nv_bfloat16));   // slot outputs
+    size_t tot = gemm_ws_up(SWIMBA_MAX_EXPERTS * sizeof(int));
+    tot += gemm_ws_up((size_t)E * T * sizeof(int));
+    if (k > 1) tot += gemm_ws_up((size_t)T * k * S * sizeof(__nv_bfloat16));
     return tot;
+}
+
+int *expert_gemm_counts(void *workspace) { return (int *)workspace; }
+int *expert_gemm_perm(void *workspace)
+{
+    return (int *)((char *)workspace + gemm_ws_up(SWIMBA_MAX_EXPERTS * sizeof(int)));
 }
 
 bool expert_gemm_supported(int F, int S)
@@ -268,44 +231,28 @@ bool expert_gemm_supported(int F, int S)
     return S % 32 == 0 && F >= 64;
 }
 
-int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int32_t *idx,
-                       const float *w, int64_t T, int F, int S, int E, int k, void *BC,
-                       void *workspace)
+int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const float *w, int64_t T,
+                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace)
 {
     if (T <= 0) return SWIMBA_OK;
-    const size_t a = 256;
-    auto up = [&](size_t v) { return (v + a - 1) / a * a; };
     const int max_tiles = (int)ceil_div64(T * k, GM_BM) + E;
-    char *p = (char *)workspace;
-    int *counts = (int *)p;
-    int *cursor = counts + SWIMBA_MAX_EXPERTS;
-    int *offsets = cursor + SWIMBA_MAX_EXPERTS;
-    int *num_tiles = offsets + SWIMBA_MAX_EXPERTS;
-    p += up(4 * SWIMBA_MAX_EXPERTS * sizeof(int));
-    int *tile_expert = (int *)p; p += up((size_t)max_tiles * sizeof(int));
-    int *tile_row0 = (int *)p;   p += up((size_t)max_tiles * sizeof(int));
-    int *tile_rows = (int *)p;   p += up((size_t)max_tiles * sizeof(int));
-    int *perm = (int *)p;        p += up((size_t)T * k * sizeof(int));
-    __nv_bfloat16 *slots = (k > 1) ? (__nv_bfloat16 *)p : (__nv_bfloat16 *)BC;
+    int *counts = expert_gemm_counts(workspace);
+    int *perm = expert_gemm_perm(workspace);
+    __nv_bfloat16 *slots = (k > 1)
+        ? (__nv_bfloat16 *)((char *)perm + gemm_ws_up((size_t)E * T * sizeof(int)))
+        : (__nv_bfloat16 *)BC;
 
+    // Widest column tile that divides S; narrower when there are too few row tiles to fill the
+    // GPU (decode-sized calls), so that the weight rows are spread over more SMs.
     int BN = 32;
     for (int c : {256, 128, 64}) if (S % c == 0) { BN = c; break; }
+    while (BN > 32 && (int64_t)max_tiles * (S / BN) < sm_count) BN >>= 1;
 
     CUtensorMap tmap;
     const uint64_t dims[3] = {(uint64_t)F, (uint64_t)S, (uint64_t)E};
     const uint64_t strides[2] = {(uint64_t)F * 2, (uint64_t)S * F * 2};
     const uint32_t box[3] = {(uint32_t)GM_BK, (uint32_t)BN, 1};
     if (!encode_tmap_bf16(&tmap, W_e, 3, dims, strides, box)) return SWIMBA_ERR_CUDA;
-
-    ctx.begin(STAGE_TILE_TABLE);
-    tile_table_kernel<<<1, SWIMBA_MAX_EXPERTS, 0, ctx.stream>>>(counts, E, offsets, cursor, num_tiles,
-                                                               tile_expert, tile_row0, tile_rows);
-    ctx.end();
-    const int64_t n_entries = T * k;
-    ctx.begin(STAGE_SCATTER);
-    scatter_rows_kernel<<<(unsigned)ceil_div64(n_entries, 256), 256, 0, ctx.stream>>>(
-        idx, n_entries, offsets, cursor, perm);
-    ctx.end();
 
     const size_t smem = gemm_smem_bytes(BN);
     dim3 grid((unsigned)max_tiles, (unsigned)(S / BN));
@@ -315,9 +262,8 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != \
             cudaSuccess)                                                                        \
             return SWIMBA_ERR_CUDA;                                                             \
-        kern<<<grid, GM_THREADS, smem, ctx.stream>>>(tmap, (const __nv_bfloat16 *)u, perm, w,     \
-                                                     num_tiles, tile_expert, tile_row0,         \
-                                                     tile_rows, F, S, k, slots, ctx.d_status);  \
+        kern<<<grid, GM_THREADS, smem, ctx.stream>>>(tmap, (const __nv_bfloat16 *)u, perm, T, w,  \
+                                                     counts, E, F, S, k, slots, ctx.d_status);  \
     } while (0)
     ctx.begin(STAGE_EXPERT_GEMM);
     if (BN == 256) SWIMBA_GEMM_CASE(256);
@@ -329,7 +275,7 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int
     if (k > 1) {
         const int64_t nvec = T * (S / 8);
         int64_t blocks = ceil_div64(nvec, 256);
-        if (blocks > 148 * 16) blocks = 148 * 16;
+        if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;
         ctx.begin(STAGE_MIX_SLOTS);
         mix_slots_kernel<<<(unsigned)blocks, 256, 0, ctx.stream>>>(slots, T, S, k,
                                                                   (__nv_bfloat16 *)BC);
@@ -337,7 +283,5 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const int
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
-
-int *expert_gemm_counts(void *workspace) { return (int *)workspace; }
 
 }  // namespace swimba

@@ -4,97 +4,238 @@
 
 namespace swimba {
 
-// One warp per token.  Logit summation order (fixed, so results are reproducible run to run):
-// lane l accumulates features f = 256*c + 8*l + i (c ascending, i = 0..7) with fused
-// multiply-adds, then the 32 partial sums are combined by an xor butterfly (16,8,4,2,1).
-// bf16 products are exact in fp32, so the only rounding is in the additions.
-template <typename T, int EP>
+// Router: a block handles chunks of `chunk` consecutive tokens, one warp TPW tokens at a time;
+// the router matrix is staged in shared memory once per block (when it fits) so that every token
+// costs one pass over its own features.
+//
+// Logit summation order (fixed, so results are reproducible run to run): lane l accumulates
+// features f = 256*c + 8*l + i (c ascending, i = 0..7) with fused multiply-adds; the 32 partial
+// sums of each (token, expert) are then combined by a halving butterfly over lane distances
+// 16, 8, 4, 2, 1 in which each step also halves the number of values a lane still carries, so
+// that afterwards every lane owns the complete logit of one (token, expert) pair (or of V/32
+// adjacent experts when V = TPW*EP exceeds 32).  bf16 products are exact in fp32, so the only
+// rounding is in the additions.  Softmax and top-k then run across the lanes of a token's group.
+//
+// Grouping by expert is done here as well: entry (t, j) goes to its expert's list,
+// perm[e * cap + pos] = t*k + j.  Positions are handed out per chunk: a shared-memory histogram
+// gives every entry its rank inside the chunk, one global atomic per (chunk, expert) on counts[e]
+// (zeroed by the caller) reserves the chunk's range.  The order inside a list is arbitrary; every
+// output row is computed independently of its position, so results do not depend on it.
+constexpr int ROUTER_MAX_CHUNK = 512;
+
+template <typename T, int EP, int TPW>
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
-                   int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts)
+                   int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts,
+                   int *__restrict__ perm, int64_t cap, int stage_w, int chunk)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (t >= Ttok) return;
-    float g[EP];
+    constexpr int V = TPW * EP;                 // values per lane before the butterfly
+    constexpr int R = V > 32 ? V / 32 : 1;      // values per lane after it (adjacent experts)
+    constexpr int DUP = V >= 32 ? 1 : 32 / V;   // lanes holding the same value after it
+    constexpr int GW = 32 / TPW;                // lanes per token group
+    static_assert(V >= 2 && (V & (V - 1)) == 0 && R <= EP, "unsupported router shape");
+    extern __shared__ __align__(16) unsigned char router_smem[];
+    __shared__ int s_cnt[SWIMBA_MAX_EXPERTS], s_base[SWIMBA_MAX_EXPERTS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+    int *s_ent = reinterpret_cast<int *>(router_smem);              // [chunk * k] expert | rank << 8
+    const T *Wsrc = W_r;
+    if (stage_w) {
+        T *sW = reinterpret_cast<T *>(router_smem + (size_t)ROUTER_MAX_CHUNK * SWIMBA_MAX_TOPK * sizeof(int));
+        const int nvec = (int)(((int64_t)E * F * sizeof(T)) >> 4);
+        const uint4 *src = reinterpret_cast<const uint4 *>(W_r);
+        uint4 *dst = reinterpret_cast<uint4 *>(sW);
+        for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = src[i];
+        Wsrc = sW;
+    }
+    // after the butterfly this lane owns experts e0 .. e0+R-1 of token q_own of the pass
+    const int q_own = lane / GW;
+    const int e0 = ((lane % GW) / DUP) * R;
+    const int64_t nchunks = ceil_div64(Ttok, chunk);
+    for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const int64_t tbeg = c * chunk;
+        const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
+        if (threadIdx.x < SWIMBA_MAX_EXPERTS) s_cnt[threadIdx.x] = 0;
+        __syncthreads();
+        for (int64_t t0 = tbeg + warp * TPW; t0 < tend; t0 += nwarp * TPW) {
+            float g[V];                                  // g[q * EP + e]
 #pragma unroll
-    for (int e = 0; e < EP; ++e) g[e] = 0.f;
-    const T *urow = u + t * F;
-    for (int f = lane * 8; f < F; f += 256) {
-        float uv[8];
-        load8(urow + f, uv);
+            for (int i = 0; i < V; ++i) g[i] = 0.f;
+#pragma unroll 2
+            for (int f = lane * 8; f < F; f += 256) {
+                float uv[TPW][8];
 #pragma unroll
-        for (int e = 0; e < EP; ++e) {
-            if (e < E) {
-                float wv[8];
-                load8(W_r + (int64_t)e * F + f, wv);
+                for (int q = 0; q < TPW; ++q) {
+                    const int64_t t = (t0 + q < tend) ? t0 + q : t0;
+                    load8(u + t * F + f, uv[q]);
+                }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) g[e] = fmaf(wv[i], uv[i], g[e]);
+                for (int e = 0; e < EP; ++e) {
+                    if (e < E) {
+                        float wv[8];
+                        load8(Wsrc + (int64_t)e * F + f, wv);
+#pragma unroll
+                        for (int q = 0; q < TPW; ++q)
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                g[q * EP + e] = fmaf(wv[i], uv[q][i], g[q * EP + e]);
+                    }
+                }
+            }
+            // halving butterfly: V values on 32 lanes -> R values on this lane
+            {
+                int n = V;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    if (n > R) {
+                        n >>= 1;
+                        const bool up = (lane & o) != 0;
+#pragma unroll
+                        for (int i = 0; i < V / 2; ++i) {
+                            if (i < n) {
+                                const float send = up ? g[i] : g[i + n];
+                                const float keep = up ? g[i + n] : g[i];
+                                g[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < R; ++i) g[i] += __shfl_xor_sync(0xffffffffu, g[i], o);
+                    }
+                }
+            }
+            // softmax over ALL experts of the token (padding experts count as -inf)
+            float gv[R], pv[R];
+            float m = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                gv[i] = (e0 + i < E) ? g[i] : -INFINITY;
+                m = fmaxf(m, gv[i]);
+            }
+#pragma unroll
+            for (int o = GW / 2; o >= DUP; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            float z = 0.f;
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                pv[i] = expf(gv[i] - m);
+                z += pv[i];
+            }
+#pragma unroll
+            for (int o = GW / 2; o >= DUP; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+            // k rounds of "largest remaining logit, lowest index on ties"; weights are NOT
+            // renormalised
+            const int64_t t = t0 + q_own;
+            for (int j = 0; j < k; ++j) {
+                float bg = gv[0], bp = pv[0];
+                int be = e0;
+#pragma unroll
+                for (int i = 1; i < R; ++i)
+                    if (gv[i] > bg) { bg = gv[i]; bp = pv[i]; be = e0 + i; }
+#pragma unroll
+                for (int o = GW / 2; o >= DUP; o >>= 1) {
+                    const float og = __shfl_xor_sync(0xffffffffu, bg, o);
+                    const float op = __shfl_xor_sync(0xffffffffu, bp, o);
+                    const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+                    if (og > bg || (og == bg && oe < be)) { bg = og; bp = op; be = oe; }
+                }
+#pragma unroll
+                for (int i = 0; i < R; ++i) if (e0 + i == be) gv[i] = -INFINITY;
+                if (lane % GW == 0 && t < tend) {
+                    idx[t * k + j] = be;
+                    w[t * k + j] = bp / z;
+                    if (counts) {
+                        const int rank = atomicAdd(&s_cnt[be], 1);
+                        s_ent[(int)(t - tbeg) * k + j] = be | (rank << 8);
+                    }
+                }
             }
         }
-    }
-#pragma unroll
-    for (int e = 0; e < EP; ++e) g[e] = warp_sum(g[e]);
-    // softmax over ALL experts, ascending expert order
-    float m = g[0];
-#pragma unroll
-    for (int e = 1; e < EP; ++e) if (e < E) m = fmaxf(m, g[e]);
-    float z = 0.f;
-    float p[EP];
-#pragma unroll
-    for (int e = 0; e < EP; ++e) {
-        p[e] = (e < E) ? expf(g[e] - m) : 0.f;
-        z += p[e];
-    }
-    // k rounds of "largest remaining logit, lowest index on ties"; weights are NOT renormalised
-    unsigned long long taken = 0ull;
-    for (int j = 0; j < k; ++j) {
-        int best = -1;
-        float bestg = 0.f, bestp = 0.f;
-#pragma unroll
-        for (int e = 0; e < EP; ++e) {
-            if (e < E && !((taken >> e) & 1ull) && (best < 0 || g[e] > bestg)) {
-                best = e; bestg = g[e]; bestp = p[e];
+        if (counts) {
+            __syncthreads();
+            if (threadIdx.x < E) s_base[threadIdx.x] = atomicAdd(&counts[threadIdx.x], s_cnt[threadIdx.x]);
+            __syncthreads();
+            const int n_ent = (int)(tend - tbeg) * k;
+            for (int i = threadIdx.x; i < n_ent; i += blockDim.x) {
+                const int ent = s_ent[i], e = ent & 255;
+                perm[(int64_t)e * cap + s_base[e] + (ent >> 8)] = (int)(tbeg * k + i);
             }
         }
-        taken |= 1ull << best;
-        if (lane == 0) {
-            idx[t * k + j] = best;
-            w[t * k + j] = bestp / z;
-            if (counts) atomicAdd(&counts[best], 1);
-        }
+        __syncthreads();
     }
+}
+
+// One expert: the softmax is identically 1 and every token is routed to expert 0.
+__global__ void __launch_bounds__(256)
+router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__restrict__ w,
+                            int *__restrict__ counts, int *__restrict__ perm)
+{
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < Ttok;
+         t += (int64_t)gridDim.x * blockDim.x) {
+        idx[t] = 0;
+        w[t] = 1.f;
+        if (counts) perm[t] = (int)t;
+    }
+    if (counts && blockIdx.x == 0 && threadIdx.x == 0) counts[0] = (int)Ttok;
 }
 
 template <typename T>
 static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Ttok, int F, int E,
-                           int k, int32_t *idx, float *w, int *counts)
+                           int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
+                           int sm_count)
 {
     const int warps = 8;
-    dim3 grid((unsigned)ceil_div64(Ttok, warps)), block(warps * 32);
+    if (E == 1) {
+        int64_t blocks = ceil_div64(Ttok, 256);
+        if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
+        ctx.begin(STAGE_ROUTER);
+        router_single_expert_kernel<<<(unsigned)blocks, 256, 0, ctx.stream>>>(Ttok, idx, w, counts, perm);
+        ctx.end();
+        return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+    }
+    const size_t w_bytes = (size_t)E * F * sizeof(T);
+    const int stage_w = (w_bytes <= 64 * 1024 && (w_bytes & 15) == 0) ? 1 : 0;
+    const size_t smem = (size_t)ROUTER_MAX_CHUNK * SWIMBA_MAX_TOPK * sizeof(int) + (stage_w ? w_bytes : 0);
+    // chunk: enough chunks to give every SM two blocks, between 32 and ROUTER_MAX_CHUNK tokens
+    int chunk = (int)(Ttok / (2 * (int64_t)sm_count));
+    chunk = (chunk + 31) / 32 * 32;
+    if (chunk < 32) chunk = 32;
+    if (chunk > ROUTER_MAX_CHUNK) chunk = ROUTER_MAX_CHUNK;
     ctx.begin(STAGE_ROUTER);
-#define SWIMBA_ROUTER_CASE(EPV)                                                              \
-    router_topk_kernel<T, EPV><<<grid, block, 0, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, counts)
-    if (E <= 1) SWIMBA_ROUTER_CASE(1);
-    else if (E <= 2) SWIMBA_ROUTER_CASE(2);
-    else if (E <= 4) SWIMBA_ROUTER_CASE(4);
-    else if (E <= 8) SWIMBA_ROUTER_CASE(8);
-    else if (E <= 16) SWIMBA_ROUTER_CASE(16);
-    else if (E <= 32) SWIMBA_ROUTER_CASE(32);
-    else SWIMBA_ROUTER_CASE(64);
+#define SWIMBA_ROUTER_CASE(EPV, TPWV)                                                          \
+    do {                                                                                       \
+        auto kern = router_topk_kernel<T, EPV, TPWV>;                                          \
+        if (smem > 32 * 1024 &&  /* static shared memory counts toward the 48 KB default */    \
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
+                                 (int)smem) != cudaSuccess)                                    \
+            return SWIMBA_ERR_CUDA;                                                            \
+        int64_t blocks = ceil_div64(Ttok, chunk);                                              \
+        const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);             \
+        if (blocks > cap_blocks) blocks = cap_blocks;                                          \
+        kern<<<(unsigned)blocks, warps * 32, smem, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, \
+                                                                 counts, perm, cap, stage_w,   \
+                                                                 chunk);                       \
+    } while (0)
+    if (E <= 2) SWIMBA_ROUTER_CASE(2, 8);
+    else if (E <= 4) SWIMBA_ROUTER_CASE(4, 8);
+    else if (E <= 8) SWIMBA_ROUTER_CASE(8, 4);
+    else if (E <= 16) SWIMBA_ROUTER_CASE(16, 2);
+    else if (E <= 32) SWIMBA_ROUTER_CASE(32, 1);
+    else SWIMBA_ROUTER_CASE(64, 1);
 #undef SWIMBA_ROUTER_CASE
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
-                  int E, int k, int32_t *idx, float *w, int *counts)
+                  int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
+                  int sm_count)
 {
     if (T <= 0) return SWIMBA_OK;
     if (dtype == SWIMBA_DTYPE_FP32)
-        return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w, counts);
+        return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w,
+                                      counts, perm, cap, sm_count);
     return launch_router_t<__nv_bfloat16>(ctx, (const __nv_bfloat16 *)u,
-                                          (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w, counts);
+                                          (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w, counts,
+                                          perm, cap, sm_count);
 }
 
 // One warp per (token, block of RW stream rows): BC[t, r] = sum_j w_j <W_e[e_j, r, :], u_t>.

@@ -136,9 +136,20 @@ int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *
 // ------------------------------------------------------------------------------------------
 constexpr int DEC_ROWS = 4;
 
-template <typename T>
+__device__ __forceinline__ float4 load_bc4(const float *p, int v)
+{
+    return reinterpret_cast<const float4 *>(p)[v];
+}
+__device__ __forceinline__ float4 load_bc4(const __nv_bfloat16 *p, int v)
+{
+    const uint2 raw = reinterpret_cast<const uint2 *>(p)[v];
+    return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                       __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+}
+
+template <typename T, typename TBC>
 __global__ void __launch_bounds__(256)
-decode_update_kernel(const T *__restrict__ x, const float *__restrict__ BC,
+decode_update_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
                      const float *__restrict__ dt, const float *__restrict__ A,
                      const float *__restrict__ dt_bias, const float *__restrict__ D,
                      float *__restrict__ state, int B, int H, int P, int N, int G,
@@ -149,7 +160,7 @@ decode_update_kernel(const T *__restrict__ x, const float *__restrict__ BC,
     const int pgroups = ceil_div(P, DEC_ROWS);
     const int64_t nwork = (int64_t)B * H * pgroups;
     const int64_t nwarps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int nv = N >> 2;   // float4 per row
+    const int nv = N >> 2;   // groups of 4 state entries per row
     for (int64_t wk = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); wk < nwork;
          wk += nwarps) {
         const int pg = (int)(wk % pgroups);
@@ -159,8 +170,8 @@ decode_update_kernel(const T *__restrict__ x, const float *__restrict__ BC,
         const float delta = softplus_f((dt ? dt[bh] : 0.f) + dt_bias[h]);
         const float a = expf(delta * A[h]);
         const float Dh = D ? D[h] : 0.f;
-        const float4 *Bv = reinterpret_cast<const float4 *>(BC + (int64_t)b * S + g * N);
-        const float4 *Cv = reinterpret_cast<const float4 *>(BC + (int64_t)b * S + (G + g) * N);
+        const TBC *Bp = BC + (int64_t)b * S + g * N;
+        const TBC *Cp = BC + (int64_t)b * S + (G + g) * N;
         float xv[DEC_ROWS], acc[DEC_ROWS];
 #pragma unroll
         for (int r = 0; r < DEC_ROWS; ++r) {
@@ -176,7 +187,7 @@ decode_update_kernel(const T *__restrict__ x, const float *__restrict__ BC,
                 if (p < P)
                     s[r] = __ldcs(reinterpret_cast<const float4 *>(state + (bh * P + p) * N) + v);
             }
-            const float4 bb = Bv[v], cc = Cv[v];
+            const float4 bb = load_bc4(Bp, v), cc = load_bc4(Cp, v);
 #pragma unroll
             for (int r = 0; r < DEC_ROWS; ++r) {
                 const int p = pg * DEC_ROWS + r;
@@ -203,27 +214,28 @@ decode_update_kernel(const T *__restrict__ x, const float *__restrict__ BC,
     }
 }
 
-int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const float *BC,
+int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
                          const float *dt, const float *A, const float *dt_bias, const float *D,
-                         float *state, int B, int H, int P, int N, int G, void *y)
+                         float *state, int B, int H, int P, int N, int G, int sm_count, void *y)
 {
     if (B <= 0) return SWIMBA_OK;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int64_t nwork = (int64_t)B * H * ceil_div(P, DEC_ROWS);
     const int warps = 8;
     int64_t blocks = ceil_div64(nwork, warps);
-    const int64_t cap = (int64_t)sms * 8;
+    const int64_t cap = (int64_t)sm_count * 8;
     if (blocks > cap) blocks = cap;
     ctx.begin(STAGE_DECODE_UPDATE);
     if (dtype == SWIMBA_DTYPE_FP32)
-        decode_update_kernel<float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
-            (const float *)x, BC, dt, A, dt_bias, D, state, B, H, P, N, G, (float *)y);
-    else
-        decode_update_kernel<__nv_bfloat16><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
-            (const __nv_bfloat16 *)x, BC, dt, A, dt_bias, D, state, B, H, P, N, G,
+        decode_update_kernel<float, float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
+            (const float *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N, G, (float *)y);
+    else if (bc_fp32)
+        decode_update_kernel<__nv_bfloat16, float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
+            (const __nv_bfloat16 *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N, G,
             (__nv_bfloat16 *)y);
+    else
+        decode_update_kernel<__nv_bfloat16, __nv_bfloat16><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
+            (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)BC, dt, A, dt_bias, D, state, B, H, P, N,
+            G, (__nv_bfloat16 *)y);
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }

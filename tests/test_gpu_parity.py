@@ -49,6 +49,9 @@ CASES = [
     cfg_of("fp32", L=150, N=16, P=64, H=3, F=48),
     cfg_of("fp32", L=97, N=32, P=16, H=2, G=2, E=3, k=2, F=24),
     cfg_of("fp32", L=64, N=128, P=64, H=2, E=5, k=5, F=72),
+    cfg_of("bf16", L=130, B=1, H=2, F=2048, E=8, k=2),     # router matrix of 32 KB in shared memory
+    cfg_of("bf16", L=150, B=1, H=2, F=1024, E=64, k=8),    # router matrix too large to stage
+    cfg_of("bf16", L=2100, B=1, H=2, F=256, E=16, k=2),    # several router chunks per block
 ]
 
 
