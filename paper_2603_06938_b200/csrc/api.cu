@@ -52,7 +52,7 @@ FwdLayout fwd_layout(const swimba_config &c, int B, int L, int sm_count)
     if (use_tensor_k1(c)) off += align_up(expert_gemm_workspace_bytes(T, (int)S, c.n_experts, c.top_k));
     l.ssd = off;
     if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
-        off += align_up(ssd_workspace_bytes(B, L, c.n_heads, c.chunk, sm_count));
+        off += align_up(ssd_workspace_bytes(B, L, c.n_heads, c.n_groups, c.chunk, sm_count));
     l.total = off;
     return l;
 }

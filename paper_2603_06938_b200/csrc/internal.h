@@ -29,7 +29,7 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
 
 // K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
 bool ssd_tiles_supported(int dtype, int P, int N);
-size_t ssd_workspace_bytes(int B, int L, int H, int chunk, int sm_count);
+size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
                      const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
                      int chunk, int sm_count, void *y, float *h_final, void *workspace);

@@ -3,16 +3,28 @@
 // chunks; the recurrence itself is Theorem 1's h_t = a_t h_{t-1} + Delta_t Btilde_t x_t^T,
 // y_t = Ctilde_t^T h_t + D x_t).
 //
-// One CTA owns one (sequence, head, segment) and walks its segment in tiles of 128 tokens.  With
-// l_i = sum_{r<=i} Delta_r A (inside the tile), for every tile:
-//   G      = Ctilde Btilde^T                                  [128 x 128]   (MMA 1)
-//   M[i,s] = G[i,s] exp(l_i - l_s) Delta_s  for s <= i, else 0               (CUDA cores -> TMEM)
-//   Ydiag  = M X                                              [128 x 64]    (MMA 2, A from TMEM)
-//   Yoff   = Ctilde H_prev^T                                  [128 x 64]    (MMA 3)
-//   y_i    = Ydiag_i + exp(l_i) Yoff_i + D x_i
-//   dH^T   = Btilde^T (w . X),  w_s = exp(l_last - l_s) Delta_s   [128 x 64] (MMA 4)
-//   H      = exp(l_last) H_prev + dH                                         (fp32, registers)
+// One CTA owns one (sequence, pair of heads of one B/C group, segment) and walks its segment in
+// tiles of 128 tokens.  With l_i = sum_{r<=i} Delta_r A (inside the tile), per tile:
+//   G      = Ctilde Btilde^T                      [128 x 128]  (MMA 1, once for both heads)
+// and for each of the two heads
+//   Y      = Ctilde H_prev^T                      [128 x 64]   (MMA 3), then scaled in place by
+//            exp(l_i) on the CUDA cores
+//   M[i,s] = G[i,s] exp(l_i - l_s) Delta_s  for s <= i, else 0      (CUDA cores -> TMEM, bf16)
+//   Y     += M X                                               (MMA 2, A operand from TMEM)
+//   y_i    = Y_i + D x_i
+//   dH^T   = Btilde^T (w . X),  w_s = exp(l_last - l_s) Delta_s  [128 x 64]  (MMA 4)
+//   H      = exp(l_last) H_prev + dH                           (fp32, registers)
 // The carried state never leaves the SM inside a segment: the inter-chunk recurrence is fused.
+// The two heads run on two compute warpgroups with their own MMA-issuing warps, so that one
+// head's tensor-core and memory latencies are covered by the other head's CUDA-core work.
+//
+// The decay mask needs exp(l_i - l_s) for every kept (i, s).  Only the four 32x32 blocks on the
+// diagonal evaluate it entry by entry.  A block strictly below the diagonal (rows in block w,
+// columns in block b < w) factors as
+//   exp(l_i - L_w) * exp(L_w - L_{b+1}) * exp(L_{b+1} - l_s),     L_w = l at the end of block w-1,
+// every exponent being <= 0 (no overflow, underflow only where the true value underflows), so
+// that it costs two multiplications per entry.
+//
 // Long sequences with few (sequence, head) pairs are cut into segments: a first pass of this
 // kernel computes every segment's local end state (MMA 4 only), segment_scan_kernel (K3) chains
 // them, and a second pass evaluates each segment from its true incoming state.
@@ -25,14 +37,23 @@ namespace {
 constexpr int ST = 128;                 // tokens per tile
 constexpr int SP = 64;                  // head dim this kernel is built for
 constexpr int SN = 128;                 // state size this kernel is built for
-constexpr int SSD_THREADS = 192;        // warps 0-3 compute, warp 4 TMA, warp 5 MMA
-constexpr int SSD_STAGES = 2;
+constexpr int NHD = 2;                  // heads per CTA
+// warps 0-3: head 0 compute, 4-7: head 1 compute, 8: TMA, 9: MMA issuer head 0 (+ MMA 1),
+// 10: MMA issuer head 1
+constexpr int SSD_THREADS = 128 * NHD + 32 * (1 + NHD);
+constexpr int WARP_TMA = 4 * NHD, WARP_MMA0 = 4 * NHD + 1;
 constexpr uint32_t SLAB = 16384;        // 128 rows x 128 bytes
-constexpr uint32_t STAGE_BYTES = 5 * SLAB;   // C (2 slabs), B (2 slabs), X (1 slab)
 constexpr float LOG2E = 1.4426950408889634f;
 
-// TMEM columns
-constexpr uint32_t TM_G = 0, TM_M = 128, TM_YD = 192, TM_YOFF = 256, TM_DH = 320, TM_COLS = 512;
+// shared memory map (bytes from the 1024-aligned base)
+constexpr uint32_t SM_CB = 0;                        // C0 C1 B0 B1 slabs (single stage)
+constexpr uint32_t SM_HEAD = 4 * SLAB;               // per head: X[2] XP HB
+constexpr uint32_t SM_HEAD_BYTES = 4 * SLAB;
+constexpr uint32_t SM_SMALL = SM_HEAD + NHD * SM_HEAD_BYTES;
+
+// TMEM columns: G, then per head M (bf16 A operand), Y, dH
+constexpr uint32_t TM_G = 0, TM_HEAD = 128, TM_HEAD_COLS = 192, TM_COLS = 512;
+constexpr uint32_t TM_M = 0, TM_Y = 64, TM_DH = 128;
 
 enum { MODE_FULL = 0, MODE_STATE_ONLY = 1 };
 
@@ -48,138 +69,198 @@ struct SsdParams {
     int *d_status;
 };
 
-struct __align__(8) SsdBars {
-    uint64_t load_full[SSD_STAGES], load_empty[SSD_STAGES];
-    uint64_t g_full, m_full, yd_full, yoff_full, dh_full, h_ready;
+struct __align__(8) HeadBars {
+    uint64_t x_full[2], x_free[2];
+    uint64_t yoff_full, m_full, yd_full, xp_full, dh_full, h_ready, y_free;
 };
+struct __align__(8) SsdBars {
+    uint64_t cb_full, cb_empty, g_full, g_free;
+    HeadBars hd[NHD];
+};
+
+struct __align__(16) SsdSmall {
+    float cs[NHD][ST];       // log2(Delta_s) - l_s          (diagonal blocks)
+    float cb[NHD][ST];       // Delta_s exp(L_{b(s)+1} - l_s) (blocks below the diagonal)
+    float scan[NHD][4];      // per-warp totals of the log-decay
+    SsdBars bars;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+// pairs of heads never straddle a B/C group
+__host__ __device__ inline int pairs_per_group(int H, int G) { return (H / G + NHD - 1) / NHD; }
 }  // namespace
 
 __global__ void __launch_bounds__(SSD_THREADS, 1)
 ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
                  const SsdParams prm)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *s_stage = smem;                                  // SSD_STAGES x (C0 C1 B0 B1 X)
-    uint8_t *s_xp = smem + SSD_STAGES * STAGE_BYTES;          // w . X      (MN-major B operand)
-    uint8_t *s_hb = s_xp + SLAB;                              // bf16 state (MN-major B operand)
-    float *s_cs = (float *)(s_hb + SLAB);                     // [128] log2(Delta_s) - l2_s
-    float *s_scan = s_cs + ST;                                // [8] warp totals
-    SsdBars *bars = (SsdBars *)(s_scan + 8);
-    uint32_t *tmem_slot = (uint32_t *)(bars + 1);
-    int *abort_flag = (int *)(tmem_slot + 1);
+    extern __shared__ __align__(1024) uint8_t smem[];
+    SsdSmall *sm = (SsdSmall *)(smem + SM_SMALL);
+    SsdBars *bars = &sm->bars;
+    int *abort_flag = &sm->abort_flag;
+    int *d_status = prm.d_status;
+    if ((tc::smem_u32(smem) & 1023u) != 0) {      // the swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
+        return;
+    }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int g = h / (prm.H / prm.G);
+    const int seg = blockIdx.x, b = blockIdx.z;
     const int L = prm.L, H = prm.H;
+    const int HG = H / prm.G, ppg = pairs_per_group(H, prm.G);
+    const int g = blockIdx.y / ppg, pr = blockIdx.y % ppg;
+    const int head0 = g * HG + pr * NHD;
+    const int nh = min(NHD, HG - pr * NHD);          // heads this CTA really has
     const int t_begin = seg * prm.seg_len;
     const int t_end = min(L, t_begin + prm.seg_len);
     const int ntiles = (t_end - t_begin + ST - 1) / ST;
     const bool full = prm.mode == MODE_FULL;
-    int *d_status = prm.d_status;
 
     if (tid == 0) {
-        for (int s = 0; s < SSD_STAGES; ++s) {
-            tc::mbar_init(&bars->load_full[s], 1);
-            tc::mbar_init(&bars->load_empty[s], 1);
-        }
+        tc::mbar_init(&bars->cb_full, 1);
+        tc::mbar_init(&bars->cb_empty, nh);
         tc::mbar_init(&bars->g_full, 1);
-        tc::mbar_init(&bars->m_full, 128);
-        tc::mbar_init(&bars->yd_full, 1);
-        tc::mbar_init(&bars->yoff_full, 1);
-        tc::mbar_init(&bars->dh_full, 1);
-        tc::mbar_init(&bars->h_ready, 128);
+        tc::mbar_init(&bars->g_free, 128 * nh);
+        for (int hd = 0; hd < NHD; ++hd) {
+            HeadBars *hb = &bars->hd[hd];
+            for (int s = 0; s < 2; ++s) {
+                tc::mbar_init(&hb->x_full[s], 1);
+                tc::mbar_init(&hb->x_free[s], 129);
+            }
+            tc::mbar_init(&hb->yoff_full, 1);
+            tc::mbar_init(&hb->m_full, 128);
+            tc::mbar_init(&hb->yd_full, 1);
+            tc::mbar_init(&hb->xp_full, 128);
+            tc::mbar_init(&hb->dh_full, 1);
+            tc::mbar_init(&hb->h_ready, 128);
+            tc::mbar_init(&hb->y_free, 128);
+        }
         *abort_flag = 0;
         tc::fence_mbar_init();
     }
-    if (warp == 5) {
-        tc::tmem_alloc(tmem_slot, TM_COLS);
+    if (warp == WARP_MMA0) {
+        tc::tmem_alloc(&sm->tmem_slot, TM_COLS);
         tc::tmem_relinquish();
     }
-    if (warp == 4 && lane == 0) {
+    if (warp == WARP_TMA && lane == 0) {
         tc::prefetch_tmap(&tmap_bc);
         tc::prefetch_tmap(&tmap_x);
     }
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
+    const uint32_t tmem = sm->tmem_slot;
 
-    if (warp == 4) {
+    if (warp == WARP_TMA) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
+            for (int hd = 0; hd < nh; ++hd) {               // X of tile 0
+                HeadBars *hb = &bars->hd[hd];
+                tc::mbar_arrive_expect_tx(&hb->x_full[0], SLAB);
+                tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES, &tmap_x, &hb->x_full[0], 0,
+                                head0 + hd, t_begin, b);
+            }
             for (int j = 0; j < ntiles; ++j) {
-                const int st = j % SSD_STAGES;
-                tc::mbar_wait(&bars->load_empty[st], ((j / SSD_STAGES) & 1) ^ 1, abort_flag, d_status);
-                uint8_t *base = s_stage + st * STAGE_BYTES;
                 const int t0 = t_begin + j * ST;
-                tc::mbar_arrive_expect_tx(&bars->load_full[st], full ? STAGE_BYTES : 3 * SLAB);
+                tc::mbar_wait(&bars->cb_empty, (j & 1) ^ 1, abort_flag, d_status);
+                tc::mbar_arrive_expect_tx(&bars->cb_full, full ? 4 * SLAB : 2 * SLAB);
                 if (full) {
-                    tc::tma_load_3d(base + 0 * SLAB, &tmap_bc, &bars->load_full[st], (prm.G + g) * SN, t0, b);
-                    tc::tma_load_3d(base + 1 * SLAB, &tmap_bc, &bars->load_full[st], (prm.G + g) * SN + 64, t0, b);
+                    tc::tma_load_3d(smem + SM_CB + 0 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN, t0, b);
+                    tc::tma_load_3d(smem + SM_CB + 1 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN + 64, t0, b);
                 }
-                tc::tma_load_3d(base + 2 * SLAB, &tmap_bc, &bars->load_full[st], g * SN, t0, b);
-                tc::tma_load_3d(base + 3 * SLAB, &tmap_bc, &bars->load_full[st], g * SN + 64, t0, b);
-                tc::tma_load_4d(base + 4 * SLAB, &tmap_x, &bars->load_full[st], 0, h, t0, b);
+                tc::tma_load_3d(smem + SM_CB + 2 * SLAB, &tmap_bc, &bars->cb_full, g * SN, t0, b);
+                tc::tma_load_3d(smem + SM_CB + 3 * SLAB, &tmap_bc, &bars->cb_full, g * SN + 64, t0, b);
+                if (j + 1 < ntiles) {                        // X one tile ahead
+                    const int jn = j + 1, sx = jn & 1;
+                    for (int hd = 0; hd < nh; ++hd) {
+                        HeadBars *hb = &bars->hd[hd];
+                        tc::mbar_wait(&hb->x_free[sx], ((jn >> 1) & 1) ^ 1, abort_flag, d_status);
+                        tc::mbar_arrive_expect_tx(&hb->x_full[sx], SLAB);
+                        tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES + sx * SLAB, &tmap_x,
+                                        &hb->x_full[sx], 0, head0 + hd, t0 + ST, b);
+                    }
+                }
             }
         }
-    } else if (warp == 5) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+    } else if (warp >= WARP_MMA0) {
+        // ------------------------------------------------------------------ MMA issuers
+        const int hd = warp - WARP_MMA0;
+        if (lane == 0 && hd < nh) {
             constexpr uint32_t id_g = tc::idesc_bf16(128, 128, 0, 0);     // C (K-major) x B (K-major)
             constexpr uint32_t id_y = tc::idesc_bf16(128, 64, 0, 1);      // K-major / TMEM A, MN-major B
             constexpr uint32_t id_h = tc::idesc_bf16(128, 64, 1, 1);      // MN-major A and B
-            const uint32_t xp_addr = tc::smem_u32(s_xp), hb_addr = tc::smem_u32(s_hb);
+            HeadBars *hb = &bars->hd[hd];
+            const uint32_t c_addr = tc::smem_u32(smem + SM_CB), b_addr = c_addr + 2 * SLAB;
+            const uint32_t head_addr = tc::smem_u32(smem + SM_HEAD + hd * SM_HEAD_BYTES);
+            const uint32_t xp_addr = head_addr + 2 * SLAB, hb_addr = head_addr + 3 * SLAB;
+            const uint32_t tm = tmem + TM_HEAD + hd * TM_HEAD_COLS;
             for (int j = 0; j < ntiles; ++j) {
-                const int st = j % SSD_STAGES;
-                const uint32_t base = tc::smem_u32(s_stage + st * STAGE_BYTES);
-                const uint32_t c_addr = base, b_addr = base + 2 * SLAB, x_addr = base + 4 * SLAB;
-                tc::mbar_wait(&bars->load_full[st], (j / SSD_STAGES) & 1, abort_flag, d_status);
+                const int sx = j & 1;
+                tc::mbar_wait(&bars->cb_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 if (full) {
-                    // MMA 1: G = Ctilde Btilde^T  (K = state index)
+                    if (hd == 0) {
+                        // MMA 1: G = Ctilde Btilde^T  (K = state index), shared by both heads
+                        if (j > 0) {
+                            tc::mbar_wait(&bars->g_free, (j - 1) & 1, abort_flag, d_status);
+                            tc::tc_fence_after();
+                        }
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
-                        tc::mma_ss(tmem + TM_G, tc::smem_desc_sw128(c_addr + off, 16, 1024),
-                                   tc::smem_desc_sw128(b_addr + off, 16, 1024), id_g, kk > 0);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
+                            tc::mma_ss(tmem + TM_G, tc::smem_desc_sw128(c_addr + off, 16, 1024),
+                                       tc::smem_desc_sw128(b_addr + off, 16, 1024), id_g, kk > 0);
+                        }
+                        tc::mma_commit(&bars->g_full);
                     }
-                    tc::mma_commit(&bars->g_full);
-                    // MMA 3: Yoff = Ctilde Hprev^T  (K = state index; B = bf16 state, rows = n)
-                    tc::mbar_wait(&bars->h_ready, j & 1, abort_flag, d_status);
+                    // MMA 3: Y = Ctilde Hprev^T  (K = state index; B = bf16 state, rows = n)
+                    tc::mbar_wait(&hb->h_ready, j & 1, abort_flag, d_status);
+                    if (j > 0) tc::mbar_wait(&hb->y_free, (j - 1) & 1, abort_flag, d_status);
                     tc::tc_fence_after();
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk) {
                         const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
-                        tc::mma_ss(tmem + TM_YOFF, tc::smem_desc_sw128(c_addr + off, 16, 1024),
+                        tc::mma_ss(tm + TM_Y, tc::smem_desc_sw128(c_addr + off, 16, 1024),
                                    tc::smem_desc_sw128(hb_addr + kk * 2048, SLAB, 1024), id_y, kk > 0);
                     }
-                    tc::mma_commit(&bars->yoff_full);
-                }
-                tc::mbar_wait(&bars->m_full, j & 1, abort_flag, d_status);
-                tc::tc_fence_after();
-                if (full) {
-                    // MMA 2: Ydiag = M X  (A = masked tile in TMEM, 8 columns per 16 tokens of K)
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        tc::mma_ts(tmem + TM_YD, tmem + TM_M + kk * 8,
-                                   tc::smem_desc_sw128(x_addr + kk * 2048, SLAB, 1024), id_y, kk > 0);
-                    tc::mma_commit(&bars->yd_full);
+                    tc::mma_commit(&hb->yoff_full);
                 }
                 // MMA 4: dH^T[n,p] = sum_s Btilde[s,n] (w_s x_s[p])   (K = token)
+                tc::mbar_wait(&hb->xp_full, j & 1, abort_flag, d_status);
+                tc::tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)
-                    tc::mma_ss(tmem + TM_DH, tc::smem_desc_sw128(b_addr + kk * 2048, SLAB, 1024),
+                    tc::mma_ss(tm + TM_DH, tc::smem_desc_sw128(b_addr + kk * 2048, SLAB, 1024),
                                tc::smem_desc_sw128(xp_addr + kk * 2048, SLAB, 1024), id_h, kk > 0);
-                tc::mma_commit(&bars->dh_full);
-                tc::mma_commit(&bars->load_empty[st]);
+                tc::mma_commit(&hb->dh_full);
+                tc::mma_commit(&bars->cb_empty);         // C and B tiles are no longer needed
+                if (full) {
+                    // MMA 2: Y += M X  (A = masked tile in TMEM, 8 columns per 16 tokens of K)
+                    tc::mbar_wait(&hb->m_full, j & 1, abort_flag, d_status);
+                    tc::tc_fence_after();
+                    const uint32_t x_addr = head_addr + sx * SLAB;
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk)
+                        tc::mma_ts(tm + TM_Y, tm + TM_M + kk * 8,
+                                   tc::smem_desc_sw128(x_addr + kk * 2048, SLAB, 1024), id_y, 1);
+                    tc::mma_commit(&hb->yd_full);
+                }
+                tc::mma_commit(&hb->x_free[sx]);
             }
         }
-    } else {
-        // ------------------------------------------------------------------ compute warps
-        const int i = tid;                                   // token row in the tile == state index n
-        const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    } else if ((warp >> 2) < nh) {
+        // ------------------------------------------------------------------ compute warpgroups
+        const int hd = warp >> 2, wq = warp & 3;
+        const int h = head0 + hd;
+        const int i = tid & 127;                             // token row in the tile == state index n
+        HeadBars *hb = &bars->hd[hd];
+        uint8_t *s_head = smem + SM_HEAD + hd * SM_HEAD_BYTES;
+        uint8_t *s_xp = s_head + 2 * SLAB, *s_hb = s_head + 3 * SLAB;
+        float *s_cs = sm->cs[hd], *s_cb = sm->cb[hd], *s_scan = sm->scan[hd];
+        const int bar_id = 1 + hd;
+        const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
+        const uint32_t tm = tmem + TM_HEAD + hd * TM_HEAD_COLS + lane_base;
         const float Ah = prm.A[h] * LOG2E, bias = prm.dt_bias[h];
         const float Dh = prm.D ? prm.D[h] : 0.f;
         // fp32 master copy of the state: this thread holds H[n = i][p = 0..63]
@@ -206,50 +287,54 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     *reinterpret_cast<uint4 *>(s_hb + tc::sw128_offset(i, ch)) = v;
                 }
                 tc::fence_proxy_async_smem();
-                tc::mbar_arrive(&bars->h_ready);
+                tc::mbar_arrive(&hb->h_ready);
+                // blocks of M above the diagonal stay zero for the whole kernel
+                uint32_t zero[16];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) zero[q] = 0u;
+                for (int c = wq + 1; c < 4; ++c) tc::tmem_st16(tm + TM_M + c * 16, zero);
+                tc::tmem_st_wait();
             }
         }
         float seg_l2 = 0.f;      // log2 of the product of a_t over the tiles done so far
+        const float *dt_row = prm.dt ? prm.dt + ((int64_t)b * L) * H + h : nullptr;
+        float raw_next = (dt_row && t_begin + i < t_end) ? dt_row[(int64_t)(t_begin + i) * H] : 0.f;
 
         for (int j = 0; j < ntiles; ++j) {
-            const int st = j % SSD_STAGES;
-            uint8_t *stage = s_stage + st * STAGE_BYTES;
+            const int sx = j & 1;
+            const uint8_t *s_x = s_head + sx * SLAB;
             const int t = t_begin + j * ST + i;
             const bool valid = t < t_end;
             // ---- per-token scalars: Delta, cumulative log2 decay inside the tile
-            float delta = 0.f;
-            if (valid) {
-                const float raw = prm.dt ? prm.dt[((int64_t)b * L + t) * H + h] : 0.f;
-                delta = softplus_f(raw + bias);
-            }
+            const float raw = raw_next;
+            raw_next = (dt_row && t + ST < t_end) ? dt_row[(int64_t)(t + ST) * H] : 0.f;
+            const float delta = valid ? softplus_f(raw + bias) : 0.f;
             float l2 = delta * Ah;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const float nb = __shfl_up_sync(0xffffffffu, l2, o);
                 if (lane >= o) l2 += nb;
             }
-            tc::named_bar_sync(1, 128);                       // previous tile's readers of s_cs/s_scan done
-            if (lane == 31) s_scan[warp] = l2;
-            tc::named_bar_sync(1, 128);
-            float l2_last = 0.f;
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                const float tot = s_scan[w];
-                if (w < warp) l2 += tot;
-                l2_last += tot;
-            }
+            tc::named_bar_sync(bar_id, 128);                 // previous tile's readers of cs/cb/scan done
+            if (lane == 31) s_scan[wq] = l2;
+            tc::named_bar_sync(bar_id, 128);
+            const float4 tot = *reinterpret_cast<const float4 *>(s_scan);
+            const float L1 = tot.x, L2 = L1 + tot.y, L3 = L2 + tot.z, l2_last = L3 + tot.w;
+            const float Lw = wq == 0 ? 0.f : (wq == 1 ? L1 : (wq == 2 ? L2 : L3));    // l before my block
+            const float Lend = wq == 0 ? L1 : (wq == 1 ? L2 : (wq == 2 ? L3 : l2_last));
+            l2 += Lw;
             s_cs[i] = (delta > 0.f ? tc::lg2_approx(delta) : -INFINITY) - l2;
+            s_cb[i] = delta * tc::ex2_approx(Lend - l2);
             const float w_s = delta * tc::ex2_approx(l2_last - l2);
-            tc::named_bar_sync(1, 128);
+            tc::named_bar_sync(bar_id, 128);
 
-            // ---- w . X  (row i of the X slab -> row i of the X' slab), keep x_i for the epilogue
-            tc::mbar_wait(&bars->load_full[st], (j / SSD_STAGES) & 1, abort_flag, d_status);
-            uint4 xrow[8];
+            // ---- w . X  (row i of the X slab -> row i of the X' slab)
+            tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
                 const uint32_t off = tc::sw128_offset(i, ch);
-                xrow[ch] = *reinterpret_cast<const uint4 *>(stage + 4 * SLAB + off);
-                const uint32_t wv[4] = {xrow[ch].x, xrow[ch].y, xrow[ch].z, xrow[ch].w};
+                const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
+                const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
                 uint32_t o[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
@@ -257,85 +342,70 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                                            w_s * __uint_as_float(wv[q] & 0xffff0000u));
                 *reinterpret_cast<uint4 *>(s_xp + off) = make_uint4(o[0], o[1], o[2], o[3]);
             }
+            tc::fence_proxy_async_smem();
+            tc::mbar_arrive(&hb->xp_full);
 
             if (full) {
+                // ---- Y = exp(l_i) * (Ctilde Hprev^T), in place
+                tc::mbar_wait(&hb->yoff_full, j & 1, abort_flag, d_status);
+                tc::tc_fence_after();
+                const float e_i = tc::ex2_approx(l2);
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t yo[32];
+                    tc::tmem_ld32(tm + TM_Y + half * 32, yo);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) yo[q] = __float_as_uint(e_i * __uint_as_float(yo[q]));
+                    tc::tmem_st32(tm + TM_Y + half * 32, yo);
+                }
                 // ---- decay mask: G (fp32, TMEM) -> M (bf16, TMEM), this thread owns row i
                 tc::mbar_wait(&bars->g_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
+                const float r_i = tc::ex2_approx(l2 - Lw);
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
-                    if (c <= warp) {
-                        uint32_t gv[32];
-                        tc::tmem_ld32(tmem + lane_base + TM_G + c * 32, gv);
-                        tc::tmem_ld_wait();
-                        const bool diag = (c == warp);
+                for (int c = 0; c <= wq; ++c) {
+                    uint32_t gv[32], pk[16];
+                    tc::tmem_ld32(tmem + lane_base + TM_G + c * 32, gv);
+                    tc::tmem_ld_wait();
+                    if (c == wq) {
 #pragma unroll
                         for (int q = 0; q < 16; ++q) {
                             const float2 cs = *reinterpret_cast<const float2 *>(&s_cs[c * 32 + 2 * q]);
                             float m0 = __uint_as_float(gv[2 * q]) * tc::ex2_approx(l2 + cs.x);
                             float m1 = __uint_as_float(gv[2 * q + 1]) * tc::ex2_approx(l2 + cs.y);
-                            if (diag) {
-                                if (2 * q > lane) m0 = 0.f;
-                                if (2 * q + 1 > lane) m1 = 0.f;
-                            }
+                            if (2 * q > lane) m0 = 0.f;
+                            if (2 * q + 1 > lane) m1 = 0.f;
                             pk[q] = tc::pack_bf16x2(m0, m1);
                         }
                     } else {
+                        // l at the end of column block c, relative to the start of my block
+                        const float Lc1 = c == 0 ? L1 : (c == 1 ? L2 : L3);
+                        const float rowf = r_i * tc::ex2_approx(Lw - Lc1);
 #pragma unroll
-                        for (int q = 0; q < 16; ++q) pk[q] = 0u;
-                    }
-                    tc::tmem_st16(tmem + lane_base + TM_M + c * 16, pk);
-                }
-                tc::tmem_st_wait();
-            }
-            tc::fence_proxy_async_smem();
-            tc::tc_fence_before();
-            tc::mbar_arrive(&bars->m_full);
-
-            if (full) {
-                // ---- epilogue: y_i = Ydiag_i + exp(l_i) Yoff_i + D x_i
-                tc::mbar_wait(&bars->yoff_full, j & 1, abort_flag, d_status);
-                tc::mbar_wait(&bars->yd_full, j & 1, abort_flag, d_status);
-                tc::tc_fence_after();
-                const float e_i = tc::ex2_approx(l2);
-                __nv_bfloat16 *yrow = prm.y + (((int64_t)b * L + t) * H + h) * SP;
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t yd[32], yo[32];
-                    tc::tmem_ld32(tmem + lane_base + TM_YD + half * 32, yd);
-                    tc::tmem_ld32(tmem + lane_base + TM_YOFF + half * 32, yo);
-                    tc::tmem_ld_wait();
-                    if (valid) {
-#pragma unroll
-                        for (int ch = 0; ch < 4; ++ch) {
-                            const uint4 xr = xrow[half * 4 + ch];
-                            const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
-                            uint32_t o[4];
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const int e0 = ch * 8 + 2 * q;
-                                const float x0 = __uint_as_float(xw[q] << 16);
-                                const float x1 = __uint_as_float(xw[q] & 0xffff0000u);
-                                const float y0 = __uint_as_float(yd[e0]) + e_i * __uint_as_float(yo[e0]) + Dh * x0;
-                                const float y1 = __uint_as_float(yd[e0 + 1]) + e_i * __uint_as_float(yo[e0 + 1]) + Dh * x1;
-                                o[q] = tc::pack_bf16x2(y0, y1);
-                            }
-                            *reinterpret_cast<uint4 *>(yrow + half * 32 + ch * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                        for (int q = 0; q < 16; ++q) {
+                            const float2 cb = *reinterpret_cast<const float2 *>(&s_cb[c * 32 + 2 * q]);
+                            pk[q] = tc::pack_bf16x2(__uint_as_float(gv[2 * q]) * cb.x * rowf,
+                                                    __uint_as_float(gv[2 * q + 1]) * cb.y * rowf);
                         }
                     }
+                    tc::tmem_st16(tm + TM_M + c * 16, pk);
                 }
+                tc::tmem_st_wait();
+                tc::tc_fence_before();
+                tc::mbar_arrive(&bars->g_free);
+                tc::mbar_arrive(&hb->m_full);
             }
 
             // ---- state: H = exp(l_last) H + dH  (thread i owns state index n = i)
-            tc::mbar_wait(&bars->dh_full, j & 1, abort_flag, d_status);
+            tc::mbar_wait(&hb->dh_full, j & 1, abort_flag, d_status);
             tc::tc_fence_after();
             const float dec = tc::ex2_approx(l2_last);
             seg_l2 += l2_last;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t dh[32];
-                tc::tmem_ld32(tmem + lane_base + TM_DH + half * 32, dh);
+                tc::tmem_ld32(tm + TM_DH + half * 32, dh);
                 tc::tmem_ld_wait();
 #pragma unroll
                 for (int q = 0; q < 32; ++q)
@@ -352,10 +422,40 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 tc::fence_proxy_async_smem();
                 tc::tc_fence_before();
-                tc::mbar_arrive(&bars->h_ready);
+                tc::mbar_arrive(&hb->h_ready);
+
+                // ---- epilogue: y_i = Y_i + D x_i
+                tc::mbar_wait(&hb->yd_full, j & 1, abort_flag, d_status);
+                tc::tc_fence_after();
+                __nv_bfloat16 *yrow = prm.y + (((int64_t)b * L + t) * H + h) * SP;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t yd[32];
+                    tc::tmem_ld32(tm + TM_Y + half * 32, yd);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(i, half * 4 + ch));
+                        const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int e0 = ch * 8 + 2 * q;
+                            const float x0 = __uint_as_float(xw[q] << 16);
+                            const float x1 = __uint_as_float(xw[q] & 0xffff0000u);
+                            o[q] = tc::pack_bf16x2(fmaf(Dh, x0, __uint_as_float(yd[e0])),
+                                                   fmaf(Dh, x1, __uint_as_float(yd[e0 + 1])));
+                        }
+                        if (valid)
+                            *reinterpret_cast<uint4 *>(yrow + half * 32 + ch * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+                tc::tc_fence_before();
+                tc::mbar_arrive(&hb->y_free);
             } else {
                 tc::tc_fence_before();
             }
+            tc::mbar_arrive(&hb->x_free[sx]);
         }
 
         // ---- final state of the segment
@@ -374,7 +474,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 5) tc::tmem_dealloc(tmem, TM_COLS);
+    if (warp == WARP_MMA0) tc::tmem_dealloc(tmem, TM_COLS);
 }
 
 // K3: chain the segments.  states[b,s,h,:,:] holds segment s's local end state (computed from a
@@ -407,19 +507,16 @@ bool ssd_tiles_supported(int dtype, int P, int N)
     return dtype == SWIMBA_DTYPE_BF16 && P == SP && N == SN;
 }
 
-static size_t ssd_smem_bytes()
-{
-    return 1024 + SSD_STAGES * STAGE_BYTES + 2 * SLAB + (ST + 8) * sizeof(float) + sizeof(SsdBars) + 64;
-}
+static size_t ssd_smem_bytes() { return SM_SMALL + sizeof(SsdSmall); }
 
 // Segment length (tokens, multiple of 128) so that the grid fills the SMs; L itself if one
 // segment per sequence is enough.
-int ssd_segment_len(int B, int L, int H, int chunk, int sm_count)
+int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count)
 {
-    const int64_t pairs = (int64_t)B * H;
+    const int64_t ctas = (int64_t)B * G * pairs_per_group(H, G);
     const int tiles = ceil_div(L, ST);
-    if (pairs >= sm_count || tiles <= 2) return tiles * ST;
-    int want = (int)ceil_div64(2 * (int64_t)sm_count, pairs);        // segments per sequence
+    if (2 * ctas > sm_count || tiles <= 2) return tiles * ST;
+    int want = (int)ceil_div64(2 * (int64_t)sm_count, ctas);          // segments per sequence
     int q_tiles = chunk >= ST ? chunk / ST : 1;                       // segments are whole chunks
     int seg_tiles = ceil_div(tiles, want);
     seg_tiles = ceil_div(seg_tiles, q_tiles) * q_tiles;
@@ -427,9 +524,9 @@ int ssd_segment_len(int B, int L, int H, int chunk, int sm_count)
     return seg_tiles * ST;
 }
 
-size_t ssd_workspace_bytes(int B, int L, int H, int chunk, int sm_count)
+size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count)
 {
-    const int seg_len = ssd_segment_len(B, L, H, chunk, sm_count);
+    const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
     const int nseg = ceil_div(L, seg_len);
     if (nseg <= 1) return 0;
     return (size_t)B * nseg * H * SP * SN * sizeof(float) + ((size_t)B * nseg * H * sizeof(float) + 255) / 256 * 256;
@@ -458,14 +555,14 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     if (cudaFuncSetAttribute(ssd_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SWIMBA_ERR_CUDA;
 
-    const int seg_len = ssd_segment_len(B, L, H, chunk, sm_count);
+    const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
     const int nseg = ceil_div(L, seg_len);
     SsdParams p;
     p.dt = dt; p.A = A; p.dt_bias = dt_bias; p.D = D;
     p.y = (__nv_bfloat16 *)y;
     p.L = L; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
     p.d_status = ctx.d_status;
-    dim3 grid((unsigned)nseg, (unsigned)H, (unsigned)B);
+    dim3 grid((unsigned)nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
     if (nseg == 1) {
         p.h_in = h0; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);

@@ -1,6 +1,6 @@
 // Thin inline-PTX wrappers for the Blackwell (sm_100a) async machinery used by the tensor-core
 // kernels: mbarriers, TMA tile loads, tcgen05 MMA with TMEM accumulators, and the shared-memory /
-// instruction descriptors they take.  Every wait is bounded: after WAIT_LIMIT_NS it records
+// instruction descriptors they take.  Every wait is bounded: after WAIT_LIMIT_CYCLES it records
 // SWIMBA_ERR_DEVICE_TIMEOUT in the device status word, raises a CTA-wide abort flag and returns,
 // and all later waits of that CTA return at once, so that the kernel always runs to its normal
 // exit (releasing its TMEM) with garbage results instead of hanging.
@@ -12,15 +12,10 @@
 namespace swimba {
 namespace tc {
 
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // 2 s
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about 2 s of SM clock
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
 }
 
 // ---------------------------------------------------------------- mbarrier
@@ -53,11 +48,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
                                           int *d_status) {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
+    const long long t0 = clock64();             // the SM's own cycle counter: cheap to read
     while (true) {
-        if (*abort_flag) return false;
         if (mbar_try_wait(bar, parity)) return true;
-        if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             *abort_flag = 1;
             atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_TIMEOUT);
             return false;
