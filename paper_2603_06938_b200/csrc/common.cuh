@@ -10,9 +10,9 @@ namespace swimba {
 
 // Kernel ids reported by the optional per-kernel timing (swimba_profile_read).
 enum Stage {
-    STAGE_ROUTER = 1, STAGE_TILE_TABLE = 2, STAGE_SCATTER = 3, STAGE_EXPERT_GEMM = 4,
+    STAGE_ROUTER = 1, STAGE_EXPERT_GEMM = 4,
     STAGE_MIX_SLOTS = 5, STAGE_PROJECT_SIMT = 6, STAGE_SSD_SEQUENTIAL = 7, STAGE_DECODE_UPDATE = 8,
-    STAGE_SSD_TILES = 9, STAGE_SEGMENT_SCAN = 10, STAGE_DECODE_PROJECT = 11,
+    STAGE_SSD_TILES = 9, STAGE_SEGMENT_SCAN = 10, STAGE_SSD_SCALARS = 11,
 };
 
 constexpr int PROF_MAX = 64;

@@ -3,20 +3,22 @@
 // chunks; the recurrence itself is Theorem 1's h_t = a_t h_{t-1} + Delta_t Btilde_t x_t^T,
 // y_t = Ctilde_t^T h_t + D x_t).
 //
-// One CTA owns one (sequence, pair of heads of one B/C group, segment) and walks its segment in
-// tiles of 128 tokens.  With l_i = sum_{r<=i} Delta_r A (inside the tile), per tile:
+// A small kernel first turns dt into Delta and the log-decay accumulated inside each 128-token
+// tile.  Then one CTA owns one (sequence, pair of heads of one B/C group, segment) and walks its
+// segment in tiles of 128 tokens.  With l_i = sum_{r<=i} Delta_r A (inside the tile), per tile:
 //   G      = Ctilde Btilde^T                      [128 x 128]  (MMA 1, once for both heads)
 // and for each of the two heads
 //   Y      = Ctilde H_prev^T                      [128 x 64]   (MMA 3), then scaled in place by
 //            exp(l_i) on the CUDA cores
 //   M[i,s] = G[i,s] exp(l_i - l_s) Delta_s  for s <= i, else 0      (CUDA cores -> TMEM, bf16)
 //   Y     += M X                                               (MMA 2, A operand from TMEM)
-//   y_i    = Y_i + D x_i
+//   y_i    = Y_i + D x_i                                       (staged in shared memory, TMA store)
 //   dH^T   = Btilde^T (w . X),  w_s = exp(l_last - l_s) Delta_s  [128 x 64]  (MMA 4)
 //   H      = exp(l_last) H_prev + dH                           (fp32, registers)
 // The carried state never leaves the SM inside a segment: the inter-chunk recurrence is fused.
-// The two heads run on two compute warpgroups with their own MMA-issuing warps, so that one
-// head's tensor-core and memory latencies are covered by the other head's CUDA-core work.
+// Each head has eight compute warps (a thread owns one token row / state index and one half of
+// the head dimension) and its own MMA-issuing warp, so that one head's tensor-core and memory
+// latencies are covered by the other warps' CUDA-core work.
 //
 // The decay mask needs exp(l_i - l_s) for every kept (i, s).  Only the four 32x32 blocks on the
 // diagonal evaluate it entry by entry.  A block strictly below the diagonal (rows in block w,
@@ -38,17 +40,19 @@ constexpr int ST = 128;                 // tokens per tile
 constexpr int SP = 64;                  // head dim this kernel is built for
 constexpr int SN = 128;                 // state size this kernel is built for
 constexpr int NHD = 2;                  // heads per CTA
-// warps 0-3: head 0 compute, 4-7: head 1 compute, 8: TMA, 9: MMA issuer head 0 (+ MMA 1),
-// 10: MMA issuer head 1
-constexpr int SSD_THREADS = 128 * NHD + 32 * (1 + NHD);
-constexpr int WARP_TMA = 4 * NHD, WARP_MMA0 = 4 * NHD + 1;
+constexpr int NCW = 8 * NHD;            // compute warps
+// warps 0-7: head 0 compute, 8-15: head 1 compute (warp = 8 head + 4 half + row block),
+// 16: TMA, 17: MMA issuer head 0 (+ MMA 1), 18: MMA issuer head 1
+constexpr int WARP_TMA = NCW, WARP_MMA0 = NCW + 1;
+constexpr int SSD_THREADS = 32 * (NCW + 1 + NHD);
+constexpr int HEAD_THREADS = 256;
 constexpr uint32_t SLAB = 16384;        // 128 rows x 128 bytes
 constexpr float LOG2E = 1.4426950408889634f;
 
 // shared memory map (bytes from the 1024-aligned base)
 constexpr uint32_t SM_CB = 0;                        // C0 C1 B0 B1 slabs (single stage)
-constexpr uint32_t SM_HEAD = 4 * SLAB;               // per head: X[2] XP HB
-constexpr uint32_t SM_HEAD_BYTES = 4 * SLAB;
+constexpr uint32_t SM_HEAD = 4 * SLAB;               // per head: X[2] XP HB YS
+constexpr uint32_t SM_HEAD_BYTES = 5 * SLAB;
 constexpr uint32_t SM_SMALL = SM_HEAD + NHD * SM_HEAD_BYTES;
 
 // TMEM columns: G, then per head M (bf16 A operand), Y, dH
@@ -58,20 +62,19 @@ constexpr uint32_t TM_M = 0, TM_Y = 64, TM_DH = 128;
 enum { MODE_FULL = 0, MODE_STATE_ONLY = 1 };
 
 struct SsdParams {
-    const float *dt;        // [B,L,H] or null
-    const float *A, *dt_bias, *D;
+    const float2 *dl;       // [B,H,Lpad] (Delta, log2-decay accumulated inside the 128-token tile)
+    const float *D;
     const float *h_in;      // initial states: [B,H,P,N] (nseg == 1) or [B,nseg,H,P,N]; may be null
-    __nv_bfloat16 *y;       // [B,L,H,P]
     float *h_out;           // MODE_FULL: h_final [B,H,P,N] (last segment writes) or null
                             // MODE_STATE_ONLY: local end states [B,nseg,H,P,N]
     float *seg_decay;       // MODE_STATE_ONLY: [B,nseg,H] product of a_t over the segment
-    int L, H, G, nseg, seg_len, mode;
+    int L, Lpad, H, G, nseg, seg_len, mode;
     int *d_status;
 };
 
 struct __align__(8) HeadBars {
     uint64_t x_full[2], x_free[2];
-    uint64_t yoff_full, m_full, yd_full, xp_full, dh_full, h_ready, y_free;
+    uint64_t yoff_full, m_full, yd_full, xp_full, dh_full, h_ready, y_free, y_staged;
 };
 struct __align__(8) SsdBars {
     uint64_t cb_full, cb_empty, g_full, g_free;
@@ -81,7 +84,7 @@ struct __align__(8) SsdBars {
 struct __align__(16) SsdSmall {
     float cs[NHD][ST];       // log2(Delta_s) - l_s          (diagonal blocks)
     float cb[NHD][ST];       // Delta_s exp(L_{b(s)+1} - l_s) (blocks below the diagonal)
-    float scan[NHD][4];      // per-warp totals of the log-decay
+    float ends[NHD][4];      // l at the end of each 32-row block of the tile
     SsdBars bars;
     uint32_t tmem_slot;
     int abort_flag;
@@ -91,9 +94,35 @@ struct __align__(16) SsdSmall {
 __host__ __device__ inline int pairs_per_group(int H, int G) { return (H / G + NHD - 1) / NHD; }
 }  // namespace
 
+// Delta_t = softplus(dt_t + dt_bias_h) and the log2-decay accumulated inside each 128-token tile,
+// dl[(b*H + h)*Lpad + t] = (Delta_t, sum_{r <= t, r in t's tile} Delta_r A_h log2 e); positions
+// past L carry Delta = 0, so the last entry of a tile is always the tile's total.
+__global__ void __launch_bounds__(ST)
+ssd_scalars_kernel(const float *__restrict__ dt, const float *__restrict__ A,
+                   const float *__restrict__ dt_bias, int L, int Lpad, int H,
+                   float2 *__restrict__ dl)
+{
+    __shared__ float s_tot[4];
+    const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int i = threadIdx.x, lane = i & 31, wq = i >> 5;
+    const int t = tile * ST + i;
+    const float raw = (dt && t < L) ? dt[((int64_t)b * L + t) * H + h] : 0.f;
+    const float delta = t < L ? softplus_f(raw + dt_bias[h]) : 0.f;
+    float l2 = delta * (A[h] * LOG2E);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float nb = __shfl_up_sync(0xffffffffu, l2, o);
+        if (lane >= o) l2 += nb;
+    }
+    if (lane == 31) s_tot[wq] = l2;
+    __syncthreads();
+    for (int w = 0; w < wq; ++w) l2 += s_tot[w];
+    dl[((int64_t)b * H + h) * Lpad + t] = make_float2(delta, l2);
+}
+
 __global__ void __launch_bounds__(SSD_THREADS, 1)
 ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
-                 const SsdParams prm)
+                 const __grid_constant__ CUtensorMap tmap_y, const SsdParams prm)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     SsdSmall *sm = (SsdSmall *)(smem + SM_SMALL);
@@ -121,20 +150,21 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         tc::mbar_init(&bars->cb_full, 1);
         tc::mbar_init(&bars->cb_empty, nh);
         tc::mbar_init(&bars->g_full, 1);
-        tc::mbar_init(&bars->g_free, 128 * nh);
+        tc::mbar_init(&bars->g_free, HEAD_THREADS * nh);
         for (int hd = 0; hd < NHD; ++hd) {
             HeadBars *hb = &bars->hd[hd];
             for (int s = 0; s < 2; ++s) {
                 tc::mbar_init(&hb->x_full[s], 1);
-                tc::mbar_init(&hb->x_free[s], 129);
+                tc::mbar_init(&hb->x_free[s], HEAD_THREADS + 1);
             }
             tc::mbar_init(&hb->yoff_full, 1);
-            tc::mbar_init(&hb->m_full, 128);
+            tc::mbar_init(&hb->m_full, HEAD_THREADS);
             tc::mbar_init(&hb->yd_full, 1);
-            tc::mbar_init(&hb->xp_full, 128);
+            tc::mbar_init(&hb->xp_full, HEAD_THREADS);
             tc::mbar_init(&hb->dh_full, 1);
-            tc::mbar_init(&hb->h_ready, 128);
-            tc::mbar_init(&hb->y_free, 128);
+            tc::mbar_init(&hb->h_ready, HEAD_THREADS);
+            tc::mbar_init(&hb->y_free, HEAD_THREADS);
+            tc::mbar_init(&hb->y_staged, HEAD_THREADS);
         }
         *abort_flag = 0;
         tc::fence_mbar_init();
@@ -146,24 +176,31 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     if (warp == WARP_TMA && lane == 0) {
         tc::prefetch_tmap(&tmap_bc);
         tc::prefetch_tmap(&tmap_x);
+        tc::prefetch_tmap(&tmap_y);
     }
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = sm->tmem_slot;
 
-    if (warp == WARP_TMA) {
+    // Warp index as a value the compiler knows to be warp-uniform.
+    const int uwarp = __shfl_sync(0xffffffffu, warp, 0);
+    if (uwarp == WARP_TMA) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // (the whole warp runs the loop; one elected lane issues the copies)
+        const bool leader = tc::elect_one();
+        if (leader) {
             for (int hd = 0; hd < nh; ++hd) {               // X of tile 0
                 HeadBars *hb = &bars->hd[hd];
                 tc::mbar_arrive_expect_tx(&hb->x_full[0], SLAB);
                 tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES, &tmap_x, &hb->x_full[0], 0,
                                 head0 + hd, t_begin, b);
             }
-            for (int j = 0; j < ntiles; ++j) {
-                const int t0 = t_begin + j * ST;
-                tc::mbar_wait(&bars->cb_empty, (j & 1) ^ 1, abort_flag, d_status);
+        }
+        for (int j = 0; j < ntiles; ++j) {
+            const int t0 = t_begin + j * ST;
+            tc::mbar_wait(&bars->cb_empty, (j & 1) ^ 1, abort_flag, d_status);
+            if (leader) {
                 tc::mbar_arrive_expect_tx(&bars->cb_full, full ? 4 * SLAB : 2 * SLAB);
                 if (full) {
                     tc::tma_load_3d(smem + SM_CB + 0 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN, t0, b);
@@ -171,22 +208,28 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 tc::tma_load_3d(smem + SM_CB + 2 * SLAB, &tmap_bc, &bars->cb_full, g * SN, t0, b);
                 tc::tma_load_3d(smem + SM_CB + 3 * SLAB, &tmap_bc, &bars->cb_full, g * SN + 64, t0, b);
-                if (j + 1 < ntiles) {                        // X one tile ahead
-                    const int jn = j + 1, sx = jn & 1;
-                    for (int hd = 0; hd < nh; ++hd) {
-                        HeadBars *hb = &bars->hd[hd];
-                        tc::mbar_wait(&hb->x_free[sx], ((jn >> 1) & 1) ^ 1, abort_flag, d_status);
+            }
+            if (j + 1 < ntiles) {                            // X one tile ahead
+                const int jn = j + 1, sx = jn & 1;
+                for (int hd = 0; hd < nh; ++hd) {
+                    HeadBars *hb = &bars->hd[hd];
+                    tc::mbar_wait(&hb->x_free[sx], ((jn >> 1) & 1) ^ 1, abort_flag, d_status);
+                    if (leader) {
                         tc::mbar_arrive_expect_tx(&hb->x_full[sx], SLAB);
                         tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES + sx * SLAB, &tmap_x,
                                         &hb->x_full[sx], 0, head0 + hd, t0 + ST, b);
                     }
                 }
             }
+            __syncwarp();
         }
-    } else if (warp >= WARP_MMA0) {
+    } else if (uwarp >= WARP_MMA0) {
         // ------------------------------------------------------------------ MMA issuers
-        const int hd = warp - WARP_MMA0;
-        if (lane == 0 && hd < nh) {
+        // The whole warp runs the loop and the waits; one elected lane issues the MMAs, the
+        // commits and the y stores.
+        const int hd = uwarp - WARP_MMA0;
+        const bool leader = tc::elect_one();
+        if (hd < nh) {
             constexpr uint32_t id_g = tc::idesc_bf16(128, 128, 0, 0);     // C (K-major) x B (K-major)
             constexpr uint32_t id_y = tc::idesc_bf16(128, 64, 0, 1);      // K-major / TMEM A, MN-major B
             constexpr uint32_t id_h = tc::idesc_bf16(128, 64, 1, 1);      // MN-major A and B
@@ -194,77 +237,111 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             const uint32_t c_addr = tc::smem_u32(smem + SM_CB), b_addr = c_addr + 2 * SLAB;
             const uint32_t head_addr = tc::smem_u32(smem + SM_HEAD + hd * SM_HEAD_BYTES);
             const uint32_t xp_addr = head_addr + 2 * SLAB, hb_addr = head_addr + 3 * SLAB;
-            const uint32_t tm = tmem + TM_HEAD + hd * TM_HEAD_COLS;
+            const uint8_t *s_y = smem + SM_HEAD + hd * SM_HEAD_BYTES + 4 * SLAB;
+            const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+            const uint32_t tm = tmem_u + TM_HEAD + hd * TM_HEAD_COLS;
+            // descriptors of the first K step; later steps advance the address field
+            const uint64_t dC = tc::smem_desc_sw128(c_addr, 16, 1024);          // K-major
+            const uint64_t dB = tc::smem_desc_sw128(b_addr, 16, 1024);          // K-major
+            const uint64_t dBt = tc::smem_desc_sw128(b_addr, SLAB, 1024);       // MN-major
+            const uint64_t dH = tc::smem_desc_sw128(hb_addr, SLAB, 1024);       // MN-major
+            const uint64_t dXp = tc::smem_desc_sw128(xp_addr, SLAB, 1024);      // MN-major
+            const uint64_t dX0 = tc::smem_desc_sw128(head_addr, SLAB, 1024);    // MN-major
+            // MMA 1 of tile jj: G = Ctilde Btilde^T (K = state index), shared by both heads
+            auto issue_g = [&](int jj) {
+                tc::mbar_wait(&bars->cb_full, jj & 1, abort_flag, d_status);
+                if (jj > 0) tc::mbar_wait(&bars->g_free, (jj - 1) & 1, abort_flag, d_status);
+                tc::tc_fence_after();
+                if (leader) {
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) {
+                        const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
+                        tc::mma_ss(tmem_u + TM_G, tc::smem_desc_advance(dC, off),
+                                   tc::smem_desc_advance(dB, off), id_g, kk > 0);
+                    }
+                    tc::mma_commit(&bars->g_full);
+                }
+                __syncwarp();
+            };
+            if (full && hd == 0) issue_g(0);
             for (int j = 0; j < ntiles; ++j) {
                 const int sx = j & 1;
                 tc::mbar_wait(&bars->cb_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 if (full) {
-                    if (hd == 0) {
-                        // MMA 1: G = Ctilde Btilde^T  (K = state index), shared by both heads
-                        if (j > 0) {
-                            tc::mbar_wait(&bars->g_free, (j - 1) & 1, abort_flag, d_status);
-                            tc::tc_fence_after();
-                        }
-#pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
-                            tc::mma_ss(tmem + TM_G, tc::smem_desc_sw128(c_addr + off, 16, 1024),
-                                       tc::smem_desc_sw128(b_addr + off, 16, 1024), id_g, kk > 0);
-                        }
-                        tc::mma_commit(&bars->g_full);
-                    }
                     // MMA 3: Y = Ctilde Hprev^T  (K = state index; B = bf16 state, rows = n)
                     tc::mbar_wait(&hb->h_ready, j & 1, abort_flag, d_status);
                     if (j > 0) tc::mbar_wait(&hb->y_free, (j - 1) & 1, abort_flag, d_status);
                     tc::tc_fence_after();
+                    if (leader) {
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk) {
-                        const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
-                        tc::mma_ss(tm + TM_Y, tc::smem_desc_sw128(c_addr + off, 16, 1024),
-                                   tc::smem_desc_sw128(hb_addr + kk * 2048, SLAB, 1024), id_y, kk > 0);
+                        for (int kk = 0; kk < 8; ++kk) {
+                            const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
+                            tc::mma_ss(tm + TM_Y, tc::smem_desc_advance(dC, off),
+                                       tc::smem_desc_advance(dH, kk * 2048), id_y, kk > 0);
+                        }
+                        tc::mma_commit(&hb->yoff_full);
                     }
-                    tc::mma_commit(&hb->yoff_full);
+                    __syncwarp();
                 }
                 // MMA 4: dH^T[n,p] = sum_s Btilde[s,n] (w_s x_s[p])   (K = token)
                 tc::mbar_wait(&hb->xp_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
+                if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    tc::mma_ss(tm + TM_DH, tc::smem_desc_sw128(b_addr + kk * 2048, SLAB, 1024),
-                               tc::smem_desc_sw128(xp_addr + kk * 2048, SLAB, 1024), id_h, kk > 0);
-                tc::mma_commit(&hb->dh_full);
-                tc::mma_commit(&bars->cb_empty);         // C and B tiles are no longer needed
+                    for (int kk = 0; kk < 8; ++kk)
+                        tc::mma_ss(tm + TM_DH, tc::smem_desc_advance(dBt, kk * 2048),
+                                   tc::smem_desc_advance(dXp, kk * 2048), id_h, kk > 0);
+                    tc::mma_commit(&hb->dh_full);
+                    tc::mma_commit(&bars->cb_empty);     // C and B tiles are no longer needed
+                }
+                __syncwarp();
                 if (full) {
                     // MMA 2: Y += M X  (A = masked tile in TMEM, 8 columns per 16 tokens of K)
                     tc::mbar_wait(&hb->m_full, j & 1, abort_flag, d_status);
                     tc::tc_fence_after();
-                    const uint32_t x_addr = head_addr + sx * SLAB;
+                    const uint64_t dX = tc::smem_desc_advance(dX0, sx * SLAB);
+                    if (leader) {
+                        tc::bulk_wait_read_all();        // previous y tile has left its staging buffer
 #pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        tc::mma_ts(tm + TM_Y, tm + TM_M + kk * 8,
-                                   tc::smem_desc_sw128(x_addr + kk * 2048, SLAB, 1024), id_y, 1);
-                    tc::mma_commit(&hb->yd_full);
+                        for (int kk = 0; kk < 8; ++kk)
+                            tc::mma_ts(tm + TM_Y, tm + TM_M + kk * 8, tc::smem_desc_advance(dX, kk * 2048),
+                                       id_y, 1);
+                        tc::mma_commit(&hb->yd_full);
+                    }
                 }
-                tc::mma_commit(&hb->x_free[sx]);
+                if (leader) tc::mma_commit(&hb->x_free[sx]);
+                __syncwarp();
+                if (full) {
+                    if (hd == 0 && j + 1 < ntiles) issue_g(j + 1);
+                    // the staged y tile goes out as one TMA store (rows past the end of the
+                    // sequence are clipped by the tensor map)
+                    tc::mbar_wait(&hb->y_staged, j & 1, abort_flag, d_status);
+                    if (leader) {
+                        tc::tma_store_4d(&tmap_y, s_y, 0, head0 + hd, t_begin + j * ST, b);
+                        tc::bulk_commit_group();
+                    }
+                    __syncwarp();
+                }
             }
+            if (full && leader) tc::bulk_wait_read_all();
         }
-    } else if ((warp >> 2) < nh) {
-        // ------------------------------------------------------------------ compute warpgroups
-        const int hd = warp >> 2, wq = warp & 3;
+    } else if ((uwarp >> 3) < nh) {
+        // ------------------------------------------------------------------ compute warps
+        const int hd = warp >> 3, hf = (warp >> 2) & 1, wq = warp & 3;
         const int h = head0 + hd;
-        const int i = tid & 127;                             // token row in the tile == state index n
+        const int i = wq * 32 + lane;                        // token row in the tile == state index n
+        const int p0 = 32 * hf;                              // this thread's half of the head dim
         HeadBars *hb = &bars->hd[hd];
         uint8_t *s_head = smem + SM_HEAD + hd * SM_HEAD_BYTES;
-        uint8_t *s_xp = s_head + 2 * SLAB, *s_hb = s_head + 3 * SLAB;
-        float *s_cs = sm->cs[hd], *s_cb = sm->cb[hd], *s_scan = sm->scan[hd];
+        uint8_t *s_xp = s_head + 2 * SLAB, *s_hb = s_head + 3 * SLAB, *s_y = s_head + 4 * SLAB;
+        float *s_cs = sm->cs[hd], *s_cb = sm->cb[hd], *s_ends = sm->ends[hd];
         const int bar_id = 1 + hd;
         const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
         const uint32_t tm = tmem + TM_HEAD + hd * TM_HEAD_COLS + lane_base;
-        const float Ah = prm.A[h] * LOG2E, bias = prm.dt_bias[h];
         const float Dh = prm.D ? prm.D[h] : 0.f;
-        // fp32 master copy of the state: this thread holds H[n = i][p = 0..63]
-        float Hst[SP];
+        // fp32 master copy of the state: this thread holds H[n = i][p = p0 .. p0+31]
+        float Hst[32];
         {
             const float *h_in = prm.h_in;
             if (h_in && full) {
@@ -272,67 +349,62 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     ? ((((int64_t)b * prm.nseg + seg) * H + h) * SP) * SN
                     : (((int64_t)b * H + h) * SP) * SN;
 #pragma unroll
-                for (int p = 0; p < SP; ++p) Hst[p] = h_in[base + (int64_t)p * SN + i];
+                for (int q = 0; q < 32; ++q) Hst[q] = h_in[base + (int64_t)(p0 + q) * SN + i];
             } else {
 #pragma unroll
-                for (int p = 0; p < SP; ++p) Hst[p] = 0.f;
+                for (int q = 0; q < 32; ++q) Hst[q] = 0.f;
             }
             if (full) {
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
+                for (int ch = 0; ch < 4; ++ch) {
                     uint4 v = make_uint4(tc::pack_bf16x2(Hst[8 * ch + 0], Hst[8 * ch + 1]),
                                          tc::pack_bf16x2(Hst[8 * ch + 2], Hst[8 * ch + 3]),
                                          tc::pack_bf16x2(Hst[8 * ch + 4], Hst[8 * ch + 5]),
                                          tc::pack_bf16x2(Hst[8 * ch + 6], Hst[8 * ch + 7]));
-                    *reinterpret_cast<uint4 *>(s_hb + tc::sw128_offset(i, ch)) = v;
+                    *reinterpret_cast<uint4 *>(s_hb + tc::sw128_offset(i, 4 * hf + ch)) = v;
                 }
                 tc::fence_proxy_async_smem();
                 tc::mbar_arrive(&hb->h_ready);
                 // blocks of M above the diagonal stay zero for the whole kernel
-                uint32_t zero[16];
+                uint32_t zero[8];
 #pragma unroll
-                for (int q = 0; q < 16; ++q) zero[q] = 0u;
-                for (int c = wq + 1; c < 4; ++c) tc::tmem_st16(tm + TM_M + c * 16, zero);
+                for (int q = 0; q < 8; ++q) zero[q] = 0u;
+                for (int c = wq + 1; c < 4; ++c) tc::tmem_st8(tm + TM_M + c * 16 + 8 * hf, zero);
                 tc::tmem_st_wait();
             }
         }
         float seg_l2 = 0.f;      // log2 of the product of a_t over the tiles done so far
-        const float *dt_row = prm.dt ? prm.dt + ((int64_t)b * L) * H + h : nullptr;
-        float raw_next = (dt_row && t_begin + i < t_end) ? dt_row[(int64_t)(t_begin + i) * H] : 0.f;
+        const float2 *dlp = prm.dl + ((int64_t)b * H + h) * prm.Lpad + t_begin;
+        float2 dl_next = dlp[i];
 
         for (int j = 0; j < ntiles; ++j) {
             const int sx = j & 1;
             const uint8_t *s_x = s_head + sx * SLAB;
-            const int t = t_begin + j * ST + i;
-            const bool valid = t < t_end;
             // ---- per-token scalars: Delta, cumulative log2 decay inside the tile
-            const float raw = raw_next;
-            raw_next = (dt_row && t + ST < t_end) ? dt_row[(int64_t)(t + ST) * H] : 0.f;
-            const float delta = valid ? softplus_f(raw + bias) : 0.f;
-            float l2 = delta * Ah;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const float nb = __shfl_up_sync(0xffffffffu, l2, o);
-                if (lane >= o) l2 += nb;
+            const float delta = dl_next.x, l2 = dl_next.y;
+            if (j + 1 < ntiles) dl_next = dlp[(j + 1) * ST + i];
+            const float Lend = __shfl_sync(0xffffffffu, l2, 31);       // l at the end of my block
+            if (hf == 0) {
+                // safe to overwrite: every reader of the previous tile's values had finished its
+                // mask before MMA 2 of that tile could start, and this thread has seen it end
+                // (in the state-only pass the readers are ordered by the barrier below instead)
+                if (lane == 31) s_ends[wq] = l2;
+                if (full) {
+                    s_cs[i] = (delta > 0.f ? tc::lg2_approx(delta) : -INFINITY) - l2;
+                    s_cb[i] = delta * tc::ex2_approx(Lend - l2);
+                }
             }
-            tc::named_bar_sync(bar_id, 128);                 // previous tile's readers of cs/cb/scan done
-            if (lane == 31) s_scan[wq] = l2;
-            tc::named_bar_sync(bar_id, 128);
-            const float4 tot = *reinterpret_cast<const float4 *>(s_scan);
-            const float L1 = tot.x, L2 = L1 + tot.y, L3 = L2 + tot.z, l2_last = L3 + tot.w;
+            tc::named_bar_sync(bar_id, HEAD_THREADS);        // ends / cs / cb of this tile are visible
+            const float4 ends = *reinterpret_cast<const float4 *>(s_ends);
+            const float L1 = ends.x, L2 = ends.y, L3 = ends.z, l2_last = ends.w;
             const float Lw = wq == 0 ? 0.f : (wq == 1 ? L1 : (wq == 2 ? L2 : L3));    // l before my block
-            const float Lend = wq == 0 ? L1 : (wq == 1 ? L2 : (wq == 2 ? L3 : l2_last));
-            l2 += Lw;
-            s_cs[i] = (delta > 0.f ? tc::lg2_approx(delta) : -INFINITY) - l2;
-            s_cb[i] = delta * tc::ex2_approx(Lend - l2);
             const float w_s = delta * tc::ex2_approx(l2_last - l2);
-            tc::named_bar_sync(bar_id, 128);
 
-            // ---- w . X  (row i of the X slab -> row i of the X' slab)
+            // ---- w . X  (row i of the X slab -> row i of the X' slab, this thread's half)
             tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                const uint32_t off = tc::sw128_offset(i, ch);
+            for (int ch = 0; ch < 4; ++ch) {
+                const uint32_t off = tc::sw128_offset(i, 4 * hf + ch);
                 const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
                 const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
                 uint32_t o[4];
@@ -349,47 +421,53 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 // ---- Y = exp(l_i) * (Ctilde Hprev^T), in place
                 tc::mbar_wait(&hb->yoff_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
-                const float e_i = tc::ex2_approx(l2);
+                {
+                    const float e_i = tc::ex2_approx(l2);
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t yo[32];
-                    tc::tmem_ld32(tm + TM_Y + half * 32, yo);
-                    tc::tmem_ld_wait();
+                    for (int hh = 0; hh < 2; ++hh) {
+                        uint32_t yo[16];
+                        tc::tmem_ld16(tm + TM_Y + p0 + 16 * hh, yo);
+                        tc::tmem_ld_wait();
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) yo[q] = __float_as_uint(e_i * __uint_as_float(yo[q]));
-                    tc::tmem_st32(tm + TM_Y + half * 32, yo);
+                        for (int q = 0; q < 16; ++q) yo[q] = __float_as_uint(e_i * __uint_as_float(yo[q]));
+                        tc::tmem_st16(tm + TM_Y + p0 + 16 * hh, yo);
+                    }
                 }
-                // ---- decay mask: G (fp32, TMEM) -> M (bf16, TMEM), this thread owns row i
+                // ---- decay mask: G (fp32, TMEM) -> M (bf16, TMEM); this thread owns row i and
+                // columns 16 hf .. 16 hf + 15 of every 32-column block
                 tc::mbar_wait(&bars->g_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 const float r_i = tc::ex2_approx(l2 - Lw);
-#pragma unroll 1
-                for (int c = 0; c <= wq; ++c) {
-                    uint32_t gv[32], pk[16];
-                    tc::tmem_ld32(tmem + lane_base + TM_G + c * 32, gv);
-                    tc::tmem_ld_wait();
-                    if (c == wq) {
+                const uint32_t g_addr = tmem + lane_base + TM_G + 16 * hf;
 #pragma unroll
-                        for (int q = 0; q < 16; ++q) {
-                            const float2 cs = *reinterpret_cast<const float2 *>(&s_cs[c * 32 + 2 * q]);
-                            float m0 = __uint_as_float(gv[2 * q]) * tc::ex2_approx(l2 + cs.x);
-                            float m1 = __uint_as_float(gv[2 * q + 1]) * tc::ex2_approx(l2 + cs.y);
-                            if (2 * q > lane) m0 = 0.f;
-                            if (2 * q + 1 > lane) m1 = 0.f;
-                            pk[q] = tc::pack_bf16x2(m0, m1);
-                        }
-                    } else {
-                        // l at the end of column block c, relative to the start of my block
-                        const float Lc1 = c == 0 ? L1 : (c == 1 ? L2 : L3);
-                        const float rowf = r_i * tc::ex2_approx(Lw - Lc1);
+                for (int c = 0; c < 4; ++c) {
+                    if (c <= wq) {
+                        uint32_t cur[16], pk[8];
+                        tc::tmem_ld16(g_addr + c * 32, cur);
+                        tc::tmem_ld_wait();
+                        if (c == wq) {
 #pragma unroll
-                        for (int q = 0; q < 16; ++q) {
-                            const float2 cb = *reinterpret_cast<const float2 *>(&s_cb[c * 32 + 2 * q]);
-                            pk[q] = tc::pack_bf16x2(__uint_as_float(gv[2 * q]) * cb.x * rowf,
-                                                    __uint_as_float(gv[2 * q + 1]) * cb.y * rowf);
+                            for (int q = 0; q < 8; ++q) {
+                                const float2 cs = *reinterpret_cast<const float2 *>(&s_cs[c * 32 + 16 * hf + 2 * q]);
+                                float m0 = __uint_as_float(cur[2 * q]) * tc::ex2_approx(l2 + cs.x);
+                                float m1 = __uint_as_float(cur[2 * q + 1]) * tc::ex2_approx(l2 + cs.y);
+                                if (16 * hf + 2 * q > lane) m0 = 0.f;
+                                if (16 * hf + 2 * q + 1 > lane) m1 = 0.f;
+                                pk[q] = tc::pack_bf16x2(m0, m1);
+                            }
+                        } else {
+                            // l at the end of column block c, relative to the start of my block
+                            const float Lc1 = c == 0 ? L1 : (c == 1 ? L2 : L3);
+                            const float rowf = r_i * tc::ex2_approx(Lw - Lc1);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q) {
+                                const float2 cb = *reinterpret_cast<const float2 *>(&s_cb[c * 32 + 16 * hf + 2 * q]);
+                                pk[q] = tc::pack_bf16x2(__uint_as_float(cur[2 * q]) * cb.x * rowf,
+                                                        __uint_as_float(cur[2 * q + 1]) * cb.y * rowf);
+                            }
                         }
+                        tc::tmem_st8(tm + TM_M + c * 16 + 8 * hf, pk);
                     }
-                    tc::tmem_st16(tm + TM_M + c * 16, pk);
                 }
                 tc::tmem_st_wait();
                 tc::tc_fence_before();
@@ -397,61 +475,65 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 tc::mbar_arrive(&hb->m_full);
             }
 
-            // ---- state: H = exp(l_last) H + dH  (thread i owns state index n = i)
+            // ---- state: H = exp(l_last) H + dH  (thread owns state index n = i, 32 channels)
             tc::mbar_wait(&hb->dh_full, j & 1, abort_flag, d_status);
             tc::tc_fence_after();
             const float dec = tc::ex2_approx(l2_last);
             seg_l2 += l2_last;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t dh[32];
-                tc::tmem_ld32(tm + TM_DH + half * 32, dh);
+            for (int hh = 0; hh < 2; ++hh) {
+                uint32_t dh[16];
+                tc::tmem_ld16(tm + TM_DH + p0 + 16 * hh, dh);
                 tc::tmem_ld_wait();
 #pragma unroll
-                for (int q = 0; q < 32; ++q)
-                    Hst[half * 32 + q] = fmaf(dec, Hst[half * 32 + q], __uint_as_float(dh[q]));
+                for (int q = 0; q < 16; ++q)
+                    Hst[16 * hh + q] = fmaf(dec, Hst[16 * hh + q], __uint_as_float(dh[q]));
+                if (full) {
+#pragma unroll
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        const int ch = 2 * hh + c2;
+                        uint4 v = make_uint4(tc::pack_bf16x2(Hst[8 * ch + 0], Hst[8 * ch + 1]),
+                                             tc::pack_bf16x2(Hst[8 * ch + 2], Hst[8 * ch + 3]),
+                                             tc::pack_bf16x2(Hst[8 * ch + 4], Hst[8 * ch + 5]),
+                                             tc::pack_bf16x2(Hst[8 * ch + 6], Hst[8 * ch + 7]));
+                        *reinterpret_cast<uint4 *>(s_hb + tc::sw128_offset(i, 4 * hf + ch)) = v;
+                    }
+                }
             }
             if (full) {
-#pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
-                    uint4 v = make_uint4(tc::pack_bf16x2(Hst[8 * ch + 0], Hst[8 * ch + 1]),
-                                         tc::pack_bf16x2(Hst[8 * ch + 2], Hst[8 * ch + 3]),
-                                         tc::pack_bf16x2(Hst[8 * ch + 4], Hst[8 * ch + 5]),
-                                         tc::pack_bf16x2(Hst[8 * ch + 6], Hst[8 * ch + 7]));
-                    *reinterpret_cast<uint4 *>(s_hb + tc::sw128_offset(i, ch)) = v;
-                }
                 tc::fence_proxy_async_smem();
                 tc::tc_fence_before();
                 tc::mbar_arrive(&hb->h_ready);
 
-                // ---- epilogue: y_i = Y_i + D x_i
+                // ---- epilogue: y_i = Y_i + D x_i, staged in shared memory for the TMA store
                 tc::mbar_wait(&hb->yd_full, j & 1, abort_flag, d_status);
                 tc::tc_fence_after();
-                __nv_bfloat16 *yrow = prm.y + (((int64_t)b * L + t) * H + h) * SP;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t yd[32];
-                    tc::tmem_ld32(tm + TM_Y + half * 32, yd);
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t yd[16];
+                    tc::tmem_ld16(tm + TM_Y + p0 + 16 * hh, yd);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(i, half * 4 + ch));
+                    for (int c2 = 0; c2 < 2; ++c2) {
+                        const uint32_t off = tc::sw128_offset(i, 4 * hf + 2 * hh + c2);
+                        const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
                         const uint32_t xw[4] = {xr.x, xr.y, xr.z, xr.w};
                         uint32_t o[4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
-                            const int e0 = ch * 8 + 2 * q;
+                            const int e0 = c2 * 8 + 2 * q;
                             const float x0 = __uint_as_float(xw[q] << 16);
                             const float x1 = __uint_as_float(xw[q] & 0xffff0000u);
                             o[q] = tc::pack_bf16x2(fmaf(Dh, x0, __uint_as_float(yd[e0])),
                                                    fmaf(Dh, x1, __uint_as_float(yd[e0 + 1])));
                         }
-                        if (valid)
-                            *reinterpret_cast<uint4 *>(yrow + half * 32 + ch * 8) = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4 *>(s_y + off) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 }
                 tc::tc_fence_before();
                 tc::mbar_arrive(&hb->y_free);
+                tc::fence_proxy_async_smem();
+                tc::mbar_arrive(&hb->y_staged);
             } else {
                 tc::tc_fence_before();
             }
@@ -463,13 +545,13 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             if (prm.h_out && seg == prm.nseg - 1) {
                 float *dst = prm.h_out + (((int64_t)b * H + h) * SP) * SN;
 #pragma unroll
-                for (int p = 0; p < SP; ++p) dst[(int64_t)p * SN + i] = Hst[p];
+                for (int q = 0; q < 32; ++q) dst[(int64_t)(p0 + q) * SN + i] = Hst[q];
             }
         } else {
             float *dst = prm.h_out + ((((int64_t)b * prm.nseg + seg) * H + h) * SP) * SN;
 #pragma unroll
-            for (int p = 0; p < SP; ++p) dst[(int64_t)p * SN + i] = Hst[p];
-            if (i == 0) prm.seg_decay[((int64_t)b * prm.nseg + seg) * H + h] = tc::ex2_approx(seg_l2);
+            for (int q = 0; q < 32; ++q) dst[(int64_t)(p0 + q) * SN + i] = Hst[q];
+            if (i == 0 && hf == 0) prm.seg_decay[((int64_t)b * prm.nseg + seg) * H + h] = tc::ex2_approx(seg_l2);
         }
     }
     tc::tc_fence_before();
@@ -524,12 +606,21 @@ int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count)
     return seg_tiles * ST;
 }
 
+// Workspace: [Delta / log-decay pairs B*H*Lpad float2] [segment states] [segment decays].
+static size_t ssd_scalars_bytes(int B, int L, int H)
+{
+    const size_t Lpad = (size_t)ceil_div(L, ST) * ST;
+    return ((size_t)B * H * Lpad * sizeof(float2) + 255) / 256 * 256;
+}
+
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count)
 {
     const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
     const int nseg = ceil_div(L, seg_len);
-    if (nseg <= 1) return 0;
-    return (size_t)B * nseg * H * SP * SN * sizeof(float) + ((size_t)B * nseg * H * sizeof(float) + 255) / 256 * 256;
+    size_t tot = ssd_scalars_bytes(B, L, H);
+    if (nseg > 1)
+        tot += (size_t)B * nseg * H * SP * SN * sizeof(float) + ((size_t)B * nseg * H * sizeof(float) + 255) / 256 * 256;
+    return tot;
 }
 
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
@@ -538,7 +629,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
 {
     if (B <= 0 || L <= 0) return SWIMBA_OK;
     const int S = 2 * G * SN;
-    CUtensorMap tm_bc, tm_x;
+    CUtensorMap tm_bc, tm_x, tm_y;
     {
         const uint64_t dims[3] = {(uint64_t)S, (uint64_t)L, (uint64_t)B};
         const uint64_t str[2] = {(uint64_t)S * 2, (uint64_t)L * S * 2};
@@ -550,6 +641,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         const uint64_t str[3] = {(uint64_t)SP * 2, (uint64_t)H * SP * 2, (uint64_t)L * H * SP * 2};
         const uint32_t box[4] = {SP, 1, ST, 1};
         if (!encode_tmap_bf16(&tm_x, x, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
+        if (!encode_tmap_bf16(&tm_y, y, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
     }
     const size_t smem = ssd_smem_bytes();
     if (cudaFuncSetAttribute(ssd_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
@@ -557,23 +649,29 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
 
     const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
     const int nseg = ceil_div(L, seg_len);
+    const int Lpad = ceil_div(L, ST) * ST;
+    float2 *dl = (float2 *)workspace;
+    char *seg_ws = (char *)workspace + ssd_scalars_bytes(B, L, H);
+    ctx.begin(STAGE_SSD_SCALARS);
+    ssd_scalars_kernel<<<dim3((unsigned)(Lpad / ST), (unsigned)H, (unsigned)B), ST, 0, ctx.stream>>>(
+        dt, A, dt_bias, L, Lpad, H, dl);
+    ctx.end();
     SsdParams p;
-    p.dt = dt; p.A = A; p.dt_bias = dt_bias; p.D = D;
-    p.y = (__nv_bfloat16 *)y;
-    p.L = L; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
+    p.dl = dl; p.D = D;
+    p.L = L; p.Lpad = Lpad; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
     p.d_status = ctx.d_status;
     dim3 grid((unsigned)nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
     if (nseg == 1) {
         p.h_in = h0; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, p);
+        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
         ctx.end();
     } else {
-        float *states = (float *)workspace;
+        float *states = (float *)seg_ws;
         float *decay = states + (size_t)B * nseg * H * SP * SN;
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, p);
+        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
         ctx.end();
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
@@ -582,7 +680,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         ctx.end();
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, p);
+        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
         ctx.end();
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
