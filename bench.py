@@ -194,6 +194,8 @@ def main():
     ap.add_argument("--config", default="small_lm", choices=[c for c in synth.CONFIG_ORDER if c != "decode"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--decode-steps", type=int, default=512,
+                    help="consecutive steps timed by the decode leg (the workload has 512)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -319,7 +321,7 @@ def main():
 
     decode = None
     if rank == 0 and world == 1 and not args.no_decode:
-        decode = bench_decode(sb, pk)
+        decode = bench_decode(sb, pk, steps=args.decode_steps)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

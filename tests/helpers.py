@@ -76,7 +76,9 @@ def max_rel(got, ref) -> float:
 
 
 def check_routing(cfg: synth.LayerConfig, inp, idx_gpu, w_gpu, require_all_certified=False):
-    """Certified tokens must match exactly; returns (#ambiguous tokens, oracle router output)."""
+    """Certified tokens must match exactly; returns (#uncertified tokens, oracle router output).
+    r["mismatch"] counts the tokens (necessarily uncertified) whose routing differs from the
+    oracle's own."""
     F = cfg.F
     u2 = synth.f64(inp["u"]).reshape(-1, F)
     r = oracle.router(u2, synth.f64(inp["W_r"]), cfg.k)
@@ -88,6 +90,7 @@ def check_routing(cfg: synth.LayerConfig, inp, idx_gpu, w_gpu, require_all_certi
         certified[:] = True
     assert np.array_equal(idx_gpu[certified], r["idx"][certified]), "certified routing differs"
     n_amb = int((~certified).sum())
+    r["mismatch"] = int(np.any(idx_gpu != r["idx"], axis=-1).sum())
     if require_all_certified:
         assert n_amb == 0
     # ambiguous tokens must still pick k distinct valid experts
@@ -103,7 +106,7 @@ def check_routing(cfg: synth.LayerConfig, inp, idx_gpu, w_gpu, require_all_certi
 
 def compare_forward(cfg: synth.LayerConfig, inp, got, tol_y, tol_h, h0=None,
                     require_all_certified=False):
-    n_amb, _ = check_routing(cfg, inp, got["idx"], got["w"], require_all_certified)
+    n_amb, r0 = check_routing(cfg, inp, got["idx"], got["w"], require_all_certified)
     B, L = inp["u"].shape[:2]
     forced_idx = got["idx"].numpy().reshape(B, L, cfg.k)
     forced_w = None
@@ -118,7 +121,7 @@ def compare_forward(cfg: synth.LayerConfig, inp, got, tol_y, tol_h, h0=None,
     eh = max_rel(got["h_final"].double().numpy(), ref["h_final"])
     assert ey <= tol_y, f"y max-rel error {ey:.3e} > {tol_y}"
     assert eh <= tol_h, f"h_final max-rel error {eh:.3e} > {tol_h}"
-    return dict(err_y=ey, err_h=eh, ambiguous=n_amb, ref=ref)
+    return dict(err_y=ey, err_h=eh, ambiguous=n_amb, mismatch=r0["mismatch"], ref=ref)
 
 
 def tolerances(cfg: synth.LayerConfig):
