@@ -12,11 +12,12 @@
 namespace swimba {
 
 namespace {
-constexpr int GM_BM = 128;     // rows (token, slot pairs) per tile
+constexpr int GM_BM = 256;     // rows (token, slot pairs) per tile: two 128-row MMA halves that
+                               // share every weight tile
 constexpr int GM_BK = 64;      // features per pipeline stage (128 bytes of bf16)
-constexpr int GM_STAGES = 4;
 constexpr int GM_LAG = 2;      // cp.async groups kept in flight per gather thread
 constexpr int GM_THREADS = 192;
+__host__ __device__ constexpr int gm_stages(int BN) { return BN >= 256 ? 3 : 4; }
 }  // namespace
 
 // ------------------------------------------------------------------------------------------
@@ -30,39 +31,58 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
                    const int *__restrict__ counts, int E, int F, int S, int k,
                    __nv_bfloat16 *__restrict__ out, int *d_status)
 {
-    // Tile -> (expert, rows): tiles are numbered expert by expert, ceil(counts[e] / 128) each.
-    int e = 0, row0 = (int)blockIdx.x, cnt = 0;
-    for (; e < E; ++e) {
-        cnt = counts[e];
-        const int nt = (cnt + GM_BM - 1) / GM_BM;
-        if (row0 < nt) break;
-        row0 -= nt;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // Tile -> (expert, rows): tiles are numbered expert by expert, ceil(counts[e] / GM_BM) each.
+    // Every warp finds its tile with one load per lane and a shuffle scan.
+    int e = -1, row0 = 0, cnt = 0;
+    {
+        int before = 0;
+        for (int base = 0; base < E && e < 0; base += 32) {
+            const int c = (base + lane < E) ? counts[base + lane] : 0;
+            const int nt = (c + GM_BM - 1) / GM_BM;
+            int incl = nt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int nb = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += nb;
+            }
+            const unsigned hit = __ballot_sync(0xffffffffu, before + incl > (int)blockIdx.x);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                e = base + src;
+                cnt = __shfl_sync(0xffffffffu, c, src);
+                const int excl = __shfl_sync(0xffffffffu, incl - nt, src);
+                row0 = ((int)blockIdx.x - before - excl) * GM_BM;
+            }
+            before += __shfl_sync(0xffffffffu, incl, 31);
+        }
     }
-    if (e == E) return;
-    row0 *= GM_BM;
+    if (e < 0) return;
     const int nrows = min(GM_BM, cnt - row0);
+    const int nhalf = nrows > 128 ? 2 : 1;          // 128-row halves that hold rows
     perm += (int64_t)e * cap;
     const int n0 = blockIdx.y * BN;
+    constexpr int STAGES = gm_stages(BN);
     constexpr uint32_t A_BYTES = GM_BM * 128, B_BYTES = BN * 128;
-    constexpr uint32_t TMEM_COLS = BN < 32 ? 32 : BN;
+    constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sA = smem;
-    uint8_t *sB = smem + GM_STAGES * A_BYTES;
-    uint64_t *full = (uint64_t *)(sB + GM_STAGES * B_BYTES);
-    uint64_t *empty = full + GM_STAGES;
-    uint64_t *acc_bar = empty + GM_STAGES;
+    uint8_t *sB = smem + STAGES * A_BYTES;
+    uint64_t *full = (uint64_t *)(sB + STAGES * B_BYTES);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_bar = empty + STAGES;
     uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
     int *abort_flag = (int *)(tmem_slot + 1);
-    int *row_src = abort_flag + 1;            // [128] token index or -1
-    int *row_dst = row_src + GM_BM;           // [128] output row
+    int *row_src = abort_flag + 1;            // [256] token index or -1
+    int *row_dst = row_src + GM_BM;           // [256] output row
     float *row_w = (float *)(row_dst + GM_BM);
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int uwarp = __shfl_sync(0xffffffffu, warp, 0);   // warp-uniform for the compiler
 
     if (tid == 0) {
-        for (int s = 0; s < GM_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             tc::mbar_init(&full[s], 128 + 1);
             tc::mbar_init(&empty[s], 1);
         }
@@ -70,41 +90,45 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
         *abort_flag = 0;
         tc::fence_mbar_init();
     }
-    if (tid < GM_BM) {
-        if (tid < nrows) {
-            const int entry = perm[row0 + tid];
-            row_src[tid] = entry / k;
-            row_dst[tid] = entry;
-            row_w[tid] = w_slot[entry];
+    for (int r = tid; r < GM_BM; r += GM_THREADS) {
+        if (r < nrows) {
+            const int entry = perm[row0 + r];
+            row_src[r] = entry / k;
+            row_dst[r] = entry;
+            row_w[r] = w_slot[entry];
         } else {
-            row_src[tid] = -1;
-            row_dst[tid] = 0;
-            row_w[tid] = 0.f;
+            row_src[r] = -1;
+            row_dst[r] = 0;
+            row_w[r] = 0.f;
         }
     }
-    if (warp == 5) {
+    if (uwarp == 5) {
         tc::tmem_alloc(tmem_slot, TMEM_COLS);
         tc::tmem_relinquish();
     }
-    if (warp == 4 && lane == 0) tc::prefetch_tmap(&tmap_w);
+    if (uwarp == 4 && lane == 0) tc::prefetch_tmap(&tmap_w);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const int KB = ceil_div(F, GM_BK);
 
-    if (warp < 4) {
-        // ---- gather producers
+    if (uwarp < 4) {
+        // ---- gather producers: thread -> 16-byte chunk (lane & 7) of rows 4 i + (lane >> 3)
+        // of its warp's 64-row quarter
+        int tsrc[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) tsrc[i] = row_src[warp * 64 + i * 4 + (lane >> 3)];
         for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % GM_STAGES;
-            tc::mbar_wait(&empty[s], ((kb / GM_STAGES) & 1) ^ 1, abort_flag, d_status);
+            const int s = kb % STAGES;
+            tc::mbar_wait(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag, d_status);
             const uint32_t a_base = tc::smem_u32(sA + s * A_BYTES);
             const int chunk = lane & 7;
             const int f = kb * GM_BK + chunk * 8;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const int row = warp * 32 + i * 4 + (lane >> 3);
-                const int t = row_src[row];
+            for (int i = 0; i < 16; ++i) {
+                const int row = warp * 64 + i * 4 + (lane >> 3);
+                const int t = tsrc[i];
                 const bool ok = (t >= 0) && (f < F);
                 const __nv_bfloat16 *src = ok ? (u + (int64_t)t * F + f) : u;
                 tc::cp_async16(a_base + tc::sw128_offset(row, chunk), src, ok ? 16u : 0u);
@@ -113,70 +137,93 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
             if (kb >= GM_LAG) {
                 tc::cp_async_wait<GM_LAG>();
                 tc::fence_proxy_async_smem();
-                tc::mbar_arrive(&full[(kb - GM_LAG) % GM_STAGES]);
+                tc::mbar_arrive(&full[(kb - GM_LAG) % STAGES]);
             }
         }
         tc::cp_async_wait<0>();
         tc::fence_proxy_async_smem();
         for (int kb = (KB > GM_LAG ? KB - GM_LAG : 0); kb < KB; ++kb)
-            tc::mbar_arrive(&full[kb % GM_STAGES]);
+            tc::mbar_arrive(&full[kb % STAGES]);
 
-        // ---- epilogue: thread = output row
+        // ---- epilogue: thread = output row of each half.  All MMAs have completed, so the
+        // pipeline buffers are free: the scaled bf16 rows are staged there (row stride padded by
+        // 16 bytes against bank conflicts) and leave as one bulk copy per row.
         tc::mbar_wait(acc_bar, 0, abort_flag, d_status);
         tc::tc_fence_after();
-        const int row = warp * 32 + lane;
-        const bool valid = row < nrows;
-        const float wr = row_w[row];
-        __nv_bfloat16 *orow = out + (int64_t)row_dst[row] * S + n0;
+        constexpr uint32_t ROW_STRIDE = BN * 2 + 16;
+        for (int hf = 0; hf < nhalf; ++hf) {
+            const int row = hf * 128 + warp * 32 + lane;
+            const float wr = row_w[row];
+            uint8_t *srow = smem + (uint32_t)row * ROW_STRIDE;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-            uint32_t v[32];
-            tc::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + c * 32, v);
-            tc::tmem_ld_wait();
-            if (valid) {
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_base + ((uint32_t)(warp * 32) << 16) + hf * BN + c * 32, v);
+                tc::tmem_ld_wait();
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
                     pk[i] = tc::pack_bf16x2(wr * __uint_as_float(v[2 * i]),
                                             wr * __uint_as_float(v[2 * i + 1]));
-                uint4 *dst = reinterpret_cast<uint4 *>(orow + c * 32);
+                uint4 *dst = reinterpret_cast<uint4 *>(srow + c * 64);
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
             }
         }
-    } else if (warp == 4) {
-        if (lane == 0) {
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % GM_STAGES;
-                tc::mbar_wait(&empty[s], ((kb / GM_STAGES) & 1) ^ 1, abort_flag, d_status);
+        tc::fence_proxy_async_smem();
+        for (int hf = 0; hf < nhalf; ++hf) {
+            const int row = hf * 128 + warp * 32 + lane;
+            if (row < nrows)
+                tc::bulk_store(out + (int64_t)row_dst[row] * S + n0, smem + (uint32_t)row * ROW_STRIDE,
+                               BN * 2);
+        }
+        tc::bulk_commit_group();
+        tc::bulk_wait_read_all();
+    } else if (uwarp == 4) {
+        // ---- weight tiles by TMA (whole warp in the loop, one elected lane issues)
+        const bool leader = tc::elect_one();
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % STAGES;
+            tc::mbar_wait(&empty[s], ((kb / STAGES) & 1) ^ 1, abort_flag, d_status);
+            if (leader) {
                 tc::mbar_arrive_expect_tx(&full[s], B_BYTES);
                 tc::tma_load_3d(sB + s * B_BYTES, &tmap_w, &full[s], kb * GM_BK, n0, e);
             }
+            __syncwarp();
         }
     } else {
-        if (lane == 0) {
-            constexpr uint32_t idesc = tc::idesc_bf16(GM_BM, BN, 0, 0);
-            for (int kb = 0; kb < KB; ++kb) {
-                const int s = kb % GM_STAGES;
-                tc::mbar_wait(&full[s], (kb / GM_STAGES) & 1, abort_flag, d_status);
-                tc::tc_fence_after();
-                const uint32_t a_addr = tc::smem_u32(sA + s * A_BYTES);
-                const uint32_t b_addr = tc::smem_u32(sB + s * B_BYTES);
+        // ---- MMA issue (whole warp in the loop, one elected lane issues)
+        const bool leader = tc::elect_one();
+        constexpr uint32_t idesc = tc::idesc_bf16(128, BN, 0, 0);
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint64_t dA0 = tc::smem_desc_sw128(tc::smem_u32(sA), 16, 1024);
+        const uint64_t dB0 = tc::smem_desc_sw128(tc::smem_u32(sB), 16, 1024);
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % STAGES;
+            tc::mbar_wait(&full[s], (kb / STAGES) & 1, abort_flag, d_status);
+            tc::tc_fence_after();
+            if (leader) {
+                const uint64_t dA = tc::smem_desc_advance(dA0, s * A_BYTES);
+                const uint64_t dB = tc::smem_desc_advance(dB0, s * B_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < GM_BK / 16; ++kk) {
-                    const uint64_t ad = tc::smem_desc_sw128(a_addr + kk * 32, 16, 1024);
-                    const uint64_t bd = tc::smem_desc_sw128(b_addr + kk * 32, 16, 1024);
-                    tc::mma_ss(tmem_base, ad, bd, idesc, (kb | kk) != 0);
+                    const uint64_t bd = tc::smem_desc_advance(dB, kk * 32);
+                    tc::mma_ss(tmem_u, tc::smem_desc_advance(dA, kk * 32), bd, idesc, (kb | kk) != 0);
+                    if (nhalf > 1)
+                        tc::mma_ss(tmem_u + BN, tc::smem_desc_advance(dA, 128 * 128 + kk * 32), bd, idesc,
+                                   (kb | kk) != 0);
                 }
                 tc::mma_commit(&empty[s]);
             }
-            tc::mma_commit(acc_bar);
+            __syncwarp();
         }
+        if (leader) tc::mma_commit(acc_bar);
+        __syncwarp();
     }
     tc::tc_fence_before();
     __syncthreads();
-    if (warp == 5) tc::tmem_dealloc(tmem_base, TMEM_COLS);
+    if (uwarp == 5) tc::tmem_dealloc(tmem_base, TMEM_COLS);
 }
 
 // BC[t, :] = sum_j P[t*k + j, :]   (slots already carry their router weight).
@@ -205,7 +252,8 @@ mix_slots_kernel(const __nv_bfloat16 *__restrict__ P, int64_t T, int S, int k,
 
 static size_t gemm_smem_bytes(int BN)
 {
-    return 1024 + GM_STAGES * (GM_BM * 128 + BN * 128) + 8 * (2 * GM_STAGES + 1) + 16 +
+    const int stages = gm_stages(BN);
+    return 1024 + (size_t)stages * (GM_BM * 128 + BN * 128) + 8 * (2 * stages + 1) + 16 +
            GM_BM * 12 + 64;
 }
 

@@ -107,6 +107,13 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, const void *s
         "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// Plain bulk copy shared -> global of `bytes` (a multiple of 16, both addresses 16-byte aligned),
+// tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void bulk_store(void *dst_global, const void *src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst_global),
+                 "r"(smem_u32(src_smem)), "r"(bytes)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the issuing thread's bulk stores have finished READING shared memory.
 __device__ __forceinline__ void bulk_wait_read_all() {
