@@ -33,7 +33,13 @@ NSETS = 4   # rotating input sets: together several times the 126 MB L2
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel from the ncu
 # captures summarised under profiles/; None until a capture of that kernel exists.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # workload small_lm, one launch each (profiles/forward_small_lm_kernels.md); ncu flushes caches
+    # before a launch and part of a kernel's writes can still sit in L2 when it ends
+    "ssd_tiles": 77.590e6, "router_topk": 25.224e6, "mix_slots": 16.792e6, "ssd_scalars": 1.578e6,
+    # decode workload (profiles/decode_update_kernel.md)
+    "decode_update": 479.7e6,
+}
 
 
 def peaks():
@@ -112,9 +118,8 @@ def algorithmic_work(cfg: synth.LayerConfig):
     ssd_bytes = T * (2 * H * P * es + S * es + H * 4) + cfg.B * H * P * N * 4
     w["ssd_tiles"] = dict(bound="tensor", work=ssd_flops, bytes=ssd_bytes)
     w["ssd_sequential"] = dict(bound="alu", work=4.0 * T * H * P * N, bytes=ssd_bytes)
-    w["scatter_rows"] = dict(bound="hbm", work=T * k * 8)
-    w["tile_table"] = dict(bound="hbm", work=E * 16)
     w["segment_scan"] = dict(bound="hbm", work=0)
+    w["ssd_scalars"] = dict(bound="hbm", work=T * H * 12)
     return w
 
 
@@ -122,6 +127,21 @@ def roofline_entry(name, avg_ms, work, pk):
     info = work.get(name)
     if info is None or avg_ms <= 0:
         return None
+    if name == "ssd_tiles":
+        # both roofs are close: report the one that binds (the larger ideal time), keep the other
+        t_hbm = info["bytes"] / (pk["hbm_gbs"] * 1e9)
+        t_tc = info["work"] / (pk["bf16_tflops"] * 1e12)
+        ach_b = info["bytes"] / (avg_ms * 1e-3) / 1e9
+        ach_f = info["work"] / (avg_ms * 1e-3) / 1e12
+        ent = dict(kernel=name, traffic=NCU_TRAFFIC_BYTES.get(name), peak_source=pk["source"],
+                   avg_ms=avg_ms, hbm_frac=ach_b / pk["hbm_gbs"], tensor_frac=ach_f / pk["bf16_tflops"])
+        if t_hbm >= t_tc:
+            ent.update(bound="hbm", achieved=ach_b, peak=pk["hbm_gbs"], unit="GB/s",
+                       frac=ach_b / pk["hbm_gbs"])
+        else:
+            ent.update(bound="tensor", achieved=ach_f, peak=pk["bf16_tflops"], unit="TFLOP/s",
+                       frac=ach_f / pk["bf16_tflops"])
+        return ent
     if info["bound"] == "hbm":
         ach = info["work"] / (avg_ms * 1e-3) / 1e9
         peak, unit = pk["hbm_gbs"], "GB/s"
@@ -150,6 +170,56 @@ def time_oracle_sample(cfg: synth.LayerConfig, n_seq: int, seed: int = 0):
     return dict(value=sub.tokens / dt, unit=UNIT, cores=oracle.num_threads(), kind="oracle",
                 sample=f"{n_seq} of {cfg.B} sequences x {cfg.L} tokens of {cfg.name}, fp64, "
                        f"{dt:.2f} s"), dt
+
+
+def time_layer(sb, cfg, steps, warmup, n_sets=2, seed0=5000, repeat=1):
+    """ms per forward of one layer configuration through swimba_forward (device-resident inputs)."""
+    dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
+    sets = [synth.make_inputs(cfg, seed=seed0 + i) for i in range(n_sets)]
+    wts = {n: sets[0][n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    dev = [dict(u=s_["u"].cuda(), x=s_["x"].cuda(), dt=s_["dt"].cuda()) for s_ in sets]
+    y = torch.empty_like(dev[0]["x"])
+    hf = torch.empty(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
+    ws = torch.empty(sb.swimba_workspace_bytes(h, cfg.B, cfg.L), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        d = dev[i % n_sets]
+        for _ in range(repeat):
+            sb.swimba_forward(h, w, d["u"], d["x"], d["dt"], None, cfg.B, cfg.L, y, hf, None, None, ws)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    return e0.elapsed_time(e1) / steps
+
+
+def bench_comparators(sb, cfg, steps, warmup, ms_swimba):
+    """The same shape as (1) a dense Mamba-2 layer: the library with E = k = 1 (no router, one
+    projection), and (2) E separated SSMs: every expert's streams projected for every token and E
+    independent SSD evaluations with E states (the readout sum over the active experts is left
+    out, so the figure is a lower bound of that design's cost)."""
+    import dataclasses
+    dense = dataclasses.replace(cfg, name=cfg.name + "_dense", E=1, k=1)
+    ms_dense = time_layer(sb, dense, steps, warmup)
+    ms_sep = time_layer(sb, dense, steps, warmup, repeat=cfg.E)
+    return {
+        "dense_mamba2": {"ms_per_step": ms_dense, "swimba_over_dense": ms_swimba / ms_dense,
+                         "how": "same library, E = k = 1"},
+        "separated_ssm_E_fold": {"ms_per_step": ms_sep, "swimba_over_separated": ms_swimba / ms_sep,
+                                 "how": f"{cfg.E} dense-layer passes back to back (one projection "
+                                        f"and one SSD evaluation per expert), readout sum not counted"},
+    }
 
 
 def run_reference(args, cfg, rank, world):
@@ -197,6 +267,7 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=512,
                     help="consecutive steps timed by the decode leg (the workload has 512)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-comparators", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = synth.CONFIGS[args.config]
@@ -323,9 +394,13 @@ def main():
     if rank == 0 and world == 1 and not args.no_decode:
         decode = bench_decode(sb, pk, steps=args.decode_steps)
 
+    comparators = None
+    if rank == 0 and world == 1 and not args.no_comparators:
+        comparators = bench_comparators(sb, cfg, args.steps, args.warmup, ms_step)
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu, _ = time_oracle_sample(cfg, min(cfg.B, 4))
+        cpu, _ = time_oracle_sample(cfg, cfg.B)
 
     if rank == 0:
         out = {
@@ -334,7 +409,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
             "data": "synthetic", "config": config_dict(cfg), "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
-            "kernels": kernels, "decode": decode, "cpu_baseline": cpu,
+            "kernels": kernels, "decode": decode, "comparators": comparators, "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     if dist is not None:

@@ -294,7 +294,7 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
     // GPU (decode-sized calls), so that the weight rows are spread over more SMs.
     int BN = 32;
     for (int c : {256, 128, 64}) if (S % c == 0) { BN = c; break; }
-    while (BN > 32 && (int64_t)max_tiles * (S / BN) < sm_count) BN >>= 1;
+    while (BN > 32 && 2 * (int64_t)max_tiles * (S / BN) <= sm_count) BN >>= 1;
 
     CUtensorMap tmap;
     const uint64_t dims[3] = {(uint64_t)F, (uint64_t)S, (uint64_t)E};
