@@ -74,6 +74,33 @@ __device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8]) {
     }
 }
 
+// The same eight elements as raw registers (so that a load can be issued well before its use) and
+// their widening to fp32.
+struct Raw8f { float4 a, b; };
+struct Raw8h { uint4 a; };
+__device__ __forceinline__ void load_raw8(const float *p, Raw8f &r) {
+    r.a = *reinterpret_cast<const float4 *>(p);
+    r.b = *reinterpret_cast<const float4 *>(p + 4);
+}
+__device__ __forceinline__ void load_raw8(const __nv_bfloat16 *p, Raw8h &r) {
+    r.a = *reinterpret_cast<const uint4 *>(p);
+}
+__device__ __forceinline__ void unpack8(const Raw8f &r, float (&v)[8]) {
+    v[0] = r.a.x; v[1] = r.a.y; v[2] = r.a.z; v[3] = r.a.w;
+    v[4] = r.b.x; v[5] = r.b.y; v[6] = r.b.z; v[7] = r.b.w;
+}
+__device__ __forceinline__ void unpack8(const Raw8h &r, float (&v)[8]) {
+    const uint32_t w[4] = {r.a.x, r.a.y, r.a.z, r.a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+template <typename T> struct Raw8;
+template <> struct Raw8<float> { typedef Raw8f type; };
+template <> struct Raw8<__nv_bfloat16> { typedef Raw8h type; };
+
 // Butterfly sum over the 32 lanes; every lane ends with the same bits.
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -56,18 +56,28 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
         const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
         if (threadIdx.x < SWIMBA_MAX_EXPERTS) s_cnt[threadIdx.x] = 0;
         __syncthreads();
+        // The feature loads run one step ahead of the arithmetic, across passes too: `raw` always
+        // holds the next 8-feature slice of the next TPW tokens.
+        typename Raw8<T>::type raw[TPW];
+        auto prefetch = [&](int64_t tt0, int ff) {
+#pragma unroll
+            for (int q = 0; q < TPW; ++q) {
+                const int64_t t = (tt0 + q < tend) ? tt0 + q : tt0;
+                load_raw8(u + t * F + ff, raw[q]);
+            }
+        };
+        if (tbeg + warp * TPW < tend && lane * 8 < F) prefetch(tbeg + warp * TPW, lane * 8);
         for (int64_t t0 = tbeg + warp * TPW; t0 < tend; t0 += nwarp * TPW) {
             float g[V];                                  // g[q * EP + e]
 #pragma unroll
             for (int i = 0; i < V; ++i) g[i] = 0.f;
-#pragma unroll 2
+#pragma unroll 1
             for (int f = lane * 8; f < F; f += 256) {
                 float uv[TPW][8];
 #pragma unroll
-                for (int q = 0; q < TPW; ++q) {
-                    const int64_t t = (t0 + q < tend) ? t0 + q : t0;
-                    load8(u + t * F + f, uv[q]);
-                }
+                for (int q = 0; q < TPW; ++q) unpack8(raw[q], uv[q]);
+                if (f + 256 < F) prefetch(t0, f + 256);
+                else if (t0 + nwarp * TPW < tend) prefetch(t0 + nwarp * TPW, lane * 8);
 #pragma unroll
                 for (int e = 0; e < EP; ++e) {
                     if (e < E) {
@@ -194,8 +204,8 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
     const size_t w_bytes = (size_t)E * F * sizeof(T);
     const int stage_w = (w_bytes <= 64 * 1024 && (w_bytes & 15) == 0) ? 1 : 0;
     const size_t smem = (size_t)ROUTER_MAX_CHUNK * SWIMBA_MAX_TOPK * sizeof(int) + (stage_w ? w_bytes : 0);
-    // chunk: enough chunks to give every SM two blocks, between 32 and ROUTER_MAX_CHUNK tokens
-    int chunk = (int)(Ttok / (2 * (int64_t)sm_count));
+    // chunk: enough chunks to give every SM four blocks, between 32 and ROUTER_MAX_CHUNK tokens
+    int chunk = (int)(Ttok / (4 * (int64_t)sm_count));
     chunk = (chunk + 31) / 32 * 32;
     if (chunk < 32) chunk = 32;
     if (chunk > ROUTER_MAX_CHUNK) chunk = ROUTER_MAX_CHUNK;
