@@ -135,7 +135,10 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
 /* End-to-end variant of swimba_forward for callers whose activations live in HOST memory
  * (pinned memory makes the copies asynchronous): copies u_host, x_host, dt_host (may be NULL)
  * to device staging, runs the forward of Theorem 1, copies y (and h_final / topk outputs when
- * given) back, all on the given stream; the caller synchronises the stream before reading.
+ * given) back; the batch goes through in up to eight slices of whole sequences so that the copies
+ * in, the kernels and the copies out of successive slices overlap (two copy streams owned by the
+ * handle, the kernels on the given stream).  The given stream ends after the last copy out: the
+ * caller synchronises it before reading.
  * Weights stay device pointers.  The workspace holds the staging buffers as well and is sized
  * by swimba_host_workspace_bytes. */
 size_t swimba_host_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);

@@ -15,6 +15,9 @@ struct swimba_handle {
     cudaStream_t last_stream;
     int last_launches;
     Profiler prof;
+    // host-buffer entry point: copy streams and events of its batch-slice pipeline
+    cudaStream_t s_in, s_out;
+    cudaEvent_t ev_start, ev_out, ev_in[8], ev_done[8];
     char err[256];
 };
 
@@ -79,6 +82,21 @@ DecLayout dec_layout(const swimba_config &c, int B)
 struct HostLayout {
     size_t u, x, dt, y, hf, idx, w, fwd, total;
 };
+constexpr int kHostSlices = 8;     // batch slices of the host-buffer pipeline (at most)
+// Sequences per slice.  Slices start at whole sequences inside the staged tensors, so every
+// per-sequence size has to keep the 16-byte alignment; otherwise the batch goes as one slice.
+inline int host_slice_seqs(const swimba_config &c, int B, int L)
+{
+    const size_t es = elt_size(c.dtype);
+    const size_t per_seq[5] = {(size_t)L * c.d_model * es, (size_t)L * c.n_heads * c.head_dim * es,
+                               (size_t)L * c.n_heads * sizeof(float),
+                               (size_t)L * c.top_k * sizeof(int32_t),
+                               (size_t)c.n_heads * c.head_dim * c.d_state * sizeof(float)};
+    for (size_t v : per_seq)
+        if (v % 16 != 0) return B;
+    return (B + kHostSlices - 1) / kHostSlices;
+}
+
 HostLayout host_layout(const swimba_config &c, int B, int L, int sm_count)
 {
     HostLayout l;
@@ -92,7 +110,8 @@ HostLayout host_layout(const swimba_config &c, int B, int L, int sm_count)
     l.hf = off;  off += align_up((size_t)B * HP * c.d_state * sizeof(float));
     l.idx = off; off += align_up(T * c.top_k * sizeof(int32_t));
     l.w = off;   off += align_up(T * c.top_k * sizeof(float));
-    l.fwd = off; off += fwd_layout(c, B, L, sm_count).total;
+    // the forward runs slice by slice on the same scratch
+    l.fwd = off; off += fwd_layout(c, host_slice_seqs(c, B, L), L, sm_count).total;
     l.total = off;
     return l;
 }
@@ -111,6 +130,30 @@ int check_weights(swimba_handle *h, const swimba_weights *w, bool need_experts)
     if (!aligned16(w->A) || !aligned16(w->dt_bias) || !aligned16(w->D))
         return fail(h, SWIMBA_ERR_MISALIGNED, "A/dt_bias/D must be 16-byte aligned");
     return SWIMBA_OK;
+}
+
+bool create_host_pipeline(swimba_handle *h)
+{
+    bool ok = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < 8; ++i)
+        ok = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
+    return ok;
+}
+
+void destroy_host_pipeline(swimba_handle *h)
+{
+    if (h->s_in) cudaStreamDestroy(h->s_in);
+    if (h->s_out) cudaStreamDestroy(h->s_out);
+    if (h->ev_start) cudaEventDestroy(h->ev_start);
+    if (h->ev_out) cudaEventDestroy(h->ev_out);
+    for (int i = 0; i < 8; ++i) {
+        if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
+        if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
+    }
 }
 
 int set_device(swimba_handle *h)
@@ -199,7 +242,9 @@ int swimba_create(const swimba_config *cfg, swimba_handle **out)
     h->cfg = c;
     if (cudaGetDevice(&h->device) != cudaSuccess ||
         cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device) != cudaSuccess ||
-        cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess) {
+        cudaMalloc(&h->d_status, 64) != cudaSuccess || cudaMemset(h->d_status, 0, 64) != cudaSuccess ||
+        !create_host_pipeline(h)) {
+        destroy_host_pipeline(h);
         if (h->d_status) cudaFree(h->d_status);
         delete h;
         cudaGetLastError();
@@ -368,28 +413,62 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
     int rc = check_weights(h, w, true);
     if (rc != SWIMBA_OK) return rc;
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    // Batch slices flow through three streams: copies in (s_in), kernels (the caller's stream),
+    // copies out (s_out), so that the host-to-device copy of slice i+1 and the device-to-host
+    // copy of slice i-1 overlap the kernels of slice i.  Sequences are independent, so a slice is
+    // a forward call of its own on the staged tensors.
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char *ws = (char *)workspace;
-    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const size_t es = elt_size(c.dtype);
     const size_t HP = (size_t)c.n_heads * c.head_dim;
-    bool ok = cudaMemcpyAsync(ws + l.u, u_host, T * c.d_model * es, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(ws + l.x, x_host, T * HP * es, cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (dt_host)
-        ok = ok && cudaMemcpyAsync(ws + l.dt, dt_host, T * c.n_heads * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "host-to-device copy failed"); }
-    rc = swimba_forward(h, w, ws + l.u, ws + l.x, dt_host ? (const float *)(ws + l.dt) : nullptr,
-                        nullptr, B, L, ws + l.y, h_final_host ? (float *)(ws + l.hf) : nullptr,
-                        (int32_t *)(ws + l.idx), (float *)(ws + l.w), ws + l.fwd,
-                        workspace_bytes - l.fwd, cuda_stream);
-    if (rc != SWIMBA_OK) return rc;
-    ok = cudaMemcpyAsync(y_host, ws + l.y, T * HP * es, cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (h_final_host)
-        ok = ok && cudaMemcpyAsync(h_final_host, ws + l.hf, (size_t)B * HP * c.d_state * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (topk_idx_host)
-        ok = ok && cudaMemcpyAsync(topk_idx_host, ws + l.idx, T * c.top_k * sizeof(int32_t), cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (topk_w_host)
-        ok = ok && cudaMemcpyAsync(topk_w_host, ws + l.w, T * c.top_k * sizeof(float), cudaMemcpyDeviceToHost, st) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "device-to-host copy failed"); }
+    const size_t tok_u = (size_t)c.d_model * es, tok_x = HP * es, tok_dt = c.n_heads * sizeof(float);
+    const size_t seq_hf = HP * c.d_state * sizeof(float);
+    const size_t tok_k = (size_t)c.top_k * sizeof(int32_t);
+    const int bs = host_slice_seqs(c, B, L);
+    bool ok = cudaEventRecord(h->ev_start, st) == cudaSuccess &&
+              cudaStreamWaitEvent(h->s_in, h->ev_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(h->s_out, h->ev_start, 0) == cudaSuccess;
+    int launches = 0, slice = 0;
+    for (int b0 = 0; ok && b0 < B; b0 += bs, ++slice) {
+        const int nb = (B - b0 < bs) ? B - b0 : bs;
+        const size_t t0 = (size_t)b0 * L, nt = (size_t)nb * L;
+        ok = cudaMemcpyAsync(ws + l.u + t0 * tok_u, (const char *)u_host + t0 * tok_u, nt * tok_u,
+                             cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
+             cudaMemcpyAsync(ws + l.x + t0 * tok_x, (const char *)x_host + t0 * tok_x, nt * tok_x,
+                             cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+        if (ok && dt_host)
+            ok = cudaMemcpyAsync(ws + l.dt + t0 * tok_dt, (const char *)dt_host + t0 * tok_dt, nt * tok_dt,
+                                 cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+        ok = ok && cudaEventRecord(h->ev_in[slice], h->s_in) == cudaSuccess &&
+             cudaStreamWaitEvent(st, h->ev_in[slice], 0) == cudaSuccess;
+        if (!ok) break;
+        rc = swimba_forward(h, w, ws + l.u + t0 * tok_u, ws + l.x + t0 * tok_x,
+                            dt_host ? (const float *)(ws + l.dt + t0 * tok_dt) : nullptr, nullptr, nb, L,
+                            ws + l.y + t0 * tok_x,
+                            h_final_host ? (float *)(ws + l.hf + (size_t)b0 * seq_hf) : nullptr,
+                            (int32_t *)(ws + l.idx + t0 * tok_k), (float *)(ws + l.w + t0 * tok_k),
+                            ws + l.fwd, workspace_bytes - l.fwd, cuda_stream);
+        if (rc != SWIMBA_OK) return rc;
+        launches += h->last_launches;
+        ok = cudaEventRecord(h->ev_done[slice], st) == cudaSuccess &&
+             cudaStreamWaitEvent(h->s_out, h->ev_done[slice], 0) == cudaSuccess &&
+             cudaMemcpyAsync((char *)y_host + t0 * tok_x, ws + l.y + t0 * tok_x, nt * tok_x,
+                             cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+        if (ok && h_final_host)
+            ok = cudaMemcpyAsync((char *)h_final_host + (size_t)b0 * seq_hf, ws + l.hf + (size_t)b0 * seq_hf,
+                                 (size_t)nb * seq_hf, cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+        if (ok && topk_idx_host)
+            ok = cudaMemcpyAsync((char *)topk_idx_host + t0 * tok_k, ws + l.idx + t0 * tok_k, nt * tok_k,
+                                 cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+        if (ok && topk_w_host)
+            ok = cudaMemcpyAsync((char *)topk_w_host + t0 * tok_k, ws + l.w + t0 * tok_k, nt * tok_k,
+                                 cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+    }
+    // the caller's stream ends after the last copy out: synchronising it is enough
+    ok = ok && cudaEventRecord(h->ev_out, h->s_out) == cudaSuccess &&
+         cudaStreamWaitEvent(st, h->ev_out, 0) == cudaSuccess;
+    h->last_launches = launches;
+    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "a copy or an event of the host pipeline failed"); }
     return SWIMBA_OK;
 }
 
@@ -445,6 +524,7 @@ void swimba_destroy(swimba_handle *h)
 {
     if (!h) return;
     if (h->d_status) cudaFree(h->d_status);
+    destroy_host_pipeline(h);
     if (h->prof.ev[0])
         for (int i = 0; i < 2 * PROF_MAX; ++i) if (h->prof.ev[i]) cudaEventDestroy(h->prof.ev[i]);
     delete h;

@@ -271,7 +271,12 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     idx = torch.empty(B, L, cfg.k, dtype=torch.int32).pin_memory()
     sb.swimba_forward_host(h, w, u, x, dt, B, L, y, hf, idx, None, ws)
     assert sb.swimba_status(h) == 0
-    assert torch.equal(y.view(torch.int16), dev_out["y"].view(torch.int16))
-    assert torch.equal(hf, dev_out["h_final"])
+    # the host path runs the batch in slices; a slice may be cut into other SSD segments than the
+    # whole batch, so the floats agree within the parity tolerance, the routing exactly
+    assert hp.max_rel(y.double().numpy(), dev_out["y"].double().numpy()) <= 2e-2
+    assert hp.max_rel(hf.numpy(), dev_out["h_final"].numpy()) <= 1e-2
     assert torch.equal(idx, dev_out["idx"])
+    ref = hp.oracle_forward(cfg, inp)
+    assert hp.max_rel(y.double().numpy(), ref["y"]) <= 2e-2
+    assert hp.max_rel(hf.double().numpy(), ref["h_final"]) <= 1e-2
     sb.swimba_destroy(h)
