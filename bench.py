@@ -25,7 +25,7 @@ if ROOT not in sys.path:
 
 import torch
 
-from paper_2603_06938_b200 import synth
+from paper_2603_06938_b200 import replicas, synth
 
 METRIC = "swimba_layer_fwd_tokens_per_s"
 UNIT = "tokens/s"
@@ -271,9 +271,7 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = synth.CONFIGS[args.config]
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.rank_env()
 
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
@@ -290,7 +288,7 @@ def main():
     pk = peaks()
     dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
     h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
-    sets = [synth.make_inputs(cfg, seed=1000 * rank + i) for i in range(NSETS)]
+    sets = [synth.make_inputs(cfg, seed=replicas.replica_seed(rank, i)) for i in range(NSETS)]
     wts = {n: sets[0][n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
     w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
     dev_sets = [dict(u=s["u"].cuda(), x=s["x"].cuda(), dt=s["dt"].cuda()) for s in sets]
@@ -325,14 +323,10 @@ def main():
         step(i)
     e1.record(stream)
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
     ms_step = ms_total / args.steps
-    value = world * cfg.tokens / (ms_step * 1e-3)
+    value = replicas.whole_job_throughput(world, cfg.tokens, ms_step)
 
     # per-kernel durations, live, same launch configuration (CUDA events around every kernel)
     sb.swimba_profile(h, True)
@@ -377,15 +371,11 @@ def main():
         sb.swimba_forward_host(h, w, s["u"], s["x"], s["dt"], B, L, y_host, None, None, None, hws)
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
     es = 2 if cfg.dtype == "bf16" else 4
     h2d = cfg.tokens * (cfg.F * es + cfg.H * cfg.P * es + cfg.H * 4)
     d2h = cfg.tokens * cfg.H * cfg.P * es
-    e2e = {"value": world * cfg.tokens / (e2e_ms / args.steps * 1e-3), "unit": UNIT,
+    e2e = {"value": replicas.whole_job_throughput(world, cfg.tokens, e2e_ms / args.steps), "unit": UNIT,
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     sb.swimba_destroy(h)
     del dev_sets, hws, ws, y, hf
