@@ -99,7 +99,8 @@ size_t swimba_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
  *   topk_idx [B,L,k]   int32  out, may be NULL: active experts, largest weight first, ties
  *                             to the lower expert index
  *   topk_w   [B,L,k]   float  out, may be NULL: their softmax values
- * L need not be a multiple of the chunk length.  B == 0 or L == 0 is a no-op returning OK. */
+ * L need not be a multiple of the chunk length.  B == 0 or L == 0 is a no-op returning OK.
+ * Limits: B <= 65535 and B*L*k < 2^31 (SWIMBA_ERR_UNSUPPORTED_SHAPE beyond them). */
 int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
                    const float *dt, const float *h0, int32_t B, int32_t L, void *y,
                    float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,

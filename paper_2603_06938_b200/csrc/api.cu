@@ -278,7 +278,9 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
 {
     if (!h) return SWIMBA_ERR_NULL_ARG;
     h->err[0] = 0;
-    if (T < 0 || T > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range");
+    // (token, slot) entries are indexed with 32-bit integers
+    if (T < 0 || T * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range (T * top_k must stay below 2^31)");
     int rc = check_weights(h, w, true);
     if (rc != SWIMBA_OK) return rc;
     if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
@@ -306,6 +308,7 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
     if (!h) return SWIMBA_ERR_NULL_ARG;
     h->err[0] = 0;
     if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
     int rc = check_weights(h, w, false);
     if (rc != SWIMBA_OK) return rc;
     if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
@@ -332,7 +335,9 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     if (!h) return SWIMBA_ERR_NULL_ARG;
     h->err[0] = 0;
     if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
-    if ((int64_t)B * L > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens");
+    if ((int64_t)B * L * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (B * L * top_k must stay below 2^31)");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
     int rc = check_weights(h, w, true);
     if (rc != SWIMBA_OK) return rc;
     if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
@@ -556,7 +561,9 @@ extern "C" int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w
 {
     if (!h) return SWIMBA_ERR_NULL_ARG;
     h->err[0] = 0;
-    if (T < 0 || T > (int64_t)1 << 31) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range");
+    // (token, slot) entries are indexed with 32-bit integers
+    if (T < 0 || T * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range (T * top_k must stay below 2^31)");
     if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
     int rc = set_device(h);
     if (rc != SWIMBA_OK) return rc;
