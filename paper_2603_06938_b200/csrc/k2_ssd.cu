@@ -572,15 +572,30 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
     if (v >= PN4) return;
     float4 run = h0 ? reinterpret_cast<const float4 *>(h0)[((int64_t)b * H + h) * PN4 + v]
                     : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < nseg; ++s) {
-        float4 *p = reinterpret_cast<float4 *>(states) + (((int64_t)b * nseg + s) * H + h) * PN4 + v;
-        const float4 loc = *p;
-        const float d = seg_decay[((int64_t)b * nseg + s) * H + h];
-        *p = run;
-        run.x = fmaf(d, run.x, loc.x);
-        run.y = fmaf(d, run.y, loc.y);
-        run.z = fmaf(d, run.z, loc.z);
-        run.w = fmaf(d, run.w, loc.w);
+    // the loads do not depend on the running state: four segments are fetched at a time
+    constexpr int U = 4;
+    for (int s0 = 0; s0 < nseg; s0 += U) {
+        float4 loc[U];
+        float d[U];
+#pragma unroll
+        for (int q = 0; q < U; ++q) {
+            const int s = s0 + q;
+            if (s < nseg) {
+                loc[q] = reinterpret_cast<const float4 *>(states)[(((int64_t)b * nseg + s) * H + h) * PN4 + v];
+                d[q] = seg_decay[((int64_t)b * nseg + s) * H + h];
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < U; ++q) {
+            const int s = s0 + q;
+            if (s < nseg) {
+                reinterpret_cast<float4 *>(states)[(((int64_t)b * nseg + s) * H + h) * PN4 + v] = run;
+                run.x = fmaf(d[q], run.x, loc[q].x);
+                run.y = fmaf(d[q], run.y, loc[q].y);
+                run.z = fmaf(d[q], run.z, loc[q].z);
+                run.w = fmaf(d[q], run.w, loc[q].w);
+            }
+        }
     }
 }
 
@@ -598,7 +613,10 @@ int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count)
     const int64_t ctas = (int64_t)B * G * pairs_per_group(H, G);
     const int tiles = ceil_div(L, ST);
     if (2 * ctas > sm_count || tiles <= 2) return tiles * ST;
-    int want = (int)ceil_div64(2 * (int64_t)sm_count, ctas);          // segments per sequence
+    // segments per sequence: as many as keep the grid within two CTAs per SM (a few CTAs more
+    // would cost a whole extra round)
+    int want = (int)((2 * (int64_t)sm_count) / ctas);
+    if (want < 1) want = 1;
     int q_tiles = chunk >= ST ? chunk / ST : 1;                       // segments are whole chunks
     int seg_tiles = ceil_div(tiles, want);
     seg_tiles = ceil_div(seg_tiles, q_tiles) * q_tiles;
