@@ -400,19 +400,29 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             const float Lw = wq == 0 ? 0.f : (wq == 1 ? L1 : (wq == 2 ? L2 : L3));    // l before my block
             const float w_s = delta * tc::ex2_approx(l2_last - l2);
 
-            // ---- w . X  (row i of the X slab -> row i of the X' slab, this thread's half)
+            // ---- w . X  (rows of the X slab -> rows of the X' slab, this thread's half of the
+            // head dim).  The decay mask below costs row block wq about wq + 1 units of work, so in
+            // the full pass the 16 (row block, 16-byte chunk) units of a lane are dealt 7 / 5 / 3 / 1
+            // to row blocks 0 .. 3 instead of 4 each; a foreign row's weight comes from cs:
+            // w_r = Delta_r 2^(l_last - l_r) = 2^(cs_r + l_last).
             tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
+            {
+                const int ubeg = full ? (wq == 0 ? 0 : (wq == 1 ? 7 : (wq == 2 ? 12 : 15))) : 4 * wq;
+                const int uend = full ? (wq == 0 ? 7 : (wq == 1 ? 12 : (wq == 2 ? 15 : 16))) : 4 * wq + 4;
+#pragma unroll 1
+                for (int un = ubeg; un < uend; ++un) {
+                    const int r = (un >> 2) * 32 + lane;
+                    const float w_r = full ? tc::ex2_approx(s_cs[r] + l2_last) : w_s;
+                    const uint32_t off = tc::sw128_offset(r, 4 * hf + (un & 3));
+                    const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
+                    const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
+                    uint32_t o[4];
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                const uint32_t off = tc::sw128_offset(i, 4 * hf + ch);
-                const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
-                const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
-                uint32_t o[4];
-#pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    o[q] = tc::pack_bf16x2(w_s * __uint_as_float(wv[q] << 16),
-                                           w_s * __uint_as_float(wv[q] & 0xffff0000u));
-                *reinterpret_cast<uint4 *>(s_xp + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                    for (int q = 0; q < 4; ++q)
+                        o[q] = tc::pack_bf16x2(w_r * __uint_as_float(wv[q] << 16),
+                                               w_r * __uint_as_float(wv[q] & 0xffff0000u));
+                    *reinterpret_cast<uint4 *>(s_xp + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
             }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&hb->xp_full);
