@@ -402,13 +402,13 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 
             // ---- w . X  (rows of the X slab -> rows of the X' slab, this thread's half of the
             // head dim).  The decay mask below costs row block wq about wq + 1 units of work, so in
-            // the full pass the 16 (row block, 16-byte chunk) units of a lane are dealt 7 / 5 / 3 / 1
+            // the full pass the 16 (row block, 16-byte chunk) units of a lane are dealt 6 / 5 / 3 / 2
             // to row blocks 0 .. 3 instead of 4 each; a foreign row's weight comes from cs:
             // w_r = Delta_r 2^(l_last - l_r) = 2^(cs_r + l_last).
             tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
             {
-                const int ubeg = full ? (wq == 0 ? 0 : (wq == 1 ? 7 : (wq == 2 ? 12 : 15))) : 4 * wq;
-                const int uend = full ? (wq == 0 ? 7 : (wq == 1 ? 12 : (wq == 2 ? 15 : 16))) : 4 * wq + 4;
+                const int ubeg = full ? (wq == 0 ? 0 : (wq == 1 ? 6 : (wq == 2 ? 11 : 14))) : 4 * wq;
+                const int uend = full ? (wq == 0 ? 6 : (wq == 1 ? 11 : (wq == 2 ? 14 : 16))) : 4 * wq + 4;
 #pragma unroll 1
                 for (int un = ubeg; un < uend; ++un) {
                     const int r = (un >> 2) * 32 + lane;
