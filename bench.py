@@ -106,7 +106,8 @@ class ClockSampler:
 
 
 def algorithmic_work(cfg: synth.LayerConfig):
-    """Per-launch algorithmic work of each kernel for B x L tokens ('Roofline')."""
+    """Per-launch algorithmic work of each kernel for B x L tokens: bytes the method must move or
+    flops it must execute, not what a particular kernel happens to do."""
     T, F, S, E, k = cfg.tokens, cfg.F, cfg.S, cfg.E, cfg.k
     H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.Q
     es = 2 if cfg.dtype == "bf16" else 4
