@@ -413,14 +413,21 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 for (int un = ubeg; un < uend; ++un) {
                     const int r = (un >> 2) * 32 + lane;
                     const float w_r = full ? tc::ex2_approx(s_cs[r] + l2_last) : w_s;
+                    // w_r as a two-term bf16 sum; x stays packed: round(w_hi x + round(w_lo x)) is
+                    // w_r x rounded once, up to a term of relative size 2^-17
+                    const __nv_bfloat16 w_hi = __float2bfloat16_rn(w_r);
+                    const __nv_bfloat162 w_hi2 = __bfloat162bfloat162(w_hi);
+                    const __nv_bfloat162 w_lo2 = __float2bfloat162_rn(w_r - __bfloat162float(w_hi));
                     const uint32_t off = tc::sw128_offset(r, 4 * hf + (un & 3));
                     const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
                     const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
                     uint32_t o[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q)
-                        o[q] = tc::pack_bf16x2(w_r * __uint_as_float(wv[q] << 16),
-                                               w_r * __uint_as_float(wv[q] & 0xffff0000u));
+                    for (int q = 0; q < 4; ++q) {
+                        const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
+                        const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
+                        o[q] = *reinterpret_cast<const uint32_t *>(&pr);
+                    }
                     *reinterpret_cast<uint4 *>(s_xp + off) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
