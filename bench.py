@@ -36,7 +36,7 @@ NSETS = 4   # rotating input sets: together several times the 126 MB L2
 NCU_TRAFFIC_BYTES = {
     # workload small_lm, one launch each (profiles/forward_small_lm_kernels.md); ncu flushes caches
     # before a launch and part of a kernel's writes can still sit in L2 when it ends
-    "ssd_tiles": 79.636e6, "router_topk": 25.212e6, "expert_gemm": 28.600e6, "mix_slots": 16.792e6,
+    "ssd_tiles": 77.136e6, "router_topk": 25.212e6, "expert_gemm": 28.638e6, "mix_slots": 16.792e6,
     "ssd_scalars": 1.578e6,
     # decode workload (profiles/decode_update_kernel.md)
     "decode_update": 479.8e6,
