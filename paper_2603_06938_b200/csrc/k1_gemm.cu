@@ -1,9 +1,10 @@
 // K1 (tensor-core part): the expert stream projection as a grouped GEMM on tcgen05.
 //
 // Tokens are grouped by selected expert (only the k active experts of a token are ever
-// projected, so the cost does not grow with E: Theorem 2).  For every (expert, 128-row tile)
-// one CTA computes  D[128, BN] = U_rows[128, F] * W_e[e][n0:n0+BN, :]^T  with the gathered token
-// rows as the K-major A operand and the expert's weight rows as the K-major B operand, scales
+// projected, so the cost does not grow with E: Theorem 2).  For every (expert, 256-row tile)
+// one CTA computes  D[256, BN] = U_rows[256, F] * W_e[e][n0:n0+BN, :]^T  (two 128-row MMA halves)
+// with the gathered token rows as the K-major A operand and the expert's weight rows as the
+// K-major B operand, scales
 // row r by its router weight pi_{t,e} (Theorem 1's mixed streams) and writes it to slot (t, j).
 // A last streaming kernel sums the k slots of each token.
 #include "internal.h"

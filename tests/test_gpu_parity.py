@@ -52,6 +52,10 @@ CASES = [
     cfg_of("bf16", L=130, B=1, H=2, F=2048, E=8, k=2),     # router matrix of 32 KB in shared memory
     cfg_of("bf16", L=150, B=1, H=2, F=1024, E=64, k=8),    # router matrix too large to stage
     cfg_of("bf16", L=2100, B=1, H=2, F=256, E=16, k=2),    # several router chunks per block
+    cfg_of("bf16", L=390, B=2, H=3),                       # odd head count: one CTA with a single head
+    cfg_of("bf16", L=257, B=1, H=6, G=2),                  # three heads per group: a pair and a single
+    cfg_of("bf16", L=129, B=1, H=2),                       # one token past a tile boundary
+    cfg_of("bf16", L=5000, B=1, H=2, h0_std=0.3),          # segmented sequence with an initial state
 ]
 
 
