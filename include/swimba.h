@@ -159,7 +159,7 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
  *   - The array is SWIMBA_STATIC_SCRATCH_BYTES large and is held by every GPU that loads the
  *     library until the process exits.  Token counts whose scratch need exceeds it are rejected
  *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (with bf16, S = 256,
- *     E = 8 and k = 2 the limit is about 5000 tokens per call).
+ *     E = 8 and k = 2 the limit is about 14000 tokens per call).
  *   - The first call on each device looks up the array's device address; make that first call
  *     outside any stream capture.  No call allocates or frees device memory.
  *   - All calls on a device share the one array, and it keeps the previous call's contents (the

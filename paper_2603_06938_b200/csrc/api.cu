@@ -181,8 +181,9 @@ int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, con
         if (cudaMemsetAsync(counts, 0, sizeof(int) * SWIMBA_MAX_EXPERTS, ctx.stream) != cudaSuccess)
             return fail(h, SWIMBA_ERR_CUDA, "clearing the expert histogram failed");
     }
+    const bool zero_bc = tensor && expert_gemm_adds_rows(c.top_k);
     int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts,
-                           perm, T, h->sm_count);
+                           perm, T, h->sm_count, zero_bc ? BC : nullptr, S * 2);
     if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
     if (tensor) {
         rc = launch_expert_gemm(ctx, u, w->W_expert, wt, T, c.d_model, S, c.n_experts, c.top_k,

@@ -7,15 +7,18 @@ namespace swimba {
 // K1a: router logits, softmax over all E, top-k (indices + un-renormalised weights).
 // When counts is given (zeroed beforehand) the (token, slot) pairs are also grouped by expert:
 // perm[e * cap + i], i < counts[e], lists the entries t*k + j routed to expert e.
+// zero_out (may be NULL): a [T, zero_bytes_per_token] buffer the kernel clears on the way (the
+// mixed streams, when the projection adds its slots in place).
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
                   int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                  int sm_count);
+                  int sm_count, void *zero_out, int zero_bytes_per_token);
 
 // K1b (tensor cores): grouped GEMM over the per-expert lists + slot sum.  `workspace` is sized
 // by expert_gemm_workspace_bytes and holds the histogram (zeroed by the caller before the
 // router runs), the per-expert lists (capacity T each) and the per-slot projections.
 size_t expert_gemm_workspace_bytes(int64_t T, int S, int E, int k);
 bool expert_gemm_supported(int F, int S);
+bool expert_gemm_adds_rows(int k);   // true: BC must be zero before launch_expert_gemm runs
 int *expert_gemm_counts(void *workspace);
 int *expert_gemm_perm(void *workspace);
 int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const float *w, int64_t T,

@@ -5,8 +5,11 @@
 // one CTA computes  D[256, BN] = U_rows[256, F] * W_e[e][n0:n0+BN, :]^T  (two 128-row MMA halves)
 // with the gathered token rows as the K-major A operand and the expert's weight rows as the
 // K-major B operand, scales
-// row r by its router weight pi_{t,e} (Theorem 1's mixed streams) and writes it to slot (t, j).
-// A last streaming kernel sums the k slots of each token.
+// row r by its router weight pi_{t,e} (Theorem 1's mixed streams).  With two active experts per
+// token the scaled row is added straight into the token's row of the mixed streams (zeroed by the
+// router kernel): 0 + a + b in bf16 is the same whichever slot arrives first, so the result is
+// reproducible and no slot buffer is needed.  With more experts the order of the additions would
+// matter: the rows go to slots (t, j) and a last streaming kernel sums them in a fixed order.
 #include "internal.h"
 #include "tc05.cuh"
 
@@ -29,7 +32,7 @@ template <int BN>
 __global__ void __launch_bounds__(GM_THREADS, 1)
 expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat16 *__restrict__ u,
                    const int *__restrict__ perm, int64_t cap, const float *__restrict__ w_slot,
-                   const int *__restrict__ counts, int E, int F, int S, int k,
+                   const int *__restrict__ counts, int E, int F, int S, int k, int add_rows,
                    __nv_bfloat16 *__restrict__ out, int *d_status)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -95,7 +98,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
         if (r < nrows) {
             const int entry = perm[row0 + r];
             row_src[r] = entry / k;
-            row_dst[r] = entry;
+            row_dst[r] = add_rows ? entry / k : entry;      // token row, or slot row
             row_w[r] = w_slot[entry];
         } else {
             row_src[r] = -1;
@@ -175,9 +178,11 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
         tc::fence_proxy_async_smem();
         for (int hf = 0; hf < nhalf; ++hf) {
             const int row = hf * 128 + warp * 32 + lane;
-            if (row < nrows)
-                tc::bulk_store(out + (int64_t)row_dst[row] * S + n0, smem + (uint32_t)row * ROW_STRIDE,
-                               BN * 2);
+            if (row < nrows) {
+                __nv_bfloat16 *dst = out + (int64_t)row_dst[row] * S + n0;
+                if (add_rows) tc::bulk_reduce_add_bf16(dst, smem + (uint32_t)row * ROW_STRIDE, BN * 2);
+                else tc::bulk_store(dst, smem + (uint32_t)row * ROW_STRIDE, BN * 2);
+            }
         }
         tc::bulk_commit_group();
         tc::bulk_wait_read_all();
@@ -265,7 +270,7 @@ size_t expert_gemm_workspace_bytes(int64_t T, int S, int E, int k)
 {
     size_t tot = gemm_ws_up(SWIMBA_MAX_EXPERTS * sizeof(int));
     tot += gemm_ws_up((size_t)E * T * sizeof(int));
-    if (k > 1) tot += gemm_ws_up((size_t)T * k * S * sizeof(__nv_bfloat16));
+    if (k > 1 && !expert_gemm_adds_rows(k)) tot += gemm_ws_up((size_t)T * k * S * sizeof(__nv_bfloat16));
     return tot;
 }
 
@@ -274,6 +279,9 @@ int *expert_gemm_perm(void *workspace)
 {
     return (int *)((char *)workspace + gemm_ws_up(SWIMBA_MAX_EXPERTS * sizeof(int)));
 }
+
+// k == 2: the two slots of a token are added in place (BC must be zero when the GEMM starts).
+bool expert_gemm_adds_rows(int k) { return k == 2; }
 
 bool expert_gemm_supported(int F, int S)
 {
@@ -287,7 +295,8 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
     const int max_tiles = (int)ceil_div64(T * k, GM_BM) + E;
     int *counts = expert_gemm_counts(workspace);
     int *perm = expert_gemm_perm(workspace);
-    __nv_bfloat16 *slots = (k > 1)
+    const int add_rows = expert_gemm_adds_rows(k) ? 1 : 0;
+    __nv_bfloat16 *slots = (k > 1 && !add_rows)
         ? (__nv_bfloat16 *)((char *)perm + gemm_ws_up((size_t)E * T * sizeof(int)))
         : (__nv_bfloat16 *)BC;
 
@@ -312,7 +321,8 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
             cudaSuccess)                                                                        \
             return SWIMBA_ERR_CUDA;                                                             \
         kern<<<grid, GM_THREADS, smem, ctx.stream>>>(tmap, (const __nv_bfloat16 *)u, perm, T, w,  \
-                                                     counts, E, F, S, k, slots, ctx.d_status);  \
+                                                     counts, E, F, S, k, add_rows, slots,       \
+                                                     ctx.d_status);                             \
     } while (0)
     ctx.begin(STAGE_EXPERT_GEMM);
     if (BN == 256) SWIMBA_GEMM_CASE(256);
@@ -321,7 +331,7 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
     else SWIMBA_GEMM_CASE(32);
 #undef SWIMBA_GEMM_CASE
     ctx.end();
-    if (k > 1) {
+    if (k > 1 && !add_rows) {
         const int64_t nvec = T * (S / 8);
         int64_t blocks = ceil_div64(nvec, 256);
         if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;

@@ -27,7 +27,8 @@ template <typename T, int EP, int TPW>
 __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
                    int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts,
-                   int *__restrict__ perm, int64_t cap, int stage_w, int chunk)
+                   int *__restrict__ perm, int64_t cap, int stage_w, int chunk,
+                   uint4 *__restrict__ zero_out, int zero_vec_per_token)
 {
     constexpr int V = TPW * EP;                 // values per lane before the butterfly
     constexpr int R = V > 32 ? V / 32 : 1;      // values per lane after it (adjacent experts)
@@ -55,6 +56,12 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
         const int64_t tbeg = c * chunk;
         const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
         if (threadIdx.x < SWIMBA_MAX_EXPERTS) s_cnt[threadIdx.x] = 0;
+        if (zero_out) {
+            // the mixed-stream rows of this chunk start at zero: the projection adds its slots
+            const int64_t nz = (tend - tbeg) * zero_vec_per_token;
+            uint4 *z = zero_out + tbeg * zero_vec_per_token;
+            for (int64_t i = threadIdx.x; i < nz; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
         __syncthreads();
         // The feature loads run one step ahead of the arithmetic, across passes too: `raw` always
         // holds the next 8-feature slice of the next TPW tokens.
@@ -190,7 +197,7 @@ router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__re
 template <typename T>
 static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Ttok, int F, int E,
                            int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                           int sm_count)
+                           int sm_count, void *zero_out, int zero_bytes_per_token)
 {
     const int warps = 8;
     if (E == 1) {
@@ -222,7 +229,8 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         if (blocks > cap_blocks) blocks = cap_blocks;                                          \
         kern<<<(unsigned)blocks, warps * 32, smem, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, \
                                                                  counts, perm, cap, stage_w,   \
-                                                                 chunk);                       \
+                                                                 chunk, (uint4 *)zero_out,     \
+                                                                 zero_bytes_per_token / 16);   \
     } while (0)
     if (E <= 2) SWIMBA_ROUTER_CASE(2, 8);
     else if (E <= 4) SWIMBA_ROUTER_CASE(4, 8);
@@ -237,15 +245,15 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
 
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
                   int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                  int sm_count)
+                  int sm_count, void *zero_out, int zero_bytes_per_token)
 {
     if (T <= 0) return SWIMBA_OK;
     if (dtype == SWIMBA_DTYPE_FP32)
         return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w,
-                                      counts, perm, cap, sm_count);
+                                      counts, perm, cap, sm_count, zero_out, zero_bytes_per_token);
     return launch_router_t<__nv_bfloat16>(ctx, (const __nv_bfloat16 *)u,
                                           (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w, counts,
-                                          perm, cap, sm_count);
+                                          perm, cap, sm_count, zero_out, zero_bytes_per_token);
 }
 
 // One warp per (token, block of RW stream rows): BC[t, r] = sum_j w_j <W_e[e_j, r, :], u_t>.

@@ -114,6 +114,13 @@ __device__ __forceinline__ void bulk_store(void *dst_global, const void *src_sme
                  "r"(smem_u32(src_smem)), "r"(bytes)
                  : "memory");
 }
+// The same, adding into the destination (bf16 elements, round to nearest, no flush to zero).
+__device__ __forceinline__ void bulk_reduce_add_bf16(void *dst_global, const void *src_smem, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.noftz.bf16 [%0], [%1], %2;" ::"l"(
+                     dst_global),
+                 "r"(smem_u32(src_smem)), "r"(bytes)
+                 : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the issuing thread's bulk stores have finished READING shared memory.
 __device__ __forceinline__ void bulk_wait_read_all() {
