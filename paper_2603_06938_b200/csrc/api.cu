@@ -166,7 +166,8 @@ int set_device(swimba_handle *h)
 
 // Router + projection + mix into BC (dtype, or fp32 when bc_fp32).
 int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *u,
-                  int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt, void *gemm_ws)
+                  int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt, void *gemm_ws,
+                  const ScalarsArgs *scalars = nullptr)
 {
     const swimba_config &c = h->cfg;
     const int S = 2 * c.n_groups * c.d_state;
@@ -183,7 +184,8 @@ int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, con
     }
     const bool zero_bc = tensor && expert_gemm_adds_rows(c.top_k);
     int rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts,
-                           perm, T, h->sm_count, zero_bc ? BC : nullptr, S * 2);
+                           perm, T, h->sm_count, zero_bc ? BC : nullptr, S * 2,
+                           scalars ? *scalars : ScalarsArgs{});
     if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
     if (tensor) {
         rc = launch_expert_gemm(ctx, u, w->W_expert, wt, T, c.d_model, S, c.n_experts, c.top_k,
@@ -199,12 +201,12 @@ int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, con
 
 int run_ssd(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *x,
             const void *BC, const float *dt, const float *h0, int B, int L, void *y,
-            float *h_final, void *ssd_ws)
+            float *h_final, void *ssd_ws, bool scalars_done = false)
 {
     const swimba_config &c = h->cfg;
     if (ssd_ws && ssd_tiles_supported(c.dtype, c.head_dim, c.d_state)) {
         int rc = launch_ssd_tiles(ctx, x, BC, dt, w->A, w->dt_bias, w->D, h0, B, L, c.n_heads,
-                                  c.n_groups, c.chunk, h->sm_count, y, h_final, ssd_ws);
+                                  c.n_groups, c.chunk, h->sm_count, y, h_final, ssd_ws, scalars_done);
         if (rc != SWIMBA_OK) return fail(h, rc, "SSD tile kernel launch failed");
         return SWIMBA_OK;
     }
@@ -356,8 +358,13 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
-    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
-    if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final, ws + l.ssd);
+    // The SSD step sizes depend on dt only: with more than one expert they ride along as extra
+    // blocks of the router launch.
+    const bool fuse = h->cfg.n_experts > 1 && ssd_tiles_supported(h->cfg.dtype, h->cfg.head_dim, h->cfg.d_state);
+    const ScalarsArgs sa = fuse ? ssd_scalars_args(dt, w->A, w->dt_bias, B, L, h->cfg.n_heads, ws + l.ssd)
+                                : ScalarsArgs{};
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm, fuse ? &sa : nullptr);
+    if (rc == SWIMBA_OK) rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final, ws + l.ssd, fuse);
     h->last_stream = ctx.stream;
     h->last_launches = ctx.launches;
     return rc;

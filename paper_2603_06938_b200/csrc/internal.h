@@ -1,6 +1,7 @@
 // Launchers shared between the API translation unit and the kernel files.
 #pragma once
 #include "common.cuh"
+#include "ssd_scalars.cuh"
 
 namespace swimba {
 
@@ -8,10 +9,11 @@ namespace swimba {
 // When counts is given (zeroed beforehand) the (token, slot) pairs are also grouped by expert:
 // perm[e * cap + i], i < counts[e], lists the entries t*k + j routed to expert e.
 // zero_out (may be NULL): a [T, zero_bytes_per_token] buffer the kernel clears on the way (the
-// mixed streams, when the projection adds its slots in place).
+// mixed streams, when the projection adds its slots in place).  scalars.dl != NULL: the SSD step
+// sizes are computed by extra blocks of the same launch (not with a single expert).
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
                   int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                  int sm_count, void *zero_out, int zero_bytes_per_token);
+                  int sm_count, void *zero_out, int zero_bytes_per_token, const ScalarsArgs &scalars);
 
 // K1b (tensor cores): grouped GEMM over the per-expert lists + slot sum.  `workspace` is sized
 // by expert_gemm_workspace_bytes and holds the histogram (zeroed by the caller before the
@@ -33,9 +35,14 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
 // K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
 bool ssd_tiles_supported(int dtype, int P, int N);
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);
+// scalars_done: the step sizes and tile log-decays (ssd_scalars_args over the same workspace) have
+// already been produced, as extra blocks of the router kernel.
+ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,
+                             void *workspace);
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
                      const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
-                     int chunk, int sm_count, void *y, float *h_final, void *workspace);
+                     int chunk, int sm_count, void *y, float *h_final, void *workspace,
+                     bool scalars_done);
 
 // Per-timestep SIMT evaluation of the recurrence (fp32 state in registers).
 int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,

@@ -28,8 +28,17 @@ __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
                    int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts,
                    int *__restrict__ perm, int64_t cap, int stage_w, int chunk,
-                   uint4 *__restrict__ zero_out, int zero_vec_per_token)
+                   uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks,
+                   const ScalarsArgs scalars)
 {
+    if ((int)blockIdx.x >= router_blocks) {
+        // extra blocks: SSD step sizes and tile log-decays, two (tile, head, sequence) units each
+        __shared__ float s_tot[2][4];
+        const int half = threadIdx.x >> 7;
+        const int64_t unit = ((int64_t)blockIdx.x - router_blocks) * 2 + half;
+        ssd_scalars_unit(scalars, unit, unit < scalars_units(scalars), threadIdx.x & 127, s_tot[half]);
+        return;
+    }
     constexpr int V = TPW * EP;                 // values per lane before the butterfly
     constexpr int R = V > 32 ? V / 32 : 1;      // values per lane after it (adjacent experts)
     constexpr int DUP = V >= 32 ? 1 : 32 / V;   // lanes holding the same value after it
@@ -52,7 +61,7 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
     const int q_own = lane / GW;
     const int e0 = ((lane % GW) / DUP) * R;
     const int64_t nchunks = ceil_div64(Ttok, chunk);
-    for (int64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
+    for (int64_t c = blockIdx.x; c < nchunks; c += router_blocks) {
         const int64_t tbeg = c * chunk;
         const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
         if (threadIdx.x < SWIMBA_MAX_EXPERTS) s_cnt[threadIdx.x] = 0;
@@ -197,7 +206,8 @@ router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__re
 template <typename T>
 static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Ttok, int F, int E,
                            int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                           int sm_count, void *zero_out, int zero_bytes_per_token)
+                           int sm_count, void *zero_out, int zero_bytes_per_token,
+                           const ScalarsArgs &scalars)
 {
     const int warps = 8;
     if (E == 1) {
@@ -227,10 +237,10 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         int64_t blocks = ceil_div64(Ttok, chunk);                                              \
         const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);             \
         if (blocks > cap_blocks) blocks = cap_blocks;                                          \
-        kern<<<(unsigned)blocks, warps * 32, smem, ctx.stream>>>(u, W_r, Ttok, F, E, k, idx, w, \
-                                                                 counts, perm, cap, stage_w,   \
-                                                                 chunk, (uint4 *)zero_out,     \
-                                                                 zero_bytes_per_token / 16);   \
+        const int64_t extra = (scalars_units(scalars) + 1) / 2;                                \
+        kern<<<(unsigned)(blocks + extra), warps * 32, smem, ctx.stream>>>(                    \
+            u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk, (uint4 *)zero_out, \
+            zero_bytes_per_token / 16, (int)blocks, scalars);                                  \
     } while (0)
     if (E <= 2) SWIMBA_ROUTER_CASE(2, 8);
     else if (E <= 4) SWIMBA_ROUTER_CASE(4, 8);
@@ -245,15 +255,15 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
 
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
                   int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
-                  int sm_count, void *zero_out, int zero_bytes_per_token)
+                  int sm_count, void *zero_out, int zero_bytes_per_token, const ScalarsArgs &scalars)
 {
     if (T <= 0) return SWIMBA_OK;
     if (dtype == SWIMBA_DTYPE_FP32)
         return launch_router_t<float>(ctx, (const float *)u, (const float *)W_r, T, F, E, k, idx, w,
-                                      counts, perm, cap, sm_count, zero_out, zero_bytes_per_token);
+                                      counts, perm, cap, sm_count, zero_out, zero_bytes_per_token, scalars);
     return launch_router_t<__nv_bfloat16>(ctx, (const __nv_bfloat16 *)u,
                                           (const __nv_bfloat16 *)W_r, T, F, E, k, idx, w, counts,
-                                          perm, cap, sm_count, zero_out, zero_bytes_per_token);
+                                          perm, cap, sm_count, zero_out, zero_bytes_per_token, scalars);
 }
 
 // One warp per (token, block of RW stream rows): BC[t, r] = sum_j w_j <W_e[e_j, r, :], u_t>.

@@ -31,6 +31,7 @@
 // kernel computes every segment's local end state (MMA 4 only), segment_scan_kernel (K3) chains
 // them, and a second pass evaluates each segment from its true incoming state.
 #include "internal.h"
+#include "ssd_scalars.cuh"
 #include "tc05.cuh"
 
 namespace swimba {
@@ -47,7 +48,6 @@ constexpr int WARP_TMA = NCW, WARP_MMA0 = NCW + 1;
 constexpr int SSD_THREADS = 32 * (NCW + 1 + NHD);
 constexpr int HEAD_THREADS = 256;
 constexpr uint32_t SLAB = 16384;        // 128 rows x 128 bytes
-constexpr float LOG2E = 1.4426950408889634f;
 
 // shared memory map (bytes from the 1024-aligned base)
 constexpr uint32_t SM_CB = 0;                        // C0 C1 B0 B1 slabs (single stage)
@@ -94,30 +94,12 @@ struct __align__(16) SsdSmall {
 __host__ __device__ inline int pairs_per_group(int H, int G) { return (H / G + NHD - 1) / NHD; }
 }  // namespace
 
-// Delta_t = softplus(dt_t + dt_bias_h) and the log2-decay accumulated inside each 128-token tile,
-// dl[(b*H + h)*Lpad + t] = (Delta_t, sum_{r <= t, r in t's tile} Delta_r A_h log2 e); positions
-// past L carry Delta = 0, so the last entry of a tile is always the tile's total.
-__global__ void __launch_bounds__(ST)
-ssd_scalars_kernel(const float *__restrict__ dt, const float *__restrict__ A,
-                   const float *__restrict__ dt_bias, int L, int Lpad, int H,
-                   float2 *__restrict__ dl)
+// Stand-alone launch of the step sizes and tile log-decays (one unit per block).
+__global__ void __launch_bounds__(SCALARS_TILE)
+ssd_scalars_kernel(const ScalarsArgs args)
 {
     __shared__ float s_tot[4];
-    const int tile = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int i = threadIdx.x, lane = i & 31, wq = i >> 5;
-    const int t = tile * ST + i;
-    const float raw = (dt && t < L) ? dt[((int64_t)b * L + t) * H + h] : 0.f;
-    const float delta = t < L ? softplus_f(raw + dt_bias[h]) : 0.f;
-    float l2 = delta * (A[h] * LOG2E);
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float nb = __shfl_up_sync(0xffffffffu, l2, o);
-        if (lane >= o) l2 += nb;
-    }
-    if (lane == 31) s_tot[wq] = l2;
-    __syncthreads();
-    for (int w = 0; w < wq; ++w) l2 += s_tot[w];
-    dl[((int64_t)b * H + h) * Lpad + t] = make_float2(delta, l2);
+    ssd_scalars_unit(args, blockIdx.x, true, threadIdx.x, s_tot);
 }
 
 __global__ void __launch_bounds__(SSD_THREADS, 1)
@@ -658,9 +640,19 @@ size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count)
     return tot;
 }
 
+ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,
+                             void *workspace)
+{
+    ScalarsArgs a;
+    a.dt = dt; a.A = A; a.dt_bias = dt_bias; a.dl = (float2 *)workspace;
+    a.L = L; a.Lpad = ceil_div(L, ST) * ST; a.H = H; a.B = B;
+    return a;
+}
+
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
                      const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
-                     int chunk, int sm_count, void *y, float *h_final, void *workspace)
+                     int chunk, int sm_count, void *y, float *h_final, void *workspace,
+                     bool scalars_done)
 {
     if (B <= 0 || L <= 0) return SWIMBA_OK;
     const int S = 2 * G * SN;
@@ -687,10 +679,12 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     const int Lpad = ceil_div(L, ST) * ST;
     float2 *dl = (float2 *)workspace;
     char *seg_ws = (char *)workspace + ssd_scalars_bytes(B, L, H);
-    ctx.begin(STAGE_SSD_SCALARS);
-    ssd_scalars_kernel<<<dim3((unsigned)(Lpad / ST), (unsigned)H, (unsigned)B), ST, 0, ctx.stream>>>(
-        dt, A, dt_bias, L, Lpad, H, dl);
-    ctx.end();
+    if (!scalars_done) {
+        const ScalarsArgs sa = ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace);
+        ctx.begin(STAGE_SSD_SCALARS);
+        ssd_scalars_kernel<<<(unsigned)scalars_units(sa), SCALARS_TILE, 0, ctx.stream>>>(sa);
+        ctx.end();
+    }
     SsdParams p;
     p.dl = dl; p.D = D;
     p.L = L; p.Lpad = Lpad; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
