@@ -1,5 +1,6 @@
 // Shared device/host helpers of the Swimba CUDA library (sm_100a only).
 #pragma once
+#include <utility>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -42,6 +43,33 @@ struct LaunchCtx {
         launches++;
     }
 };
+
+// Programmatic dependent launch.
+// A kernel launched with programmatic stream serialization may start while the kernel before it
+// in the stream still runs; grid_dep_wait() returns once that kernel has completed and its
+// writes are visible (a no-op under an ordinary launch).  grid_dep_launch() lets the next such
+// kernel be scheduled as soon as every block of this one has called it.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;"); }
+
+// Kernel launch; overlap = true lets the kernel's prologue run under the tail of the kernel before
+// it in the stream (the kernel itself calls grid_dep_wait() before it touches that kernel's data).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, bool overlap, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
 
 __host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 __host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }

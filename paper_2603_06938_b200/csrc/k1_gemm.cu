@@ -36,6 +36,43 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
                    __nv_bfloat16 *__restrict__ out, int *d_status)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    constexpr int STAGES = gm_stages(BN);
+    constexpr uint32_t A_BYTES = GM_BM * 128, B_BYTES = BN * 128;
+    constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sA = smem;
+    uint8_t *sB = smem + STAGES * A_BYTES;
+    uint64_t *full = (uint64_t *)(sB + STAGES * B_BYTES);
+    uint64_t *empty = full + STAGES;
+    uint64_t *acc_bar = empty + STAGES;
+    uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
+    int *abort_flag = (int *)(tmem_slot + 1);
+    int *row_src = abort_flag + 1;            // [256] token index or -1
+    int *row_dst = row_src + GM_BM;           // [256] output row
+    float *row_w = (float *)(row_dst + GM_BM);
+
+    const int uwarp = __shfl_sync(0xffffffffu, warp, 0);   // warp-uniform for the compiler
+
+    // Set-up that needs nothing from the router kernel; it may run under that kernel's tail.
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            tc::mbar_init(&full[s], 128 + 1);
+            tc::mbar_init(&empty[s], 1);
+        }
+        tc::mbar_init(acc_bar, 1);
+        *abort_flag = 0;
+        tc::fence_mbar_init();
+    }
+    if (uwarp == 5) {
+        tc::tmem_alloc(tmem_slot, TMEM_COLS);
+        tc::tmem_relinquish();
+    }
+    if (uwarp == 4 && lane == 0) tc::prefetch_tmap(&tmap_w);
+    grid_dep_launch();
+    grid_dep_wait();        // counts, lists and weights come from the router kernel
+
     // Tile -> (expert, rows): tiles are numbered expert by expert, ceil(counts[e] / GM_BM) each.
     // Every warp finds its tile with one load per lane and a shuffle scan.
     int e = -1, row0 = 0, cnt = 0;
@@ -61,39 +98,11 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
             before += __shfl_sync(0xffffffffu, incl, 31);
         }
     }
-    if (e < 0) return;
-    const int nrows = min(GM_BM, cnt - row0);
+    const bool has_tile = e >= 0;                   // (the grid is sized for the worst case)
+    const int nrows = has_tile ? min(GM_BM, cnt - row0) : 0;
     const int nhalf = nrows > 128 ? 2 : 1;          // 128-row halves that hold rows
-    perm += (int64_t)e * cap;
+    if (has_tile) perm += (int64_t)e * cap;
     const int n0 = blockIdx.y * BN;
-    constexpr int STAGES = gm_stages(BN);
-    constexpr uint32_t A_BYTES = GM_BM * 128, B_BYTES = BN * 128;
-    constexpr uint32_t TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
-
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *sA = smem;
-    uint8_t *sB = smem + STAGES * A_BYTES;
-    uint64_t *full = (uint64_t *)(sB + STAGES * B_BYTES);
-    uint64_t *empty = full + STAGES;
-    uint64_t *acc_bar = empty + STAGES;
-    uint32_t *tmem_slot = (uint32_t *)(acc_bar + 1);
-    int *abort_flag = (int *)(tmem_slot + 1);
-    int *row_src = abort_flag + 1;            // [256] token index or -1
-    int *row_dst = row_src + GM_BM;           // [256] output row
-    float *row_w = (float *)(row_dst + GM_BM);
-
-    const int uwarp = __shfl_sync(0xffffffffu, warp, 0);   // warp-uniform for the compiler
-
-    if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            tc::mbar_init(&full[s], 128 + 1);
-            tc::mbar_init(&empty[s], 1);
-        }
-        tc::mbar_init(acc_bar, 1);
-        *abort_flag = 0;
-        tc::fence_mbar_init();
-    }
     for (int r = tid; r < GM_BM; r += GM_THREADS) {
         if (r < nrows) {
             const int entry = perm[row0 + r];
@@ -106,15 +115,14 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
             row_w[r] = 0.f;
         }
     }
-    if (uwarp == 5) {
-        tc::tmem_alloc(tmem_slot, TMEM_COLS);
-        tc::tmem_relinquish();
-    }
-    if (uwarp == 4 && lane == 0) tc::prefetch_tmap(&tmap_w);
     tc::tc_fence_before();
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    if (!has_tile) {
+        if (uwarp == 5) tc::tmem_dealloc(tmem_base, TMEM_COLS);
+        return;
+    }
     const int KB = ceil_div(F, GM_BK);
 
     if (uwarp < 4) {
@@ -320,9 +328,9 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != \
             cudaSuccess)                                                                        \
             return SWIMBA_ERR_CUDA;                                                             \
-        kern<<<grid, GM_THREADS, smem, ctx.stream>>>(tmap, (const __nv_bfloat16 *)u, perm, T, w,  \
-                                                     counts, E, F, S, k, add_rows, slots,       \
-                                                     ctx.d_status);                             \
+        launch_kernel(kern, grid, dim3(GM_THREADS), smem, ctx.stream, true, tmap,               \
+                      (const __nv_bfloat16 *)u, (const int *)perm, (int64_t)T, (const float *)w, \
+                      (const int *)counts, E, F, S, k, add_rows, slots, ctx.d_status);          \
     } while (0)
     ctx.begin(STAGE_EXPERT_GEMM);
     if (BN == 256) SWIMBA_GEMM_CASE(256);

@@ -31,6 +31,7 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
                    uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks,
                    const ScalarsArgs scalars)
 {
+    grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
     if ((int)blockIdx.x >= router_blocks) {
         // extra blocks: SSD step sizes and tile log-decays, two (tile, head, sequence) units each
         __shared__ float s_tot[2][4];
@@ -194,6 +195,7 @@ __global__ void __launch_bounds__(256)
 router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__restrict__ w,
                             int *__restrict__ counts, int *__restrict__ perm)
 {
+    grid_dep_launch();
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < Ttok;
          t += (int64_t)gridDim.x * blockDim.x) {
         idx[t] = 0;

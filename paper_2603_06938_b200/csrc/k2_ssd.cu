@@ -99,6 +99,8 @@ __global__ void __launch_bounds__(SCALARS_TILE)
 ssd_scalars_kernel(const ScalarsArgs args)
 {
     __shared__ float s_tot[4];
+    grid_dep_launch();
+    grid_dep_wait();      // (launched behind the projection kernel in the single-expert path)
     ssd_scalars_unit(args, blockIdx.x, true, threadIdx.x, s_tot);
 }
 
@@ -164,6 +166,10 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = sm->tmem_slot;
+    // Everything above needs nothing from earlier kernels and may run under their tail; the
+    // mixed streams and the step sizes are read from here on.
+    grid_dep_launch();
+    grid_dep_wait();
 
     // Warp index as a value the compiler knows to be warp-uniform.
     const int uwarp = __shfl_sync(0xffffffffu, warp, 0);
@@ -682,7 +688,8 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     if (!scalars_done) {
         const ScalarsArgs sa = ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace);
         ctx.begin(STAGE_SSD_SCALARS);
-        ssd_scalars_kernel<<<(unsigned)scalars_units(sa), SCALARS_TILE, 0, ctx.stream>>>(sa);
+        launch_kernel(ssd_scalars_kernel, dim3((unsigned)scalars_units(sa)), dim3(SCALARS_TILE), 0,
+                      ctx.stream, true, sa);
         ctx.end();
     }
     SsdParams p;
@@ -693,14 +700,14 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     if (nseg == 1) {
         p.h_in = h0; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
+        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     } else {
         float *states = (float *)seg_ws;
         float *decay = states + (size_t)B * nseg * H * SP * SN;
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
+        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
@@ -709,7 +716,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         ctx.end();
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
-        ssd_tiles_kernel<<<grid, SSD_THREADS, smem, ctx.stream>>>(tm_bc, tm_x, tm_y, p);
+        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;

@@ -155,6 +155,7 @@ decode_update_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
                      float *__restrict__ state, int B, int H, int P, int N, int G,
                      T *__restrict__ y)
 {
+    grid_dep_wait();      // the mixed streams come from the projection kernel
     const int lane = threadIdx.x & 31;
     const int S = 2 * G * N;
     const int pgroups = ceil_div(P, DEC_ROWS);
@@ -225,17 +226,19 @@ int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const void *B
     const int64_t cap = (int64_t)sm_count * 8;
     if (blocks > cap) blocks = cap;
     ctx.begin(STAGE_DECODE_UPDATE);
+    const dim3 grid((unsigned)blocks), block(warps * 32);
     if (dtype == SWIMBA_DTYPE_FP32)
-        decode_update_kernel<float, float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
-            (const float *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N, G, (float *)y);
+        launch_kernel(decode_update_kernel<float, float>, grid, block, 0, ctx.stream, true,
+                      (const float *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N, G,
+                      (float *)y);
     else if (bc_fp32)
-        decode_update_kernel<__nv_bfloat16, float><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
-            (const __nv_bfloat16 *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N, G,
-            (__nv_bfloat16 *)y);
+        launch_kernel(decode_update_kernel<__nv_bfloat16, float>, grid, block, 0, ctx.stream, true,
+                      (const __nv_bfloat16 *)x, (const float *)BC, dt, A, dt_bias, D, state, B, H, P, N,
+                      G, (__nv_bfloat16 *)y);
     else
-        decode_update_kernel<__nv_bfloat16, __nv_bfloat16><<<(unsigned)blocks, warps * 32, 0, ctx.stream>>>(
-            (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)BC, dt, A, dt_bias, D, state, B, H, P, N,
-            G, (__nv_bfloat16 *)y);
+        launch_kernel(decode_update_kernel<__nv_bfloat16, __nv_bfloat16>, grid, block, 0, ctx.stream,
+                      true, (const __nv_bfloat16 *)x, (const __nv_bfloat16 *)BC, dt, A, dt_bias, D,
+                      state, B, H, P, N, G, (__nv_bfloat16 *)y);
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
