@@ -51,7 +51,6 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     int *abort_flag = (int *)(tmem_slot + 1);
     int *row_src = abort_flag + 1;            // [256] token index or -1
     int *row_dst = row_src + GM_BM;           // [256] output row
-    float *row_w = (float *)(row_dst + GM_BM);
 
     const int uwarp = __shfl_sync(0xffffffffu, warp, 0);   // warp-uniform for the compiler
 
@@ -108,11 +107,9 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
             const int entry = perm[row0 + r];
             row_src[r] = entry / k;
             row_dst[r] = add_rows ? entry / k : entry;      // token row, or slot row
-            row_w[r] = w_slot[entry];
         } else {
             row_src[r] = -1;
             row_dst[r] = 0;
-            row_w[r] = 0.f;
         }
     }
     tc::tc_fence_before();
@@ -128,6 +125,13 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     if (uwarp < 4) {
         // ---- gather producers: thread -> 16-byte chunk (lane & 7) of rows 4 i + (lane >> 3)
         // of its warp's 64-row quarter
+        // router weights of the two rows this thread scales in the epilogue (needed much later)
+        float wr2[2];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const int row = hf * 128 + warp * 32 + lane;
+            wr2[hf] = row < nrows ? w_slot[perm[row0 + row]] : 0.f;
+        }
         int tsrc[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) tsrc[i] = row_src[warp * 64 + i * 4 + (lane >> 3)];
@@ -159,13 +163,16 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
 
         // ---- epilogue: thread = output row of each half.  All MMAs have completed, so the
         // pipeline buffers are free: the scaled bf16 rows are staged there (row stride padded by
-        // 16 bytes against bank conflicts) and leave as one bulk copy per row.
+        // 16 bytes against bank conflicts).  Rows that are added in place leave as one bulk
+        // reduce-add each, issued half by half so that the second half is converted while the
+        // first is on its way; rows that are stored are sent by the warp that staged them with
+        // BN / 8 lanes per row, 16 bytes per lane (whole lines per instruction).
         tc::mbar_wait(acc_bar, 0, abort_flag, d_status);
         tc::tc_fence_after();
         constexpr uint32_t ROW_STRIDE = BN * 2 + 16;
         for (int hf = 0; hf < nhalf; ++hf) {
             const int row = hf * 128 + warp * 32 + lane;
-            const float wr = row_w[row];
+            const float wr = wr2[hf];
             uint8_t *srow = smem + (uint32_t)row * ROW_STRIDE;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
@@ -182,18 +189,28 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
                 for (int i = 0; i < 4; ++i)
                     dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
             }
-        }
-        tc::fence_proxy_async_smem();
-        for (int hf = 0; hf < nhalf; ++hf) {
-            const int row = hf * 128 + warp * 32 + lane;
-            if (row < nrows) {
-                __nv_bfloat16 *dst = out + (int64_t)row_dst[row] * S + n0;
-                if (add_rows) tc::bulk_reduce_add_bf16(dst, smem + (uint32_t)row * ROW_STRIDE, BN * 2);
-                else tc::bulk_store(dst, smem + (uint32_t)row * ROW_STRIDE, BN * 2);
+            if (add_rows) {
+                tc::fence_proxy_async_smem();
+                if (row < nrows)
+                    tc::bulk_reduce_add_bf16(out + (int64_t)row_dst[row] * S + n0, srow, BN * 2);
+                tc::bulk_commit_group();
             }
         }
-        tc::bulk_commit_group();
-        tc::bulk_wait_read_all();
+        if (add_rows) tc::bulk_wait_read_all();
+        __syncwarp();
+        constexpr int LPR = BN / 8, RPI = 32 / LPR;      // lanes per row, rows per instruction
+        const int sub = lane / LPR, piece = lane % LPR;
+        for (int hf = 0; hf < (add_rows ? 0 : nhalf); ++hf) {
+#pragma unroll 4
+            for (int r0 = 0; r0 < 32; r0 += RPI) {
+                const int row = hf * 128 + warp * 32 + r0 + sub;
+                if (row < nrows) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(smem + (uint32_t)row * ROW_STRIDE + piece * 16);
+                    __nv_bfloat16 *dst = out + (int64_t)row_dst[row] * S + n0 + piece * 8;
+                    *reinterpret_cast<uint4 *>(dst) = v;
+                }
+            }
+        }
     } else if (uwarp == 4) {
         // ---- weight tiles by TMA (whole warp in the loop, one elected lane issues)
         const bool leader = tc::elect_one();
