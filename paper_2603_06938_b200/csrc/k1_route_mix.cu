@@ -1,6 +1,7 @@
 // K1 (SIMT part): router logits + softmax + top-k, and the plain projection/mix used by the
 // fp32 path and by decode.  (Router softmax equation and top-k rule; Theorem 1, mixed streams.)
 #include "internal.h"
+#include <type_traits>
 
 namespace swimba {
 
@@ -28,18 +29,17 @@ __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
                    int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts,
                    int *__restrict__ perm, int64_t cap, int stage_w, int chunk,
-                   uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks,
+                   uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks, int scalar_blocks,
                    const ScalarsArgs scalars)
 {
     grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
-    if ((int)blockIdx.x >= router_blocks) {
-        // extra blocks: SSD step sizes and tile log-decays, two (tile, head, sequence) units each
-        __shared__ float s_tot[2][4];
-        const int half = threadIdx.x >> 7;
-        const int64_t unit = ((int64_t)blockIdx.x - router_blocks) * 2 + half;
-        ssd_scalars_unit(scalars, unit, unit < scalars_units(scalars), threadIdx.x & 127, s_tot[half]);
+    if ((int)blockIdx.x < scalar_blocks) {
+        // leading blocks: SSD step sizes and tile log-decays (they depend on dt only); being
+        // short, they also stagger the start of the router blocks that follow them on an SM
+        ssd_scalars_block(scalars, blockIdx.x);
         return;
     }
+    const int rblock = (int)blockIdx.x - scalar_blocks;       // index among the router blocks
     constexpr int V = TPW * EP;                 // values per lane before the butterfly
     constexpr int R = V > 32 ? V / 32 : 1;      // values per lane after it (adjacent experts)
     constexpr int DUP = V >= 32 ? 1 : 32 / V;   // lanes holding the same value after it
@@ -62,7 +62,7 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
     const int q_own = lane / GW;
     const int e0 = ((lane % GW) / DUP) * R;
     const int64_t nchunks = ceil_div64(Ttok, chunk);
-    for (int64_t c = blockIdx.x; c < nchunks; c += router_blocks) {
+    for (int64_t c = rblock; c < nchunks; c += router_blocks) {
         const int64_t tbeg = c * chunk;
         const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
         if (threadIdx.x < SWIMBA_MAX_EXPERTS) s_cnt[threadIdx.x] = 0;
@@ -190,6 +190,193 @@ router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t T
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Tensor-core router (bf16, F a multiple of 128).  The logits of 16 tokens and 8 experts are one
+// m16n8k16 product chain; a block step covers 32 tokens with 8 warps: warp = (row group of 16
+// tokens, quarter of the features).  The contraction runs over features in any order, so each lane
+// reads 16 contiguous bytes of its two token rows (features 32 j + 8 c .. + 8 of the warp's
+// quarter, c = lane % 4) and feeds them to two MMAs; the matching slice of the router matrix comes
+// from shared memory (rows padded by 64 bytes against bank conflicts), rows past E are zero.
+//
+// Logit summation order (fixed, so results are reproducible run to run): inside a warp the MMAs
+// run over j ascending, first the lower then the upper four features of a lane's eight; the four
+// feature quarters are then added in ascending order by the thread that owns the logit.  bf16
+// products are exact in fp32; the additions are those of the tensor core's fp32 accumulator.
+// Softmax and top-k run on 8 lanes per token, lane s holding experts s, s + 8, ...
+// ------------------------------------------------------------------------------------------
+constexpr int RM_TOK = 32;        // tokens per block step
+constexpr int RM_KSPLIT = 4;      // warps sharing the features of a row group
+constexpr int RM_UNROLL = 3;      // 32-feature blocks whose loads are issued together
+
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                 uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+        "{%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int NT>
+__global__ void __launch_bounds__(256, NT <= 2 ? 4 : 2)
+router_mma_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat16 *__restrict__ W_r,
+                  int64_t Ttok, int F, int E, int k, int32_t *__restrict__ idx, float *__restrict__ w,
+                  int *__restrict__ counts, int *__restrict__ perm, int64_t cap, int stage_w,
+                  int chunk, uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks, int scalar_blocks,
+                  const ScalarsArgs scalars)
+{
+    grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
+    if ((int)blockIdx.x < scalar_blocks) {
+        // leading blocks: SSD step sizes and tile log-decays (they depend on dt only); being
+        // short, they also stagger the start of the router blocks that follow them on an SM
+        ssd_scalars_block(scalars, blockIdx.x);
+        return;
+    }
+    const int rblock = (int)blockIdx.x - scalar_blocks;       // index among the router blocks
+    constexpr int EPAD = 8 * NT;
+    extern __shared__ __align__(16) unsigned char router_smem[];
+    __shared__ int s_cnt[SWIMBA_MAX_EXPERTS], s_base[SWIMBA_MAX_EXPERTS];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int *s_ent = reinterpret_cast<int *>(router_smem);              // [chunk * k] expert | rank << 8
+    float *s_part = reinterpret_cast<float *>(router_smem + (((size_t)chunk * k * sizeof(int) + 15) & ~(size_t)15));
+    unsigned char *sW = reinterpret_cast<unsigned char *>(s_part + RM_TOK * RM_KSPLIT * EPAD);
+    const int w_stride = F * 2 + 64;                                 // bytes per staged row
+    if (stage_w) {
+        const int vec_per_row = F >> 3;
+        const uint4 *src = reinterpret_cast<const uint4 *>(W_r);
+        for (int i = tid; i < EPAD * vec_per_row; i += blockDim.x) {
+            const int e = i / vec_per_row, v = i - e * vec_per_row;
+            const uint4 val = e < E ? src[(int64_t)e * vec_per_row + v] : make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4 *>(sW + e * w_stride + v * 16) = val;
+        }
+    }
+    const int tg = warp >> 2, ks = warp & 3;          // row group, feature quarter
+    const int g = lane >> 2, c = lane & 3;            // MMA row / column-pair of this lane
+    const int fq = F / RM_KSPLIT, nblk = fq / 32;
+    const int f_lane = ks * fq + 8 * c;               // first feature this lane reads
+    const int tl = tid >> 3, sub = tid & 7;           // finalisation: token of the step, lane of 8
+    const int64_t nchunks = ceil_div64(Ttok, chunk);
+    for (int64_t cidx = rblock; cidx < nchunks; cidx += router_blocks) {
+        const int64_t tbeg = cidx * chunk;
+        const int64_t tend = (tbeg + chunk < Ttok) ? tbeg + chunk : Ttok;
+        if (tid < SWIMBA_MAX_EXPERTS) s_cnt[tid] = 0;
+        if (zero_out) {
+            // the mixed-stream rows of this chunk start at zero: the projection adds its slots
+            const int64_t nz = (tend - tbeg) * zero_vec_per_token;
+            uint4 *z = zero_out + tbeg * zero_vec_per_token;
+            for (int64_t i = tid; i < nz; i += blockDim.x) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncthreads();
+        for (int64_t t0 = tbeg; t0 < tend; t0 += RM_TOK) {
+            // rows past the chunk repeat its last token; their results are never written
+            const int64_t r0 = t0 + tg * 16 + g, r1 = r0 + 8;
+            const __nv_bfloat16 *p0 = u + (r0 < tend ? r0 : tend - 1) * F + f_lane;
+            const __nv_bfloat16 *p1 = u + (r1 < tend ? r1 : tend - 1) * F + f_lane;
+            float acc[NT][4];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+            for (int j0 = 0; j0 < nblk; j0 += RM_UNROLL) {
+                uint4 xa[RM_UNROLL], xb[RM_UNROLL];
+#pragma unroll
+                for (int jj = 0; jj < RM_UNROLL; ++jj) {
+                    if (j0 + jj < nblk) {
+                        xa[jj] = *reinterpret_cast<const uint4 *>(p0 + (j0 + jj) * 32);
+                        xb[jj] = *reinterpret_cast<const uint4 *>(p1 + (j0 + jj) * 32);
+                    }
+                }
+#pragma unroll
+                for (int jj = 0; jj < RM_UNROLL; ++jj) {
+                    if (j0 + jj < nblk) {
+                        const int f = f_lane + (j0 + jj) * 32;
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const int e = nt * 8 + g;
+                            uint4 wv;
+                            if (stage_w) wv = *reinterpret_cast<const uint4 *>(sW + e * w_stride + f * 2);
+                            else wv = e < E ? __ldg(reinterpret_cast<const uint4 *>(W_r + (int64_t)e * F + f))
+                                            : make_uint4(0u, 0u, 0u, 0u);
+                            mma_bf16_16x8x16(acc[nt], xa[jj].x, xb[jj].x, xa[jj].y, xb[jj].y, wv.x, wv.y);
+                            mma_bf16_16x8x16(acc[nt], xa[jj].z, xb[jj].z, xa[jj].w, xb[jj].w, wv.z, wv.w);
+                        }
+                    }
+                }
+            }
+            // partial logits of this warp's feature quarter: s_part[token][quarter][expert]
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float *q0 = s_part + ((tg * 16 + g) * RM_KSPLIT + ks) * EPAD + nt * 8 + 2 * c;
+                *reinterpret_cast<float2 *>(q0) = make_float2(acc[nt][0], acc[nt][1]);
+                *reinterpret_cast<float2 *>(q0 + 8 * RM_KSPLIT * EPAD) = make_float2(acc[nt][2], acc[nt][3]);
+            }
+            __syncthreads();
+            // softmax over ALL experts of the token (padding experts count as -inf)
+            float gv[NT], pv[NT];
+            float m = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                const int e = sub + 8 * i;
+                const float *q = s_part + tl * RM_KSPLIT * EPAD + e;
+                float sum = q[0];
+#pragma unroll
+                for (int s = 1; s < RM_KSPLIT; ++s) sum += q[s * EPAD];
+                gv[i] = e < E ? sum : -INFINITY;
+                m = fmaxf(m, gv[i]);
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            float z = 0.f;
+#pragma unroll
+            for (int i = 0; i < NT; ++i) {
+                pv[i] = expf(gv[i] - m);
+                z += pv[i];
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+            // k rounds of "largest remaining logit, lowest index on ties"; weights are NOT
+            // renormalised
+            const int64_t t = t0 + tl;
+            for (int j = 0; j < k; ++j) {
+                float bg = gv[0], bp = pv[0];
+                int be = sub;
+#pragma unroll
+                for (int i = 1; i < NT; ++i)
+                    if (gv[i] > bg) { bg = gv[i]; bp = pv[i]; be = sub + 8 * i; }
+#pragma unroll
+                for (int o = 4; o > 0; o >>= 1) {
+                    const float og = __shfl_xor_sync(0xffffffffu, bg, o);
+                    const float op = __shfl_xor_sync(0xffffffffu, bp, o);
+                    const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+                    if (og > bg || (og == bg && oe < be)) { bg = og; bp = op; be = oe; }
+                }
+#pragma unroll
+                for (int i = 0; i < NT; ++i) if (sub + 8 * i == be) gv[i] = -INFINITY;
+                if (sub == 0 && t < tend) {
+                    idx[t * k + j] = be;
+                    w[t * k + j] = bp / z;
+                    if (counts) {
+                        const int rank = atomicAdd(&s_cnt[be], 1);
+                        s_ent[(int)(t - tbeg) * k + j] = be | (rank << 8);
+                    }
+                }
+            }
+            __syncthreads();        // s_part is rewritten by the next step
+        }
+        if (counts) {
+            if (tid < E) s_base[tid] = atomicAdd(&counts[tid], s_cnt[tid]);
+            __syncthreads();
+            const int n_ent = (int)(tend - tbeg) * k;
+            for (int i = tid; i < n_ent; i += blockDim.x) {
+                const int ent = s_ent[i], e = ent & 255;
+                perm[(int64_t)e * cap + s_base[e] + (ent >> 8)] = (int)(tbeg * k + i);
+            }
+        }
+        __syncthreads();
+    }
+}
+
 // One expert: the softmax is identically 1 and every token is routed to expert 0.
 __global__ void __launch_bounds__(256)
 router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__restrict__ w,
@@ -203,6 +390,52 @@ router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__re
         if (counts) perm[t] = (int)t;
     }
     if (counts && blockIdx.x == 0 && threadIdx.x == 0) counts[0] = (int)Ttok;
+}
+
+static int router_chunk(int64_t Ttok, int sm_count)
+{
+    // enough chunks to give every SM four blocks, between 32 and ROUTER_MAX_CHUNK tokens
+    int chunk = (int)(Ttok / (4 * (int64_t)sm_count));
+    chunk = (chunk + 31) / 32 * 32;
+    if (chunk < 32) chunk = 32;
+    if (chunk > ROUTER_MAX_CHUNK) chunk = ROUTER_MAX_CHUNK;
+    return chunk;
+}
+
+static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_bfloat16 *W_r,
+                             int64_t Ttok, int F, int E, int k, int32_t *idx, float *w, int *counts,
+                             int *perm, int64_t cap, int sm_count, void *zero_out,
+                             int zero_bytes_per_token, const ScalarsArgs &scalars)
+{
+    const int NT = E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8;
+    const int chunk = router_chunk(Ttok, sm_count);
+    const size_t w_bytes = (size_t)NT * 8 * (F * 2 + 64);
+    const int stage_w = w_bytes <= 64 * 1024 ? 1 : 0;
+    const size_t smem = (((size_t)chunk * k * sizeof(int) + 15) & ~(size_t)15) +
+                        (size_t)RM_TOK * RM_KSPLIT * NT * 8 * sizeof(float) + (stage_w ? w_bytes : 0);
+    int64_t blocks = ceil_div64(Ttok, chunk);
+    const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);
+    if (blocks > cap_blocks) blocks = cap_blocks;
+    const int64_t extra = scalars_blocks(scalars);
+    ctx.begin(STAGE_ROUTER);
+#define SWIMBA_ROUTER_MMA_CASE(NTV)                                                             \
+    do {                                                                                        \
+        auto kern = router_mma_kernel<NTV>;                                                     \
+        if (smem > 32 * 1024 &&  /* static shared memory counts toward the 48 KB default */     \
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,             \
+                                 (int)smem) != cudaSuccess)                                     \
+            return SWIMBA_ERR_CUDA;                                                             \
+        kern<<<(unsigned)(blocks + extra), 256, smem, ctx.stream>>>(                            \
+            u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk, (uint4 *)zero_out, \
+            zero_bytes_per_token / 16, (int)blocks, (int)extra, scalars);                                   \
+    } while (0)
+    if (NT == 1) SWIMBA_ROUTER_MMA_CASE(1);
+    else if (NT == 2) SWIMBA_ROUTER_MMA_CASE(2);
+    else if (NT == 4) SWIMBA_ROUTER_MMA_CASE(4);
+    else SWIMBA_ROUTER_MMA_CASE(8);
+#undef SWIMBA_ROUTER_MMA_CASE
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
 template <typename T>
@@ -220,14 +453,15 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         ctx.end();
         return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
     }
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (F % (32 * RM_KSPLIT) == 0 && E <= 64)
+            return launch_router_mma(ctx, u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, sm_count,
+                                     zero_out, zero_bytes_per_token, scalars);
+    }
     const size_t w_bytes = (size_t)E * F * sizeof(T);
     const int stage_w = (w_bytes <= 64 * 1024 && (w_bytes & 15) == 0) ? 1 : 0;
     const size_t smem = (size_t)ROUTER_MAX_CHUNK * SWIMBA_MAX_TOPK * sizeof(int) + (stage_w ? w_bytes : 0);
-    // chunk: enough chunks to give every SM four blocks, between 32 and ROUTER_MAX_CHUNK tokens
-    int chunk = (int)(Ttok / (4 * (int64_t)sm_count));
-    chunk = (chunk + 31) / 32 * 32;
-    if (chunk < 32) chunk = 32;
-    if (chunk > ROUTER_MAX_CHUNK) chunk = ROUTER_MAX_CHUNK;
+    const int chunk = router_chunk(Ttok, sm_count);
     ctx.begin(STAGE_ROUTER);
 #define SWIMBA_ROUTER_CASE(EPV, TPWV)                                                          \
     do {                                                                                       \
@@ -239,10 +473,10 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         int64_t blocks = ceil_div64(Ttok, chunk);                                              \
         const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);             \
         if (blocks > cap_blocks) blocks = cap_blocks;                                          \
-        const int64_t extra = (scalars_units(scalars) + 1) / 2;                                \
+        const int64_t extra = scalars_blocks(scalars);                                \
         kern<<<(unsigned)(blocks + extra), warps * 32, smem, ctx.stream>>>(                    \
             u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk, (uint4 *)zero_out, \
-            zero_bytes_per_token / 16, (int)blocks, scalars);                                  \
+            zero_bytes_per_token / 16, (int)blocks, (int)extra, scalars);                                  \
     } while (0)
     if (E <= 2) SWIMBA_ROUTER_CASE(2, 8);
     else if (E <= 4) SWIMBA_ROUTER_CASE(4, 8);

@@ -94,14 +94,13 @@ struct __align__(16) SsdSmall {
 __host__ __device__ inline int pairs_per_group(int H, int G) { return (H / G + NHD - 1) / NHD; }
 }  // namespace
 
-// Stand-alone launch of the step sizes and tile log-decays (one unit per block).
-__global__ void __launch_bounds__(SCALARS_TILE)
+// Stand-alone launch of the step sizes and tile log-decays.
+__global__ void __launch_bounds__(256)
 ssd_scalars_kernel(const ScalarsArgs args)
 {
-    __shared__ float s_tot[4];
     grid_dep_launch();
     grid_dep_wait();      // (launched behind the projection kernel in the single-expert path)
-    ssd_scalars_unit(args, blockIdx.x, true, threadIdx.x, s_tot);
+    ssd_scalars_block(args, blockIdx.x);
 }
 
 __global__ void __launch_bounds__(SSD_THREADS, 1)
@@ -688,7 +687,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     if (!scalars_done) {
         const ScalarsArgs sa = ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace);
         ctx.begin(STAGE_SSD_SCALARS);
-        launch_kernel(ssd_scalars_kernel, dim3((unsigned)scalars_units(sa)), dim3(SCALARS_TILE), 0,
+        launch_kernel(ssd_scalars_kernel, dim3((unsigned)scalars_blocks(sa)), dim3(256), 0,
                       ctx.stream, true, sa);
         ctx.end();
     }

@@ -23,33 +23,71 @@ __host__ __device__ inline int64_t scalars_units(const ScalarsArgs &a)
     return a.dl ? (int64_t)(a.Lpad / SCALARS_TILE) * a.H * a.B : 0;
 }
 
-// One (tile, head, sequence) unit, worked by 128 consecutive threads (i = 0..127 inside the unit).
-// Every thread of the block must call this (it holds a __syncthreads); threads whose unit is out
-// of range pass active = false.  s_tot: four floats of shared memory private to the unit.
-__device__ __forceinline__ void ssd_scalars_unit(const ScalarsArgs &a, int64_t unit, bool active, int i,
-                                                 float *s_tot)
+constexpr int SCALARS_UNITS_PER_BLOCK = 16;     // 256 threads: 8 warps x 2 units
+
+// NU consecutive (tile, head, sequence) units, worked by one warp without any block-level
+// synchronisation: lane l owns tokens 4l .. 4l+3 of a tile; the loads of all NU units are issued
+// before the first use.  The tile's running log-decay is summed token by token inside a lane and
+// by a shuffle scan across lanes.
+template <int NU>
+__device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t unit0, int lane)
 {
     const int ntile = a.Lpad / SCALARS_TILE;
-    const int lane = i & 31, wq = i >> 5;
-    const int tile = (int)(unit % ntile);
-    const int h = (int)((unit / ntile) % a.H);
-    const int b = (int)(unit / ((int64_t)ntile * a.H));
-    const int t = tile * SCALARS_TILE + i;
-    float delta = 0.f, l2 = 0.f;
-    if (active) {
-        const float raw = (a.dt && t < a.L) ? a.dt[((int64_t)b * a.L + t) * a.H + h] : 0.f;
-        delta = t < a.L ? softplus_f(raw + a.dt_bias[h]) : 0.f;
-        l2 = delta * (a.A[h] * 1.4426950408889634f);
+    const int64_t nunits = scalars_units(a);
+    float raw[NU][4];
+    int hh[NU], tt[NU];
+    int64_t out[NU];
+#pragma unroll
+    for (int q = 0; q < NU; ++q) {
+        const int64_t unit = unit0 + q;
+        const bool act = unit < nunits;
+        const int tile = act ? (int)(unit % ntile) : 0;
+        const int h = act ? (int)((unit / ntile) % a.H) : 0;
+        const int64_t b = act ? unit / ((int64_t)ntile * a.H) : 0;
+        const int t = tile * SCALARS_TILE + lane * 4;
+        hh[q] = h;
+        tt[q] = t;
+        out[q] = act ? (b * a.H + h) * a.Lpad + t : -1;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            raw[q][i] = (act && a.dt && t + i < a.L) ? a.dt[(b * a.L + t + i) * a.H + h] : 0.f;
     }
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float nb = __shfl_up_sync(0xffffffffu, l2, o);
-        if (lane >= o) l2 += nb;
+    for (int q = 0; q < NU; ++q) {
+        if (out[q] < 0) continue;                       // (uniform over the warp)
+        const float bias = a.dt_bias[hh[q]];
+        const float a2 = a.A[hh[q]] * 1.4426950408889634f;
+        float d[4], p[4], run = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            d[i] = tt[q] + i < a.L ? softplus_f(raw[q][i] + bias) : 0.f;
+            run += d[i] * a2;
+            p[i] = run;
+        }
+        float incl = run;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float nb = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += nb;
+        }
+        const float excl = incl - run;
+        float4 *dst = reinterpret_cast<float4 *>(a.dl + out[q]);
+        dst[0] = make_float4(d[0], excl + p[0], d[1], excl + p[1]);
+        dst[1] = make_float4(d[2], excl + p[2], d[3], excl + p[3]);
     }
-    if (lane == 31) s_tot[wq] = l2;
-    __syncthreads();
-    for (int w = 0; w < wq; ++w) l2 += s_tot[w];
-    if (active) a.dl[((int64_t)b * a.H + h) * a.Lpad + t] = make_float2(delta, l2);
+}
+
+// The block's share: SCALARS_UNITS_PER_BLOCK units starting at block * SCALARS_UNITS_PER_BLOCK
+// (256 threads).
+__device__ __forceinline__ void ssd_scalars_block(const ScalarsArgs &a, int64_t block)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    ssd_scalars_warp<2>(a, block * SCALARS_UNITS_PER_BLOCK + warp * 2, lane);
+}
+
+__host__ __device__ inline int64_t scalars_blocks(const ScalarsArgs &a)
+{
+    return (scalars_units(a) + SCALARS_UNITS_PER_BLOCK - 1) / SCALARS_UNITS_PER_BLOCK;
 }
 
 }  // namespace swimba
