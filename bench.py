@@ -36,8 +36,9 @@ NSETS = 4   # rotating input sets: together several times the 126 MB L2
 NCU_TRAFFIC_BYTES = {
     # workload small_lm, one launch each (profiles/forward_small_lm_kernels.md); ncu flushes caches
     # before a launch and part of a kernel's writes can still sit in L2 when it ends
-    "ssd_tiles": 77.136e6, "router_topk": 25.212e6, "expert_gemm": 28.638e6, "mix_slots": 16.792e6,
-    "ssd_scalars": 1.578e6,
+    # (the router launch includes the SSD step sizes; the projection reads the cleared rows it adds to;
+    # the slot-mix and stand-alone step-size kernels do not run in this workload: no capture)
+    "ssd_tiles": 78.175e6, "router_topk": 26.788e6, "expert_gemm": 36.986e6,
     # decode workload (profiles/decode_update_kernel.md)
     "decode_update": 479.8e6,
 }
@@ -112,7 +113,10 @@ def algorithmic_work(cfg: synth.LayerConfig):
     H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.Q
     es = 2 if cfg.dtype == "bf16" else 4
     w = {}
-    w["router_topk"] = dict(bound="hbm", work=T * F * es + E * F * es + T * k * 8)
+    # with more than one expert the router launch also produces the SSD step sizes (dt in, (Delta,
+    # log-decay) pairs out) of the bf16 tile path
+    fused_scalars = T * H * 12 if (E > 1 and cfg.dtype == "bf16") else 0
+    w["router_topk"] = dict(bound="hbm", work=T * F * es + E * F * es + T * k * 8 + fused_scalars)
     w["expert_gemm"] = dict(bound="tensor", work=2.0 * T * k * F * S)
     w["mix_slots"] = dict(bound="hbm", work=T * k * S * es + T * S * es)
     w["project_mix_simt"] = dict(bound="alu", work=2.0 * T * k * F * S)

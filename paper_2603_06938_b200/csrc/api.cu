@@ -164,7 +164,8 @@ int set_device(swimba_handle *h)
     return SWIMBA_OK;
 }
 
-// Router + projection + mix into BC (dtype, or fp32 when bc_fp32).
+// Router + projection + mix into BC (dtype, or fp32 when bc_fp32).  scalars != NULL: the SSD step
+// sizes of the same call (they depend on dt only) are produced beside the router.
 int run_route_mix(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const void *u,
                   int64_t T, void *BC, bool bc_fp32, int32_t *idx, float *wt, void *gemm_ws,
                   const ScalarsArgs *scalars = nullptr)
@@ -358,9 +359,8 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
-    // The SSD step sizes depend on dt only: with more than one expert they ride along as extra
-    // blocks of the router launch.
-    const bool fuse = h->cfg.n_experts > 1 && ssd_tiles_supported(h->cfg.dtype, h->cfg.head_dim, h->cfg.d_state);
+    // The SSD step sizes depend on dt only: their kernel runs beside the router.
+    const bool fuse = ssd_tiles_supported(h->cfg.dtype, h->cfg.head_dim, h->cfg.d_state);
     const ScalarsArgs sa = fuse ? ssd_scalars_args(dt, w->A, w->dt_bias, B, L, h->cfg.n_heads, ws + l.ssd)
                                 : ScalarsArgs{};
     rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm, fuse ? &sa : nullptr);

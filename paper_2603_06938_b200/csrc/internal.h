@@ -9,8 +9,9 @@ namespace swimba {
 // When counts is given (zeroed beforehand) the (token, slot) pairs are also grouped by expert:
 // perm[e * cap + i], i < counts[e], lists the entries t*k + j routed to expert e.
 // zero_out (may be NULL): a [T, zero_bytes_per_token] buffer the kernel clears on the way (the
-// mixed streams, when the projection adds its slots in place).  scalars.dl != NULL: the SSD step
-// sizes are computed by extra blocks of the same launch (not with a single expert).
+// mixed streams, when the projection adds its slots in place).  scalars.dl != NULL: the call also
+// produces the SSD step sizes and tile log-decays of the same forward (they depend on dt only and
+// run beside the router, inside its launch or as a kernel in front of it).
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,
                   int E, int k, int32_t *idx, float *w, int *counts, int *perm, int64_t cap,
                   int sm_count, void *zero_out, int zero_bytes_per_token, const ScalarsArgs &scalars);
@@ -36,9 +37,10 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
 bool ssd_tiles_supported(int dtype, int P, int N);
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);
 // scalars_done: the step sizes and tile log-decays (ssd_scalars_args over the same workspace) have
-// already been produced, as extra blocks of the router kernel.
+// already been produced earlier in the stream (launch_router with scalars, or launch_ssd_scalars).
 ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,
                              void *workspace);
+int launch_ssd_scalars(LaunchCtx &ctx, const ScalarsArgs &args);
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
                      const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
                      int chunk, int sm_count, void *y, float *h_final, void *workspace,

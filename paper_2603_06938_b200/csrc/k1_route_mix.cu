@@ -1,6 +1,7 @@
 // K1 (SIMT part): router logits + softmax + top-k, and the plain projection/mix used by the
 // fp32 path and by decode.  (Router softmax equation and top-k rule; Theorem 1, mixed streams.)
 #include "internal.h"
+#include "tc05.cuh"
 #include <type_traits>
 
 namespace swimba {
@@ -29,17 +30,10 @@ __global__ void __launch_bounds__(256)
 router_topk_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Ttok, int F, int E,
                    int k, int32_t *__restrict__ idx, float *__restrict__ w, int *__restrict__ counts,
                    int *__restrict__ perm, int64_t cap, int stage_w, int chunk,
-                   uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks, int scalar_blocks,
-                   const ScalarsArgs scalars)
+                   uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks)
 {
     grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
-    if ((int)blockIdx.x < scalar_blocks) {
-        // leading blocks: SSD step sizes and tile log-decays (they depend on dt only); being
-        // short, they also stagger the start of the router blocks that follow them on an SM
-        ssd_scalars_block(scalars, blockIdx.x);
-        return;
-    }
-    const int rblock = (int)blockIdx.x - scalar_blocks;       // index among the router blocks
+    const int rblock = (int)blockIdx.x;
     constexpr int V = TPW * EP;                 // values per lane before the butterfly
     constexpr int R = V > 32 ? V / 32 : 1;      // values per lane after it (adjacent experts)
     constexpr int DUP = V >= 32 ? 1 : 32 / V;   // lanes holding the same value after it
@@ -223,13 +217,13 @@ __global__ void __launch_bounds__(256, NT <= 2 ? 4 : 2)
 router_mma_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat16 *__restrict__ W_r,
                   int64_t Ttok, int F, int E, int k, int32_t *__restrict__ idx, float *__restrict__ w,
                   int *__restrict__ counts, int *__restrict__ perm, int64_t cap, int stage_w,
-                  int chunk, uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks, int scalar_blocks,
-                  const ScalarsArgs scalars)
+                  int chunk, uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_blocks,
+                  int scalar_blocks, const ScalarsArgs scalars)
 {
     grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
     if ((int)blockIdx.x < scalar_blocks) {
-        // leading blocks: SSD step sizes and tile log-decays (they depend on dt only); being
-        // short, they also stagger the start of the router blocks that follow them on an SM
+        // leading blocks: SSD step sizes and tile log-decays of the same call (they depend on dt
+        // only); being short, they also stagger the start of the router blocks behind them
         ssd_scalars_block(scalars, blockIdx.x);
         return;
     }
@@ -377,6 +371,247 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ u, const __nv_bfloat16 *__re
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Streaming router (bf16): the token features are the only large operand, so the kernel is built
+// around keeping HBM reads in flight and contiguous.  A CTA owns 64-token tiles (static round
+// robin); warp w of its four holds tokens 16 w .. 16 w + 15 of a tile and runs its own pipeline: an
+// elected lane issues TMA loads of [16 tokens x 64 features] boxes (128-byte rows, 128-byte swizzle;
+// rows and features past the end are zero-filled), four to a stage (512 contiguous bytes of every
+// row), into the warp's private ring of stages; the warp consumes a stage with m16n8k16 products
+// against the router matrix, which sits in shared memory already arranged as B fragments (one
+// 8-byte read per lane and product), and refills it at once with the stage that comes a ring later
+// (of the next tile if need be).  No warp waits for another inside the feature loop, and the
+// loads of the next tile proceed while a tile's softmax, top-k and list bookkeeping run.
+//
+// Logit summation order (fixed, so results are reproducible run to run): features ascending in
+// blocks of 16, each block one tensor-core product accumulated in fp32 (with at most 16 experts,
+// even and odd blocks in two accumulators that are added at the end).  bf16 products are exact
+// in fp32; the additions are those of the tensor core's accumulator.  A token's logits end up on
+// the four lanes of its row (lane c holds experts 8 n + 2 c, 8 n + 2 c + 1); softmax and top-k run
+// across them.
+// ------------------------------------------------------------------------------------------
+constexpr int RS_TOK = 64;                       // tokens per tile
+constexpr int RS_CW = RS_TOK / 16;               // warps
+constexpr int RS_BOX = 64;                       // features per TMA box (128-byte rows)
+constexpr int RS_NBOX = 4;                       // boxes per stage
+constexpr int RS_BK = RS_BOX * RS_NBOX;          // features per stage
+constexpr int RS_BOX_BYTES = 16 * 128;
+constexpr int RS_STAGE_BYTES = RS_NBOX * RS_BOX_BYTES;
+constexpr int RS_THREADS = 32 * RS_CW;
+constexpr int RS_MAX_STAGES = 4;
+
+struct RouterStreamSmall {
+    uint64_t full[RS_CW][RS_MAX_STAGES];
+    int cnt[SWIMBA_MAX_EXPERTS], base[SWIMBA_MAX_EXPERTS];
+    int abort_flag;
+};
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+template <int NT>
+__global__ void __launch_bounds__(RS_THREADS)
+router_stream_kernel(const __grid_constant__ CUtensorMap tmap_u, const __nv_bfloat16 *__restrict__ W_r,
+                     int64_t Ttok, int F, int E, int k, int32_t *__restrict__ idx, float *__restrict__ w,
+                     int *__restrict__ counts, int *__restrict__ perm, int64_t cap,
+                     uint4 *__restrict__ zero_out, int zero_vec_per_token, int router_ctas,
+                     int nstages, int *d_status)
+{
+    grid_dep_launch();      // the projection kernel may set itself up under this kernel's tail
+    const int cta = (int)blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int cw = __shfl_sync(0xffffffffu, tid >> 5, 0);
+    extern __shared__ __align__(16) unsigned char router_smem[];
+    unsigned char *ring = reinterpret_cast<unsigned char *>(((uintptr_t)router_smem + 1023) & ~(uintptr_t)1023);
+    const int KB = ceil_div(F, RS_BK);                               // stages per tile
+    constexpr int KSTEPS = RS_BK / 16;                               // products per stage
+    uint2 *sWp = reinterpret_cast<uint2 *>(ring + (size_t)RS_CW * nstages * RS_STAGE_BYTES);   // [KB*KSTEPS][NT][32]
+    int *s_ent = reinterpret_cast<int *>(sWp + (size_t)KB * KSTEPS * NT * 32);                  // [RS_TOK * k]
+    RouterStreamSmall *sm = reinterpret_cast<RouterStreamSmall *>(
+        (reinterpret_cast<uintptr_t>(s_ent + RS_TOK * k) + 15) & ~(uintptr_t)15);
+    int *abort_flag = &sm->abort_flag;
+
+    if (tid == 0) {
+        for (int q = 0; q < RS_CW; ++q)
+            for (int s = 0; s < RS_MAX_STAGES; ++s) tc::mbar_init(&sm->full[q][s], 1);
+        *abort_flag = 0;
+        tc::fence_mbar_init();
+    }
+    if (tid == 32) tc::prefetch_tmap(&tmap_u);
+    __syncthreads();
+    // Loads are numbered across the CTA's tiles: load `n` is feature block n % KB of the CTA's tile
+    // number n / KB and goes to stage n % nstages of the warp's ring.  The first ring-full is issued
+    // before the router matrix is staged, so that both latencies overlap.
+    const int64_t ntiles = ceil_div64(Ttok, RS_TOK);
+    const uint32_t n_loads = cta < ntiles ? (uint32_t)((ntiles - cta + router_ctas - 1) / router_ctas) * KB : 0u;
+    unsigned char *my_ring = ring + (size_t)cw * nstages * RS_STAGE_BYTES;
+    uint64_t *my_full = sm->full[cw];
+    const bool leader = tc::elect_one();
+    auto issue_load = [&](uint32_t n) {
+        const int s = n % nstages;
+        const int64_t tile = cta + (int64_t)(n / KB) * router_ctas;
+        tc::mbar_arrive_expect_tx(&my_full[s], RS_STAGE_BYTES);
+#pragma unroll
+        for (int bx = 0; bx < RS_NBOX; ++bx)
+            tc::tma_load_2d(my_ring + s * RS_STAGE_BYTES + bx * RS_BOX_BYTES, &tmap_u, &my_full[s],
+                            (int)(n % KB) * RS_BK + bx * RS_BOX, (int)(tile * RS_TOK) + cw * 16);
+    };
+    if (leader)
+        for (uint32_t n = 0; n < n_loads && n < (uint32_t)nstages; ++n) issue_load(n);
+    __syncwarp();
+    // Router matrix as B fragments: entry ((kk * NT + nt) * 32 + lane) holds, for the 16-feature
+    // block kk and expert e = 8 nt + lane / 4, the features 16 kk + 2 c, + 1 (low word) and
+    // 16 kk + 8 + 2 c, + 1 (high word), c = lane % 4; zero past E or F.  Sixteen contiguous bytes
+    // of an expert's row are the same word of four consecutive entries.
+    {
+        const int n_ent = KB * KSTEPS * NT * 32;
+        if ((E & 7) != 0 || F % RS_BK != 0) {
+            for (int i = tid; i < n_ent; i += RS_THREADS) sWp[i] = make_uint2(0u, 0u);
+            __syncthreads();
+        }
+        const uint4 *W4 = reinterpret_cast<const uint4 *>(W_r);
+        const int vec_per_row = F >> 3, n_vec = E * vec_per_row;
+#pragma unroll 4
+        for (int i = tid; i < n_vec; i += RS_THREADS) {
+            const int e = i / vec_per_row, v = i - e * vec_per_row;
+            const uint4 val = W4[i];
+            uint32_t *dst = reinterpret_cast<uint32_t *>(&sWp[((v >> 1) * NT + (e >> 3)) * 32 + (e & 7) * 4]) + (v & 1);
+            dst[0] = val.x;
+            dst[2] = val.y;
+            dst[4] = val.z;
+            dst[6] = val.w;
+        }
+    }
+    __syncthreads();
+
+    const int g = lane >> 2, c = lane & 3;
+    // ldmatrix: lane l addresses row (l % 8) + 8 * ((l / 8) % 2) of the warp's 16 rows and the
+    // 16-byte chunk 2 kk + l / 16 of the 128-byte row
+    const int lm_row = (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int lm_chunk = lane >> 4;
+    const uint32_t ring_addr = tc::smem_u32(my_ring) + lm_row * 128;
+    uint32_t n = 0;
+    for (int64_t tile = cta; tile < ntiles; tile += router_ctas) {
+        const int64_t tbeg = tile * RS_TOK;
+        const int64_t tend = (tbeg + RS_TOK < Ttok) ? tbeg + RS_TOK : Ttok;
+        if (tid < SWIMBA_MAX_EXPERTS) sm->cnt[tid] = 0;
+        if (zero_out) {
+            // the mixed-stream rows of this tile start at zero: the projection adds its slots
+            const int64_t nz = (tend - tbeg) * zero_vec_per_token;
+            uint4 *z = zero_out + tbeg * zero_vec_per_token;
+            for (int64_t i = tid; i < nz; i += RS_THREADS) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        // few expert tiles: even and odd feature blocks go to separate accumulators so that
+        // consecutive products do not wait on each other
+        constexpr int CH = NT <= 2 ? 2 : 1;
+        float accs[CH][NT][4];
+#pragma unroll
+        for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) accs[ch][nt][i] = 0.f;
+        for (int kb = 0; kb < KB; ++kb, ++n) {
+            const int s = n % nstages;
+            tc::mbar_wait(&my_full[s], (n / nstages) & 1, abort_flag, d_status);
+            const uint32_t st = ring_addr + s * RS_STAGE_BYTES;
+#pragma unroll
+            for (int kk = 0; kk < KSTEPS; ++kk) {
+                uint32_t a[4];
+                ldmatrix_x4(a, st + (kk >> 2) * RS_BOX_BYTES + ((((2 * kk) & 7) + lm_chunk) ^ (lm_row & 7)) * 16);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint2 bv = sWp[((kb * KSTEPS + kk) * NT + nt) * 32 + lane];
+                    mma_bf16_16x8x16(accs[kk % CH][nt], a[0], a[1], a[2], a[3], bv.x, bv.y);
+                }
+            }
+            // the reads above must be ordered before the TMA write that refills the stage
+            tc::fence_proxy_async_smem();
+            __syncwarp();
+            if (leader && n + nstages < n_loads) issue_load(n + nstages);
+        }
+        float acc[NT][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[nt][i] = CH == 2 ? accs[0][nt][i] + accs[CH - 1][nt][i] : accs[0][nt][i];
+        // the histogram is clear and the previous tile's lists have been written
+        __syncthreads();
+        // softmax over ALL experts of the token (padding experts count as -inf), top-k, for the
+        // two token rows of this lane in turn
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int64_t t = tbeg + cw * 16 + g + 8 * half;
+            float gv[2 * NT], pv[2 * NT];
+            float m = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 2 * NT; ++i) {
+                const int e = (i >> 1) * 8 + 2 * c + (i & 1);
+                gv[i] = e < E ? acc[i >> 1][2 * half + (i & 1)] : -INFINITY;
+                m = fmaxf(m, gv[i]);
+            }
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            float z = 0.f;
+#pragma unroll
+            for (int i = 0; i < 2 * NT; ++i) {
+                pv[i] = expf(gv[i] - m);
+                z += pv[i];
+            }
+            z += __shfl_xor_sync(0xffffffffu, z, 1);
+            z += __shfl_xor_sync(0xffffffffu, z, 2);
+            // k rounds of "largest remaining logit, lowest index on ties"; weights are NOT
+            // renormalised
+            for (int j = 0; j < k; ++j) {
+                float bg = gv[0], bp = pv[0];
+                int be = 2 * c;
+#pragma unroll
+                for (int i = 1; i < 2 * NT; ++i) {
+                    const int e = (i >> 1) * 8 + 2 * c + (i & 1);
+                    if (gv[i] > bg) { bg = gv[i]; bp = pv[i]; be = e; }
+                }
+#pragma unroll
+                for (int o = 1; o <= 2; o <<= 1) {
+                    const float og = __shfl_xor_sync(0xffffffffu, bg, o);
+                    const float op = __shfl_xor_sync(0xffffffffu, bp, o);
+                    const int oe = __shfl_xor_sync(0xffffffffu, be, o);
+                    if (og > bg || (og == bg && oe < be)) { bg = og; bp = op; be = oe; }
+                }
+#pragma unroll
+                for (int i = 0; i < 2 * NT; ++i)
+                    if ((i >> 1) * 8 + 2 * c + (i & 1) == be) gv[i] = -INFINITY;
+                if (c == 0 && t < tend) {
+                    idx[t * k + j] = be;
+                    w[t * k + j] = bp / z;
+                    if (counts) {
+                        const int rank = atomicAdd(&sm->cnt[be], 1);
+                        s_ent[(int)(t - tbeg) * k + j] = be | (rank << 8);
+                    }
+                }
+            }
+        }
+        if (counts) {
+            // lists: a shared-memory histogram ranked the tile's entries, one global atomic per
+            // expert reserves the tile's range
+            __syncthreads();
+            if (tid < E) sm->base[tid] = atomicAdd(&counts[tid], sm->cnt[tid]);
+            __syncthreads();
+            const int n_ent = (int)(tend - tbeg) * k;
+            for (int i = tid; i < n_ent; i += RS_THREADS) {
+                const int ent = s_ent[i], e = ent & 255;
+                perm[(int64_t)e * cap + sm->base[e] + (ent >> 8)] = (int)(tbeg * k + i);
+            }
+        }
+    }
+    // When launched behind the SSD step-size kernel (beside which it runs): this grid must not
+    // complete before that one has, so that every later kernel in the stream is ordered behind both.
+    grid_dep_wait();
+}
+
 // One expert: the softmax is identically 1 and every token is routed to expert 0.
 __global__ void __launch_bounds__(256)
 router_single_expert_kernel(int64_t Ttok, int32_t *__restrict__ idx, float *__restrict__ w,
@@ -402,6 +637,64 @@ static int router_chunk(int64_t Ttok, int sm_count)
     return chunk;
 }
 
+static size_t router_stream_smem(int F, int NT, int k, int nstages)
+{
+    const int KB = ceil_div(F, RS_BK);
+    return 1024 + (size_t)RS_CW * nstages * RS_STAGE_BYTES +
+           (size_t)KB * (RS_BK / 16) * NT * 32 * sizeof(uint2) + (size_t)RS_TOK * k * sizeof(int) + 16 +
+           sizeof(RouterStreamSmall);
+}
+
+// The streaming kernel needs rows that TMA can address (16-byte aligned base and row pitch), the
+// fragment-ordered router matrix in shared memory and enough tiles to occupy the GPU.
+static bool router_stream_usable(const void *u, int64_t Ttok, int F, int E, int sm_count)
+{
+    const int NT = E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8;
+    return E <= 64 && F >= RS_BOX && F % 8 == 0 && ((uintptr_t)u & 15) == 0 &&
+           (size_t)ceil_div(F, RS_BK) * (RS_BK / 16) * NT * 32 * sizeof(uint2) <= 64 * 1024 &&
+           ceil_div64(Ttok, RS_TOK) >= 3 * (int64_t)sm_count;
+}
+
+static int launch_router_stream(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_bfloat16 *W_r,
+                                int64_t Ttok, int F, int E, int k, int32_t *idx, float *w, int *counts,
+                                int *perm, int64_t cap, int sm_count, void *zero_out,
+                                int zero_bytes_per_token, bool behind_scalars)
+{
+    const int NT = E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8;
+    // ring depth: the deepest (up to RS_MAX_STAGES) that still lets two CTAs share an SM, else
+    // the deepest that fits one
+    int nstages = RS_MAX_STAGES, per_sm = 1;
+    for (int ns = RS_MAX_STAGES; ns >= 2; --ns)
+        if (2 * (router_stream_smem(F, NT, k, ns) + 1024) <= 227 * 1024) { nstages = ns; per_sm = 2; break; }
+    const size_t smem = router_stream_smem(F, NT, k, nstages);
+    CUtensorMap tmap;
+    const uint64_t dims[2] = {(uint64_t)F, (uint64_t)Ttok};
+    const uint64_t strides[1] = {(uint64_t)F * 2};
+    const uint32_t box[2] = {(uint32_t)RS_BOX, 16u};
+    if (!encode_tmap_bf16(&tmap, u, 2, dims, strides, box)) return SWIMBA_ERR_CUDA;
+    const int64_t ntiles = ceil_div64(Ttok, RS_TOK);
+    int64_t ctas = (int64_t)sm_count * per_sm;
+    if (ctas > ntiles) ctas = ntiles;
+    ctx.begin(STAGE_ROUTER);
+#define SWIMBA_ROUTER_STREAM_CASE(NTV)                                                          \
+    do {                                                                                        \
+        auto kern = router_stream_kernel<NTV>;                                                  \
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,             \
+                                 (int)smem) != cudaSuccess)                                     \
+            return SWIMBA_ERR_CUDA;                                                             \
+        launch_kernel(kern, dim3((unsigned)ctas), dim3(RS_THREADS), smem, ctx.stream, behind_scalars, tmap, \
+                      W_r, Ttok, F, E, k, idx, w, counts, perm, cap, (uint4 *)zero_out,         \
+                      zero_bytes_per_token / 16, (int)ctas, nstages, ctx.d_status);             \
+    } while (0)
+    if (NT == 1) SWIMBA_ROUTER_STREAM_CASE(1);
+    else if (NT == 2) SWIMBA_ROUTER_STREAM_CASE(2);
+    else if (NT == 4) SWIMBA_ROUTER_STREAM_CASE(4);
+    else SWIMBA_ROUTER_STREAM_CASE(8);
+#undef SWIMBA_ROUTER_STREAM_CASE
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
 static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_bfloat16 *W_r,
                              int64_t Ttok, int F, int E, int k, int32_t *idx, float *w, int *counts,
                              int *perm, int64_t cap, int sm_count, void *zero_out,
@@ -409,6 +702,7 @@ static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_
 {
     const int NT = E <= 8 ? 1 : E <= 16 ? 2 : E <= 32 ? 4 : 8;
     const int chunk = router_chunk(Ttok, sm_count);
+    const int64_t extra = scalars_blocks(scalars, 256);      // leading blocks for the SSD step sizes
     const size_t w_bytes = (size_t)NT * 8 * (F * 2 + 64);
     const int stage_w = w_bytes <= 64 * 1024 ? 1 : 0;
     const size_t smem = (((size_t)chunk * k * sizeof(int) + 15) & ~(size_t)15) +
@@ -416,7 +710,6 @@ static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_
     int64_t blocks = ceil_div64(Ttok, chunk);
     const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);
     if (blocks > cap_blocks) blocks = cap_blocks;
-    const int64_t extra = scalars_blocks(scalars);
     ctx.begin(STAGE_ROUTER);
 #define SWIMBA_ROUTER_MMA_CASE(NTV)                                                             \
     do {                                                                                        \
@@ -425,9 +718,10 @@ static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_
             cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,             \
                                  (int)smem) != cudaSuccess)                                     \
             return SWIMBA_ERR_CUDA;                                                             \
-        kern<<<(unsigned)(blocks + extra), 256, smem, ctx.stream>>>(                            \
-            u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk, (uint4 *)zero_out, \
-            zero_bytes_per_token / 16, (int)blocks, (int)extra, scalars);                                   \
+        launch_kernel(kern, dim3((unsigned)(extra + blocks)), dim3(256), smem, ctx.stream, false, \
+                      u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk,         \
+                      (uint4 *)zero_out, zero_bytes_per_token / 16, (int)blocks, (int)extra,    \
+                      scalars);                                                                 \
     } while (0)
     if (NT == 1) SWIMBA_ROUTER_MMA_CASE(1);
     else if (NT == 2) SWIMBA_ROUTER_MMA_CASE(2);
@@ -445,18 +739,33 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
                            const ScalarsArgs &scalars)
 {
     const int warps = 8;
+    // The SSD step sizes of the same call (scalars.dl != NULL) depend on dt only and run beside the
+    // router: as the leading blocks of the register-fed tensor-core kernel, else as a kernel of
+    // their own in front of the router (the streaming router then starts while it runs).
+    bool behind_scalars = false;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (E > 1 && !router_stream_usable(u, Ttok, F, E, sm_count) && F % (32 * RM_KSPLIT) == 0 && E <= 64)
+            return launch_router_mma(ctx, u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, sm_count,
+                                     zero_out, zero_bytes_per_token, scalars);
+        behind_scalars = E > 1 && scalars.dl && router_stream_usable(u, Ttok, F, E, sm_count);
+    }
+    if (scalars.dl) {
+        const int rc = launch_ssd_scalars(ctx, scalars);
+        if (rc != SWIMBA_OK) return rc;
+    }
     if (E == 1) {
         int64_t blocks = ceil_div64(Ttok, 256);
         if (blocks > (int64_t)sm_count * 8) blocks = (int64_t)sm_count * 8;
         ctx.begin(STAGE_ROUTER);
-        router_single_expert_kernel<<<(unsigned)blocks, 256, 0, ctx.stream>>>(Ttok, idx, w, counts, perm);
+        launch_kernel(router_single_expert_kernel, dim3((unsigned)blocks), dim3(256), 0, ctx.stream,
+                      false, Ttok, idx, w, counts, perm);
         ctx.end();
         return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
     }
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
-        if (F % (32 * RM_KSPLIT) == 0 && E <= 64)
-            return launch_router_mma(ctx, u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, sm_count,
-                                     zero_out, zero_bytes_per_token, scalars);
+        if (router_stream_usable(u, Ttok, F, E, sm_count))
+            return launch_router_stream(ctx, u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, sm_count,
+                                        zero_out, zero_bytes_per_token, behind_scalars);
     }
     const size_t w_bytes = (size_t)E * F * sizeof(T);
     const int stage_w = (w_bytes <= 64 * 1024 && (w_bytes & 15) == 0) ? 1 : 0;
@@ -473,10 +782,9 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         int64_t blocks = ceil_div64(Ttok, chunk);                                              \
         const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);             \
         if (blocks > cap_blocks) blocks = cap_blocks;                                          \
-        const int64_t extra = scalars_blocks(scalars);                                \
-        kern<<<(unsigned)(blocks + extra), warps * 32, smem, ctx.stream>>>(                    \
-            u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk, (uint4 *)zero_out, \
-            zero_bytes_per_token / 16, (int)blocks, (int)extra, scalars);                                  \
+        launch_kernel(kern, dim3((unsigned)blocks), dim3(warps * 32), smem, ctx.stream, false,   \
+                      u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk,        \
+                      (uint4 *)zero_out, zero_bytes_per_token / 16, (int)blocks);              \
     } while (0)
     if (E <= 2) SWIMBA_ROUTER_CASE(2, 8);
     else if (E <= 4) SWIMBA_ROUTER_CASE(4, 8);

@@ -98,8 +98,10 @@ __host__ __device__ inline int pairs_per_group(int H, int G) { return (H / G + N
 __global__ void __launch_bounds__(256)
 ssd_scalars_kernel(const ScalarsArgs args)
 {
+    // Everything earlier in the stream has completed once the wait returns; only then may the
+    // kernel behind this one (the streaming router, which writes without waiting) be let in.
+    grid_dep_wait();
     grid_dep_launch();
-    grid_dep_wait();      // (launched behind the projection kernel in the single-expert path)
     ssd_scalars_block(args, blockIdx.x);
 }
 
@@ -654,6 +656,16 @@ ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bi
     return a;
 }
 
+int launch_ssd_scalars(LaunchCtx &ctx, const ScalarsArgs &sa)
+{
+    if (scalars_units(sa) <= 0) return SWIMBA_OK;
+    ctx.begin(STAGE_SSD_SCALARS);
+    launch_kernel(ssd_scalars_kernel, dim3((unsigned)scalars_blocks(sa, 256)), dim3(256), 0, ctx.stream,
+                  true, sa);
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
 int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
                      const float *dt_bias, const float *D, const float *h0, int B, int L, int H, int G,
                      int chunk, int sm_count, void *y, float *h_final, void *workspace,
@@ -685,11 +697,8 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     float2 *dl = (float2 *)workspace;
     char *seg_ws = (char *)workspace + ssd_scalars_bytes(B, L, H);
     if (!scalars_done) {
-        const ScalarsArgs sa = ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace);
-        ctx.begin(STAGE_SSD_SCALARS);
-        launch_kernel(ssd_scalars_kernel, dim3((unsigned)scalars_blocks(sa)), dim3(256), 0,
-                      ctx.stream, true, sa);
-        ctx.end();
+        const int rc = launch_ssd_scalars(ctx, ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace));
+        if (rc != SWIMBA_OK) return rc;
     }
     SsdParams p;
     p.dl = dl; p.D = D;

@@ -23,7 +23,6 @@ __host__ __device__ inline int64_t scalars_units(const ScalarsArgs &a)
     return a.dl ? (int64_t)(a.Lpad / SCALARS_TILE) * a.H * a.B : 0;
 }
 
-constexpr int SCALARS_UNITS_PER_BLOCK = 16;     // 256 threads: 8 warps x 2 units
 
 // NU consecutive (tile, head, sequence) units, worked by one warp without any block-level
 // synchronisation: lane l owns tokens 4l .. 4l+3 of a tile; the loads of all NU units are issued
@@ -77,17 +76,18 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
     }
 }
 
-// The block's share: SCALARS_UNITS_PER_BLOCK units starting at block * SCALARS_UNITS_PER_BLOCK
-// (256 threads).
+// The block's share: two units per warp, blocks of any whole number of warps.
 __device__ __forceinline__ void ssd_scalars_block(const ScalarsArgs &a, int64_t block)
 {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    ssd_scalars_warp<2>(a, block * SCALARS_UNITS_PER_BLOCK + warp * 2, lane);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+    ssd_scalars_warp<2>(a, (block * nwarp + warp) * 2, lane);
 }
 
-__host__ __device__ inline int64_t scalars_blocks(const ScalarsArgs &a)
+// Blocks of `threads` threads that cover all units.
+__host__ __device__ inline int64_t scalars_blocks(const ScalarsArgs &a, int threads)
 {
-    return (scalars_units(a) + SCALARS_UNITS_PER_BLOCK - 1) / SCALARS_UNITS_PER_BLOCK;
+    const int per_block = (threads >> 5) * 2;
+    return (scalars_units(a) + per_block - 1) / per_block;
 }
 
 }  // namespace swimba

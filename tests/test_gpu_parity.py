@@ -56,6 +56,11 @@ CASES = [
     cfg_of("bf16", L=257, B=1, H=6, G=2),                  # three heads per group: a pair and a single
     cfg_of("bf16", L=129, B=1, H=2),                       # one token past a tile boundary
     cfg_of("bf16", L=5000, B=1, H=2, h0_std=0.3),          # segmented sequence with an initial state
+    # enough 64-token tiles for the streaming router (three per SM): ragged last tile and feature
+    # block, 2 / 4 / 8 expert column tiles
+    cfg_of("bf16", L=14420, B=2, H=2, F=200, E=16, k=2),
+    cfg_of("bf16", L=28810, B=1, H=2, F=72, E=32, k=3),
+    cfg_of("bf16", L=28900, B=1, H=2, F=128, E=64, k=8),
 ]
 
 
