@@ -106,16 +106,17 @@ class ClockSampler:
                     samples=len(sm))
 
 
-def algorithmic_work(cfg: synth.LayerConfig):
+def algorithmic_work(cfg: synth.LayerConfig, sm_count: int = 148):
     """Per-launch algorithmic work of each kernel for B x L tokens: bytes the method must move or
     flops it must execute, not what a particular kernel happens to do."""
     T, F, S, E, k = cfg.tokens, cfg.F, cfg.S, cfg.E, cfg.k
     H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.Q
     es = 2 if cfg.dtype == "bf16" else 4
     w = {}
-    # with more than one expert the router launch also produces the SSD step sizes (dt in, (Delta,
-    # log-decay) pairs out) of the bf16 tile path
-    fused_scalars = T * H * 12 if (E > 1 and cfg.dtype == "bf16") else 0
+    # below three 64-token tiles per SM the router launch also produces the SSD step sizes (dt in,
+    # (Delta, log-decay) pairs out) of the bf16 tile path; above, they are a kernel of their own
+    fused = E > 1 and cfg.dtype == "bf16" and F % 128 == 0 and -(-T // 64) < 3 * sm_count
+    fused_scalars = T * H * 12 if fused else 0
     w["router_topk"] = dict(bound="hbm", work=T * F * es + E * F * es + T * k * 8 + fused_scalars)
     w["expert_gemm"] = dict(bound="tensor", work=2.0 * T * k * F * S)
     w["mix_slots"] = dict(bound="hbm", work=T * k * S * es + T * S * es)
@@ -265,8 +266,8 @@ def config_dict(cfg, **extra):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", default="small_lm", choices=[c for c in synth.CONFIG_ORDER if c != "decode"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-decode", action="store_true")
@@ -315,15 +316,16 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        step(i)
-    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
-    launches_per_step = sb.swimba_last_launch_count(h)
-
+    # the clock sampler is up before the warm-up, so that the warm-up steps run right in front of
+    # the timed ones (no idle gap in which the GPU could leave its boost state)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
+    for i in range(args.warmup):
+        step(i)
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    launches_per_step = sb.swimba_last_launch_count(h)
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -349,7 +351,7 @@ def main():
     sb.swimba_profile(h, False)
     clocks = sampler.stop() if rank == 0 else None
 
-    work = algorithmic_work(cfg)
+    work = algorithmic_work(cfg, torch.cuda.get_device_properties(local).multi_processor_count)
     tot = sum(sum(v) for v in per.values())
     kernels = []
     for name, v in per.items():
