@@ -9,7 +9,7 @@ namespace swimba {
 // When counts is given (zeroed beforehand) the (token, slot) pairs are also grouped by expert:
 // perm[e * cap + i], i < counts[e], lists the entries t*k + j routed to expert e.
 // zero_out (may be NULL): a [T, zero_bytes_per_token] buffer the kernel clears on the way (the
-// mixed streams, when the projection adds its slots in place).  scalars.dl != NULL: the call also
+// mixed streams, when the projection adds its slots in place).  scalars.l2 != NULL: the call also
 // produces the SSD step sizes and tile log-decays of the same forward (they depend on dt only and
 // run beside the router, inside its launch or as a kernel in front of it).
 int launch_router(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, int64_t T, int F,

@@ -739,7 +739,7 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
                            const ScalarsArgs &scalars)
 {
     const int warps = 8;
-    // The SSD step sizes of the same call (scalars.dl != NULL) depend on dt only and run beside the
+    // The SSD step sizes of the same call (scalars.l2 != NULL) depend on dt only and run beside the
     // router: as the leading blocks of the register-fed tensor-core kernel, else as a kernel of
     // their own in front of the router (the streaming router then starts while it runs).
     bool behind_scalars = false;
@@ -747,9 +747,9 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
         if (E > 1 && !router_stream_usable(u, Ttok, F, E, sm_count) && F % (32 * RM_KSPLIT) == 0 && E <= 64)
             return launch_router_mma(ctx, u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, sm_count,
                                      zero_out, zero_bytes_per_token, scalars);
-        behind_scalars = E > 1 && scalars.dl && router_stream_usable(u, Ttok, F, E, sm_count);
+        behind_scalars = E > 1 && scalars.l2 && router_stream_usable(u, Ttok, F, E, sm_count);
     }
-    if (scalars.dl) {
+    if (scalars.l2) {
         const int rc = launch_ssd_scalars(ctx, scalars);
         if (rc != SWIMBA_OK) return rc;
     }

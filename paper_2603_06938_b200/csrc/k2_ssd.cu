@@ -55,14 +55,16 @@ constexpr uint32_t SM_HEAD = 4 * SLAB;               // per head: X[2] XP HB YS
 constexpr uint32_t SM_HEAD_BYTES = 5 * SLAB;
 constexpr uint32_t SM_SMALL = SM_HEAD + NHD * SM_HEAD_BYTES;
 
-// TMEM columns: G, then per head M (bf16 A operand), Y, dH
-constexpr uint32_t TM_G = 0, TM_HEAD = 128, TM_HEAD_COLS = 192, TM_COLS = 512;
-constexpr uint32_t TM_M = 0, TM_Y = 64, TM_DH = 128;
+// TMEM columns: G, then Y, dH and M (bf16 A operand), each 64 columns per head with the two heads
+// side by side (one MMA of N = 128 can then write both heads' Y or dH)
+constexpr uint32_t TM_G = 0, TM_HEAD = 0, TM_HEAD_COLS = 64, TM_COLS = 512;
+constexpr uint32_t TM_Y = 128, TM_DH = 256, TM_M = 384;
 
 enum { MODE_FULL = 0, MODE_STATE_ONLY = 1 };
 
 struct SsdParams {
-    const float2 *dl;       // [B,H,Lpad] (Delta, log2-decay accumulated inside the 128-token tile)
+    const float *l2;        // [B,H,Lpad] log2-decay accumulated inside the 128-token tile
+    const TileScalars *rec; // [B,H,Lpad/128] per-tile weights and block ends
     const float *D;
     const float *h_in;      // initial states: [B,H,P,N] (nseg == 1) or [B,nseg,H,P,N]; may be null
     float *h_out;           // MODE_FULL: h_final [B,H,P,N] (last segment writes) or null
@@ -74,7 +76,7 @@ struct SsdParams {
 
 struct __align__(8) HeadBars {
     uint64_t x_full[2], x_free[2];
-    uint64_t yoff_full, m_full, yd_full, xp_full, dh_full, h_ready, y_free, y_staged;
+    uint64_t yoff_full, m_full, yd_full, xp_full, dh_full, h_ready, y_free, y_staged, sc_full;
 };
 struct __align__(8) SsdBars {
     uint64_t cb_full, cb_empty, g_full, g_free;
@@ -82,9 +84,7 @@ struct __align__(8) SsdBars {
 };
 
 struct __align__(16) SsdSmall {
-    float cs[NHD][ST];       // log2(Delta_s) - l_s          (diagonal blocks)
-    float cb[NHD][ST];       // Delta_s exp(L_{b(s)+1} - l_s) (blocks below the diagonal)
-    float ends[NHD][4];      // l at the end of each 32-row block of the tile
+    TileScalars sc[NHD];     // the current tile's weights and block ends, copied in by the TMA warp
     SsdBars bars;
     uint32_t tmem_slot;
     int abort_flag;
@@ -133,7 +133,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 
     if (tid == 0) {
         tc::mbar_init(&bars->cb_full, 1);
-        tc::mbar_init(&bars->cb_empty, nh);
+        tc::mbar_init(&bars->cb_empty, 1);
         tc::mbar_init(&bars->g_full, 1);
         tc::mbar_init(&bars->g_free, HEAD_THREADS * nh);
         for (int hd = 0; hd < NHD; ++hd) {
@@ -150,6 +150,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             tc::mbar_init(&hb->h_ready, HEAD_THREADS);
             tc::mbar_init(&hb->y_free, HEAD_THREADS);
             tc::mbar_init(&hb->y_staged, HEAD_THREADS);
+            tc::mbar_init(&hb->sc_full, 1);
         }
         *abort_flag = 0;
         tc::fence_mbar_init();
@@ -178,12 +179,19 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         // ------------------------------------------------------------------ TMA producer
         // (the whole warp runs the loop; one elected lane issues the copies)
         const bool leader = tc::elect_one();
+        const int ntile_seq = prm.Lpad / ST;
+        // record of tile t_begin / ST + j of head head0 + hd
+        auto scal_rec = [&](int hd, int j) {
+            return prm.rec + ((int64_t)b * H + head0 + hd) * ntile_seq + t_begin / ST + j;
+        };
         if (leader) {
-            for (int hd = 0; hd < nh; ++hd) {               // X of tile 0
+            for (int hd = 0; hd < nh; ++hd) {               // X and scalars of tile 0
                 HeadBars *hb = &bars->hd[hd];
                 tc::mbar_arrive_expect_tx(&hb->x_full[0], SLAB);
                 tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES, &tmap_x, &hb->x_full[0], 0,
                                 head0 + hd, t_begin, b);
+                tc::mbar_arrive_expect_tx(&hb->sc_full, (uint32_t)sizeof(TileScalars));
+                tc::bulk_load(&sm->sc[hd], scal_rec(hd, 0), (uint32_t)sizeof(TileScalars), &hb->sc_full);
             }
         }
         for (int j = 0; j < ntiles; ++j) {
@@ -209,6 +217,16 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                                         &hb->x_full[sx], 0, head0 + hd, t0 + ST, b);
                     }
                 }
+                // scalars of the next tile: the record buffer is single; its last readers are the
+                // mask (full pass) or the w.X scaling (state-only pass) of this tile
+                for (int hd = 0; hd < nh; ++hd) {
+                    HeadBars *hb = &bars->hd[hd];
+                    tc::mbar_wait(full ? &hb->m_full : &hb->xp_full, j & 1, abort_flag, d_status);
+                    if (leader) {
+                        tc::mbar_arrive_expect_tx(&hb->sc_full, (uint32_t)sizeof(TileScalars));
+                        tc::bulk_load(&sm->sc[hd], scal_rec(hd, jn), (uint32_t)sizeof(TileScalars), &hb->sc_full);
+                    }
+                }
             }
             __syncwarp();
         }
@@ -219,13 +237,17 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         const int hd = uwarp - WARP_MMA0;
         const bool leader = tc::elect_one();
         if (hd < nh) {
+            // The products against the shared Ctilde / Btilde tiles (MMA 1, 3, 4) are issued by the
+            // first issuer for both heads at once: with N = 128 the shared operand is read from
+            // shared memory once instead of once per head.  MMA 2 and the y store stay per head.
             constexpr uint32_t id_g = tc::idesc_bf16(128, 128, 0, 0);     // C (K-major) x B (K-major)
             constexpr uint32_t id_y = tc::idesc_bf16(128, 64, 0, 1);      // K-major / TMEM A, MN-major B
-            constexpr uint32_t id_h = tc::idesc_bf16(128, 64, 1, 1);      // MN-major A and B
+            const uint32_t id_yn = nh == 2 ? tc::idesc_bf16(128, 128, 0, 1) : id_y;
+            const uint32_t id_hn = nh == 2 ? tc::idesc_bf16(128, 128, 1, 1) : tc::idesc_bf16(128, 64, 1, 1);
             HeadBars *hb = &bars->hd[hd];
             const uint32_t c_addr = tc::smem_u32(smem + SM_CB), b_addr = c_addr + 2 * SLAB;
-            const uint32_t head_addr = tc::smem_u32(smem + SM_HEAD + hd * SM_HEAD_BYTES);
-            const uint32_t xp_addr = head_addr + 2 * SLAB, hb_addr = head_addr + 3 * SLAB;
+            const uint32_t head0_addr = tc::smem_u32(smem + SM_HEAD);
+            const uint32_t head_addr = head0_addr + hd * SM_HEAD_BYTES;
             const uint8_t *s_y = smem + SM_HEAD + hd * SM_HEAD_BYTES + 4 * SLAB;
             const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
             const uint32_t tm = tmem_u + TM_HEAD + hd * TM_HEAD_COLS;
@@ -233,8 +255,9 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             const uint64_t dC = tc::smem_desc_sw128(c_addr, 16, 1024);          // K-major
             const uint64_t dB = tc::smem_desc_sw128(b_addr, 16, 1024);          // K-major
             const uint64_t dBt = tc::smem_desc_sw128(b_addr, SLAB, 1024);       // MN-major
-            const uint64_t dH = tc::smem_desc_sw128(hb_addr, SLAB, 1024);       // MN-major
-            const uint64_t dXp = tc::smem_desc_sw128(xp_addr, SLAB, 1024);      // MN-major
+            // MN-major operands over both heads: the second head's 64 columns lie one head region on
+            const uint64_t dH = tc::smem_desc_sw128(head0_addr + 3 * SLAB, SM_HEAD_BYTES, 1024);
+            const uint64_t dXp = tc::smem_desc_sw128(head0_addr + 2 * SLAB, SM_HEAD_BYTES, 1024);
             const uint64_t dX0 = tc::smem_desc_sw128(head_addr, SLAB, 1024);    // MN-major
             // MMA 1 of tile jj: G = Ctilde Btilde^T (K = state index), shared by both heads
             auto issue_g = [&](int jj) {
@@ -255,36 +278,44 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             if (full && hd == 0) issue_g(0);
             for (int j = 0; j < ntiles; ++j) {
                 const int sx = j & 1;
-                tc::mbar_wait(&bars->cb_full, j & 1, abort_flag, d_status);
-                tc::tc_fence_after();
-                if (full) {
-                    // MMA 3: Y = Ctilde Hprev^T  (K = state index; B = bf16 state, rows = n)
-                    tc::mbar_wait(&hb->h_ready, j & 1, abort_flag, d_status);
-                    if (j > 0) tc::mbar_wait(&hb->y_free, (j - 1) & 1, abort_flag, d_status);
+                if (hd == 0) {
+                    tc::mbar_wait(&bars->cb_full, j & 1, abort_flag, d_status);
+                    tc::tc_fence_after();
+                    if (full) {
+                        // MMA 3: Y = Ctilde Hprev^T  (K = state index; B = bf16 states, rows = n)
+                        for (int q = 0; q < nh; ++q) {
+                            tc::mbar_wait(&bars->hd[q].h_ready, j & 1, abort_flag, d_status);
+                            if (j > 0) tc::mbar_wait(&bars->hd[q].y_free, (j - 1) & 1, abort_flag, d_status);
+                        }
+                        tc::tc_fence_after();
+                        if (leader) {
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
+                                tc::mma_ss(tmem_u + TM_Y, tc::smem_desc_advance(dC, off),
+                                           tc::smem_desc_advance(dH, kk * 2048), id_yn, kk > 0);
+                            }
+                            for (int q = 0; q < nh; ++q) tc::mma_commit(&bars->hd[q].yoff_full);
+                        }
+                        __syncwarp();
+                        // MMA 1 of this tile goes behind MMA 3 in the tensor pipe: the product with
+                        // the carried state is needed first (it is scaled before the mask is built)
+                        if (j > 0) issue_g(j);
+                    }
+                    // MMA 4: dH^T[n,p] = sum_s Btilde[s,n] (w_s x_s[p])   (K = token)
+                    for (int q = 0; q < nh; ++q)
+                        tc::mbar_wait(&bars->hd[q].xp_full, j & 1, abort_flag, d_status);
                     tc::tc_fence_after();
                     if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk) {
-                            const uint32_t off = (kk >> 2) * SLAB + (kk & 3) * 32;
-                            tc::mma_ss(tm + TM_Y, tc::smem_desc_advance(dC, off),
-                                       tc::smem_desc_advance(dH, kk * 2048), id_y, kk > 0);
-                        }
-                        tc::mma_commit(&hb->yoff_full);
+                        for (int kk = 0; kk < 8; ++kk)
+                            tc::mma_ss(tmem_u + TM_DH, tc::smem_desc_advance(dBt, kk * 2048),
+                                       tc::smem_desc_advance(dXp, kk * 2048), id_hn, kk > 0);
+                        for (int q = 0; q < nh; ++q) tc::mma_commit(&bars->hd[q].dh_full);
+                        tc::mma_commit(&bars->cb_empty);     // C and B tiles are no longer needed
                     }
                     __syncwarp();
                 }
-                // MMA 4: dH^T[n,p] = sum_s Btilde[s,n] (w_s x_s[p])   (K = token)
-                tc::mbar_wait(&hb->xp_full, j & 1, abort_flag, d_status);
-                tc::tc_fence_after();
-                if (leader) {
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)
-                        tc::mma_ss(tm + TM_DH, tc::smem_desc_advance(dBt, kk * 2048),
-                                   tc::smem_desc_advance(dXp, kk * 2048), id_h, kk > 0);
-                    tc::mma_commit(&hb->dh_full);
-                    tc::mma_commit(&bars->cb_empty);     // C and B tiles are no longer needed
-                }
-                __syncwarp();
                 if (full) {
                     // MMA 2: Y += M X  (A = masked tile in TMEM, 8 columns per 16 tokens of K)
                     tc::mbar_wait(&hb->m_full, j & 1, abort_flag, d_status);
@@ -299,10 +330,12 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                         tc::mma_commit(&hb->yd_full);
                     }
                 }
+                // (state-only pass: the second issuer has no product of its own; it follows the
+                // tile loop at the pace of its head's w.X scaling, whose end frees the X slot)
+                if (!full && hd > 0) tc::mbar_wait(&hb->xp_full, j & 1, abort_flag, d_status);
                 if (leader) tc::mma_commit(&hb->x_free[sx]);
                 __syncwarp();
                 if (full) {
-                    if (hd == 0 && j + 1 < ntiles) issue_g(j + 1);
                     // the staged y tile goes out as one TMA store (rows past the end of the
                     // sequence are clipped by the tensor map)
                     tc::mbar_wait(&hb->y_staged, j & 1, abort_flag, d_status);
@@ -324,8 +357,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         HeadBars *hb = &bars->hd[hd];
         uint8_t *s_head = smem + SM_HEAD + hd * SM_HEAD_BYTES;
         uint8_t *s_xp = s_head + 2 * SLAB, *s_hb = s_head + 3 * SLAB, *s_y = s_head + 4 * SLAB;
-        float *s_cs = sm->cs[hd], *s_cb = sm->cb[hd], *s_ends = sm->ends[hd];
-        const int bar_id = 1 + hd;
+        const uint32_t *s_wp = sm->sc[hd].wp;
+        const float *s_cb = sm->sc[hd].cb, *s_ends = sm->sc[hd].ends;
         const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
         const uint32_t tm = tmem + TM_HEAD + hd * TM_HEAD_COLS + lane_base;
         const float Dh = prm.D ? prm.D[h] : 0.f;
@@ -363,37 +396,27 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             }
         }
         float seg_l2 = 0.f;      // log2 of the product of a_t over the tiles done so far
-        const float2 *dlp = prm.dl + ((int64_t)b * H + h) * prm.Lpad + t_begin;
-        float2 dl_next = dlp[i];
+        const float *l2p = prm.l2 + ((int64_t)b * H + h) * prm.Lpad + t_begin;
+        float l2_next = l2p[i];
 
         for (int j = 0; j < ntiles; ++j) {
             const int sx = j & 1;
             const uint8_t *s_x = s_head + sx * SLAB;
-            // ---- per-token scalars: Delta, cumulative log2 decay inside the tile
-            const float delta = dl_next.x, l2 = dl_next.y;
-            if (j + 1 < ntiles) dl_next = dlp[(j + 1) * ST + i];
-            const float Lend = __shfl_sync(0xffffffffu, l2, 31);       // l at the end of my block
-            if (hf == 0) {
-                // safe to overwrite: every reader of the previous tile's values had finished its
-                // mask before MMA 2 of that tile could start, and this thread has seen it end
-                // (in the state-only pass the readers are ordered by the barrier below instead)
-                if (lane == 31) s_ends[wq] = l2;
-                if (full) {
-                    s_cs[i] = (delta > 0.f ? tc::lg2_approx(delta) : -INFINITY) - l2;
-                    s_cb[i] = delta * tc::ex2_approx(Lend - l2);
-                }
-            }
-            tc::named_bar_sync(bar_id, HEAD_THREADS);        // ends / cs / cb of this tile are visible
+            // ---- per-token scalars: this row's cumulative log2 decay inside the tile (prefetched);
+            // the weights of all rows and the block ends arrive in shared memory
+            const float l2 = l2_next;
+            if (j + 1 < ntiles) l2_next = l2p[(j + 1) * ST + i];
+            tc::mbar_wait(&hb->sc_full, j & 1, abort_flag, d_status);
             const float4 ends = *reinterpret_cast<const float4 *>(s_ends);
             const float L1 = ends.x, L2 = ends.y, L3 = ends.z, l2_last = ends.w;
             const float Lw = wq == 0 ? 0.f : (wq == 1 ? L1 : (wq == 2 ? L2 : L3));    // l before my block
-            const float w_s = delta * tc::ex2_approx(l2_last - l2);
+            const float Lend = wq == 0 ? L1 : (wq == 1 ? L2 : (wq == 2 ? L3 : l2_last));  // l at its end
 
             // ---- w . X  (rows of the X slab -> rows of the X' slab, this thread's half of the
             // head dim).  The decay mask below costs row block wq about wq + 1 units of work, so in
             // the full pass the 16 (row block, 16-byte chunk) units of a lane are dealt 6 / 5 / 3 / 2
-            // to row blocks 0 .. 3 instead of 4 each; a foreign row's weight comes from cs:
-            // w_r = Delta_r 2^(l_last - l_r) = 2^(cs_r + l_last).
+            // to row blocks 0 .. 3 instead of 4 each; a foreign row's weight is read from shared
+            // memory.
             tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
             {
                 const int ubeg = full ? (wq == 0 ? 0 : (wq == 1 ? 6 : (wq == 2 ? 11 : 14))) : 4 * wq;
@@ -401,12 +424,10 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 #pragma unroll 1
                 for (int un = ubeg; un < uend; ++un) {
                     const int r = (un >> 2) * 32 + lane;
-                    const float w_r = full ? tc::ex2_approx(s_cs[r] + l2_last) : w_s;
-                    // w_r as a two-term bf16 sum; x stays packed: round(w_hi x + round(w_lo x)) is
-                    // w_r x rounded once, up to a term of relative size 2^-17
-                    const __nv_bfloat16 w_hi = __float2bfloat16_rn(w_r);
-                    const __nv_bfloat162 w_hi2 = __bfloat162bfloat162(w_hi);
-                    const __nv_bfloat162 w_lo2 = __float2bfloat162_rn(w_r - __bfloat162float(w_hi));
+                    const uint32_t wp = s_wp[r];
+                    const uint32_t hi_u = __byte_perm(wp, 0, 0x1010), lo_u = __byte_perm(wp, 0, 0x3232);
+                    const __nv_bfloat162 w_hi2 = *reinterpret_cast<const __nv_bfloat162 *>(&hi_u);
+                    const __nv_bfloat162 w_lo2 = *reinterpret_cast<const __nv_bfloat162 *>(&lo_u);
                     const uint32_t off = tc::sw128_offset(r, 4 * hf + (un & 3));
                     const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
                     const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
@@ -452,14 +473,32 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                         tc::tmem_ld16(g_addr + c * 32, cur);
                         tc::tmem_ld_wait();
                         if (c == wq) {
+                            // diagonal block: Delta_j 2^(l_i - l_j) = cb_j 2^(l_i - l_blockend).  The
+                            // second factor is >= 1; when the whole block decays by less than
+                            // 2^-96 it cannot overflow and is applied as a product, else the
+                            // exponent is formed per entry (always <= 0 where j <= i).
+                            const float up = l2 - Lend;
+                            if (Lw - Lend < 96.f) {
+                                const float rf = tc::ex2_approx(up);
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const float2 cs = *reinterpret_cast<const float2 *>(&s_cs[c * 32 + 16 * hf + 2 * q]);
-                                float m0 = __uint_as_float(cur[2 * q]) * tc::ex2_approx(l2 + cs.x);
-                                float m1 = __uint_as_float(cur[2 * q + 1]) * tc::ex2_approx(l2 + cs.y);
-                                if (16 * hf + 2 * q > lane) m0 = 0.f;
-                                if (16 * hf + 2 * q + 1 > lane) m1 = 0.f;
-                                pk[q] = tc::pack_bf16x2(m0, m1);
+                                for (int q = 0; q < 8; ++q) {
+                                    const float2 cb = *reinterpret_cast<const float2 *>(&s_cb[c * 32 + 16 * hf + 2 * q]);
+                                    float m0 = __uint_as_float(cur[2 * q]) * cb.x * rf;
+                                    float m1 = __uint_as_float(cur[2 * q + 1]) * cb.y * rf;
+                                    if (16 * hf + 2 * q > lane) m0 = 0.f;
+                                    if (16 * hf + 2 * q + 1 > lane) m1 = 0.f;
+                                    pk[q] = tc::pack_bf16x2(m0, m1);
+                                }
+                            } else {
+#pragma unroll
+                                for (int q = 0; q < 8; ++q) {
+                                    const float2 cb = *reinterpret_cast<const float2 *>(&s_cb[c * 32 + 16 * hf + 2 * q]);
+                                    float m0 = __uint_as_float(cur[2 * q]) * tc::ex2_approx(up + tc::lg2_approx(cb.x));
+                                    float m1 = __uint_as_float(cur[2 * q + 1]) * tc::ex2_approx(up + tc::lg2_approx(cb.y));
+                                    if (16 * hf + 2 * q > lane) m0 = 0.f;
+                                    if (16 * hf + 2 * q + 1 > lane) m1 = 0.f;
+                                    pk[q] = tc::pack_bf16x2(m0, m1);
+                                }
                             }
                         } else {
                             // l at the end of column block c, relative to the start of my block
@@ -478,6 +517,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 tc::tmem_st_wait();
                 tc::tc_fence_before();
                 tc::mbar_arrive(&bars->g_free);
+                // (the scalars record read above is refilled by a bulk copy once m_full completes)
+                tc::fence_proxy_async_smem();
                 tc::mbar_arrive(&hb->m_full);
             }
 
@@ -634,7 +675,9 @@ int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count)
 static size_t ssd_scalars_bytes(int B, int L, int H)
 {
     const size_t Lpad = (size_t)ceil_div(L, ST) * ST;
-    return ((size_t)B * H * Lpad * sizeof(float2) + 255) / 256 * 256;
+    const size_t l2_bytes = ((size_t)B * H * Lpad * sizeof(float) + 255) / 256 * 256;
+    const size_t rec_bytes = ((size_t)B * H * (Lpad / ST) * sizeof(TileScalars) + 255) / 256 * 256;
+    return l2_bytes + rec_bytes;
 }
 
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count)
@@ -651,7 +694,9 @@ ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bi
                              void *workspace)
 {
     ScalarsArgs a;
-    a.dt = dt; a.A = A; a.dt_bias = dt_bias; a.dl = (float2 *)workspace;
+    a.dt = dt; a.A = A; a.dt_bias = dt_bias; a.l2 = (float *)workspace;
+    a.rec = (TileScalars *)((char *)workspace +
+                            ((size_t)B * H * (ceil_div(L, ST) * ST) * sizeof(float) + 255) / 256 * 256);
     a.L = L; a.Lpad = ceil_div(L, ST) * ST; a.H = H; a.B = B;
     return a;
 }
@@ -694,14 +739,18 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
     const int nseg = ceil_div(L, seg_len);
     const int Lpad = ceil_div(L, ST) * ST;
-    float2 *dl = (float2 *)workspace;
     char *seg_ws = (char *)workspace + ssd_scalars_bytes(B, L, H);
     if (!scalars_done) {
         const int rc = launch_ssd_scalars(ctx, ssd_scalars_args(dt, A, dt_bias, B, L, H, workspace));
         if (rc != SWIMBA_OK) return rc;
     }
     SsdParams p;
-    p.dl = dl; p.D = D;
+    {
+        const ScalarsArgs sa = ssd_scalars_args(nullptr, nullptr, nullptr, B, L, H, workspace);
+        p.l2 = sa.l2;
+        p.rec = sa.rec;
+    }
+    p.D = D;
     p.L = L; p.Lpad = Lpad; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
     p.d_status = ctx.d_status;
     dim3 grid((unsigned)nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);

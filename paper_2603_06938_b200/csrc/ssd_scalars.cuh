@@ -1,8 +1,15 @@
 // Step sizes and tile log-decays of the SSD evaluation (Background, "Mamba-2 and SSD"; the
-// transition is shared by all experts: shared-A equation):
-//   Delta_t = softplus(dt_t + dt_bias_h),
-//   dl[(b*H + h)*Lpad + t] = (Delta_t, sum_{r <= t, r in t's 128-token tile} Delta_r A_h log2 e);
-// positions past L carry Delta = 0, so the last entry of a tile is always the tile's total.
+// transition is shared by all experts: shared-A equation).  Per token t of head h, with
+// Delta_t = softplus(dt_t + dt_bias_h) and l_t = sum_{r <= t, r in t's 128-token tile} Delta_r A_h log2 e,
+// two arrays are produced:
+//   l2[(b*H + h)*Lpad + t] = l_t
+//   rec[((b*H + h)*ntile + tile)] = one record per 128-token tile, copied to shared memory as a block:
+//       wp[128]  W(Delta_t 2^(l_last - l_t))      weight of token t in the tile's end state
+//       cb[128]  Delta_t 2^(l_blockend - l_t)     weight of token t at the end of its 32-token block
+//       ends[4]  l at the end of each 32-token block (ends[3] = l_last)
+// Every exponent is <= 0.  W(w) is w as a two-term bf16 sum packed in one word (high part in the low
+// half, remainder in the high half): round(w_hi x + round(w_lo x)) is w x rounded once for a bf16 x,
+// up to a term of relative size 2^-17.  Positions past L carry Delta = 0.
 // The work depends on dt only, so it runs either as a kernel of its own or as extra blocks of
 // the router kernel.
 #pragma once
@@ -12,15 +19,23 @@ namespace swimba {
 
 constexpr int SCALARS_TILE = 128;
 
+struct TileScalars {            // (the shared-memory image as well)
+    uint32_t wp[SCALARS_TILE];
+    float cb[SCALARS_TILE];
+    float ends[4];
+};
+static_assert(sizeof(TileScalars) % 16 == 0, "tile records are moved by 16-byte bulk copies");
+
 struct ScalarsArgs {
     const float *dt, *A, *dt_bias;
-    float2 *dl;           // null: nothing to do
+    float *l2;            // null: nothing to do
+    TileScalars *rec;
     int L, Lpad, H, B;
 };
 
 __host__ __device__ inline int64_t scalars_units(const ScalarsArgs &a)
 {
-    return a.dl ? (int64_t)(a.Lpad / SCALARS_TILE) * a.H * a.B : 0;
+    return a.l2 ? (int64_t)(a.Lpad / SCALARS_TILE) * a.H * a.B : 0;
 }
 
 
@@ -46,7 +61,7 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
         const int t = tile * SCALARS_TILE + lane * 4;
         hh[q] = h;
         tt[q] = t;
-        out[q] = act ? (b * a.H + h) * a.Lpad + t : -1;
+        out[q] = act ? (b * a.H + h) * ntile + tile : -1;        // record index
 #pragma unroll
         for (int i = 0; i < 4; ++i)
             raw[q][i] = (act && a.dt && t + i < a.L) ? a.dt[(b * a.L + t + i) * a.H + h] : 0.f;
@@ -70,9 +85,24 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
             if (lane >= o) incl += nb;
         }
         const float excl = incl - run;
-        float4 *dst = reinterpret_cast<float4 *>(a.dl + out[q]);
-        dst[0] = make_float4(d[0], excl + p[0], d[1], excl + p[1]);
-        dst[1] = make_float4(d[2], excl + p[2], d[3], excl + p[3]);
+        const float l_last = __shfl_sync(0xffffffffu, incl, 31);
+        const float l_blk = __shfl_sync(0xffffffffu, incl, lane | 7);   // 8 lanes = one 32-token block
+        float lv[4], cb[4];
+        uint32_t wp[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            lv[i] = excl + p[i];
+            const float w = d[i] * exp2f(l_last - lv[i]);
+            const __nv_bfloat16 w_hi = __float2bfloat16_rn(w);
+            wp[i] = (uint32_t)__bfloat16_as_ushort(w_hi) |
+                    ((uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(w - __bfloat162float(w_hi))) << 16);
+            cb[i] = d[i] * exp2f(l_blk - lv[i]);
+        }
+        TileScalars *rec = a.rec + out[q];
+        reinterpret_cast<float4 *>(a.l2 + out[q] * SCALARS_TILE)[lane] = make_float4(lv[0], lv[1], lv[2], lv[3]);
+        reinterpret_cast<uint4 *>(rec->wp)[lane] = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+        reinterpret_cast<float4 *>(rec->cb)[lane] = make_float4(cb[0], cb[1], cb[2], cb[3]);
+        if ((lane & 7) == 7) rec->ends[lane >> 3] = incl;
     }
 }
 

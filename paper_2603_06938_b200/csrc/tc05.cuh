@@ -115,6 +115,16 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, const void *s
         "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// Plain bulk copy global -> shared of `bytes` (a multiple of 16, both addresses 16-byte aligned);
+// completion is counted in bytes on the mbarrier.
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_global, uint32_t bytes,
+                                          uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(src_global), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
 // Plain bulk copy shared -> global of `bytes` (a multiple of 16, both addresses 16-byte aligned),
 // tracked by the issuing thread's bulk async-group.
 __device__ __forceinline__ void bulk_store(void *dst_global, const void *src_smem, uint32_t bytes) {
