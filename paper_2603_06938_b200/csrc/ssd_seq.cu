@@ -134,7 +134,7 @@ int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *
 // HBM stream.  One warp owns ROWS consecutive channels p of one (b,h); a row is N floats read
 // as float4 per lane, all ROWS loads are issued before any use.
 // ------------------------------------------------------------------------------------------
-constexpr int DEC_ROWS = 4;
+constexpr int DEC_ROWS = 8;
 
 __device__ __forceinline__ float4 load_bc4(const float *p, int v)
 {
