@@ -71,6 +71,8 @@ struct SsdParams {
                             // MODE_STATE_ONLY: local end states [B,nseg,H,P,N]
     float *seg_decay;       // MODE_STATE_ONLY: [B,nseg,H] product of a_t over the segment
     int L, Lpad, H, G, nseg, seg_len, mode;
+    int split_tiles;        // > 0 (MODE_FULL, nseg == 1): every (sequence, head pair) is worked by two
+                            // CTAs, see ssd_tiles_kernel
     int *d_status;
 };
 
@@ -105,6 +107,7 @@ ssd_scalars_kernel(const ScalarsArgs args)
     ssd_scalars_block(args, blockIdx.x);
 }
 
+template <bool SPLIT>
 __global__ void __launch_bounds__(SSD_THREADS, 1)
 ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
                  const __grid_constant__ CUtensorMap tmap_y, const SsdParams prm)
@@ -120,16 +123,26 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     }
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int seg = blockIdx.x, b = blockIdx.z;
+    // Split launch (grid = [B, head pairs, 2]; used when one CTA per (sequence, head pair) would
+    // leave a third of the SMs idle): the CTAs of the first z-plane, which start first, walk the whole
+    // sequence but evaluate the first split_tiles tiles for their end state only (about half the
+    // cost of a full tile) and produce y from there on; the CTAs of the second plane produce y of
+    // those first tiles.  No CTA waits for another.
+    constexpr bool split = SPLIT;                                // (prm.split_tiles > 0)
+    const bool head_part = split && blockIdx.z == 1;             // y of the leading tiles only
+    const int seg = split ? 0 : blockIdx.x, b = split ? blockIdx.x : blockIdx.z;
     const int L = prm.L, H = prm.H;
     const int HG = H / prm.G, ppg = pairs_per_group(H, prm.G);
     const int g = blockIdx.y / ppg, pr = blockIdx.y % ppg;
     const int head0 = g * HG + pr * NHD;
     const int nh = min(NHD, HG - pr * NHD);          // heads this CTA really has
     const int t_begin = seg * prm.seg_len;
-    const int t_end = min(L, t_begin + prm.seg_len);
+    const int t_end = head_part ? min(L, prm.split_tiles * ST) : min(L, t_begin + prm.seg_len);
     const int ntiles = (t_end - t_begin + ST - 1) / ST;
-    const bool full = prm.mode == MODE_FULL;
+    const bool kfull = prm.mode == MODE_FULL;
+    // leading tiles that only carry the state forward (tile j is a full tile iff kfull && j >= n_pre;
+    // barriers that only full tiles use count their phases in full tiles, jf = j - n_pre)
+    const int n_pre = split ? (head_part ? 0 : min(prm.split_tiles, ntiles)) : 0;
 
     if (tid == 0) {
         tc::mbar_init(&bars->cb_full, 1);
@@ -196,6 +209,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         }
         for (int j = 0; j < ntiles; ++j) {
             const int t0 = t_begin + j * ST;
+            const bool full = SPLIT ? (kfull && j >= n_pre) : kfull;
             tc::mbar_wait(&bars->cb_empty, (j & 1) ^ 1, abort_flag, d_status);
             if (leader) {
                 tc::mbar_arrive_expect_tx(&bars->cb_full, full ? 4 * SLAB : 2 * SLAB);
@@ -221,7 +235,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 // mask (full pass) or the w.X scaling (state-only pass) of this tile
                 for (int hd = 0; hd < nh; ++hd) {
                     HeadBars *hb = &bars->hd[hd];
-                    tc::mbar_wait(full ? &hb->m_full : &hb->xp_full, j & 1, abort_flag, d_status);
+                    if (full) tc::mbar_wait(&hb->m_full, (SPLIT ? j - n_pre : j) & 1, abort_flag, d_status);
+                    else tc::mbar_wait(&hb->xp_full, j & 1, abort_flag, d_status);
                     if (leader) {
                         tc::mbar_arrive_expect_tx(&hb->sc_full, (uint32_t)sizeof(TileScalars));
                         tc::bulk_load(&sm->sc[hd], scal_rec(hd, jn), (uint32_t)sizeof(TileScalars), &hb->sc_full);
@@ -262,7 +277,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             // MMA 1 of tile jj: G = Ctilde Btilde^T (K = state index), shared by both heads
             auto issue_g = [&](int jj) {
                 tc::mbar_wait(&bars->cb_full, jj & 1, abort_flag, d_status);
-                if (jj > 0) tc::mbar_wait(&bars->g_free, (jj - 1) & 1, abort_flag, d_status);
+                const int jjf = SPLIT ? jj - n_pre : jj;
+                if (jjf > 0) tc::mbar_wait(&bars->g_free, (jjf - 1) & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 if (leader) {
 #pragma unroll
@@ -275,17 +291,18 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 __syncwarp();
             };
-            if (full && hd == 0) issue_g(0);
             for (int j = 0; j < ntiles; ++j) {
                 const int sx = j & 1;
+                const bool full = SPLIT ? (kfull && j >= n_pre) : kfull;
+                const int jf = SPLIT ? j - n_pre : j;
                 if (hd == 0) {
                     tc::mbar_wait(&bars->cb_full, j & 1, abort_flag, d_status);
                     tc::tc_fence_after();
                     if (full) {
                         // MMA 3: Y = Ctilde Hprev^T  (K = state index; B = bf16 states, rows = n)
                         for (int q = 0; q < nh; ++q) {
-                            tc::mbar_wait(&bars->hd[q].h_ready, j & 1, abort_flag, d_status);
-                            if (j > 0) tc::mbar_wait(&bars->hd[q].y_free, (j - 1) & 1, abort_flag, d_status);
+                            tc::mbar_wait(&bars->hd[q].h_ready, jf & 1, abort_flag, d_status);
+                            if (jf > 0) tc::mbar_wait(&bars->hd[q].y_free, (jf - 1) & 1, abort_flag, d_status);
                         }
                         tc::tc_fence_after();
                         if (leader) {
@@ -300,7 +317,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                         __syncwarp();
                         // MMA 1 of this tile goes behind MMA 3 in the tensor pipe: the product with
                         // the carried state is needed first (it is scaled before the mask is built)
-                        if (j > 0) issue_g(j);
+                        issue_g(j);
                     }
                     // MMA 4: dH^T[n,p] = sum_s Btilde[s,n] (w_s x_s[p])   (K = token)
                     for (int q = 0; q < nh; ++q)
@@ -318,7 +335,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 if (full) {
                     // MMA 2: Y += M X  (A = masked tile in TMEM, 8 columns per 16 tokens of K)
-                    tc::mbar_wait(&hb->m_full, j & 1, abort_flag, d_status);
+                    tc::mbar_wait(&hb->m_full, jf & 1, abort_flag, d_status);
                     tc::tc_fence_after();
                     const uint64_t dX = tc::smem_desc_advance(dX0, sx * SLAB);
                     if (leader) {
@@ -338,7 +355,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 if (full) {
                     // the staged y tile goes out as one TMA store (rows past the end of the
                     // sequence are clipped by the tensor map)
-                    tc::mbar_wait(&hb->y_staged, j & 1, abort_flag, d_status);
+                    tc::mbar_wait(&hb->y_staged, jf & 1, abort_flag, d_status);
                     if (leader) {
                         tc::tma_store_4d(&tmap_y, s_y, 0, head0 + hd, t_begin + j * ST, b);
                         tc::bulk_commit_group();
@@ -346,7 +363,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     __syncwarp();
                 }
             }
-            if (full && leader) tc::bulk_wait_read_all();
+            if (kfull && leader) tc::bulk_wait_read_all();
         }
     } else if ((uwarp >> 3) < nh) {
         // ------------------------------------------------------------------ compute warps
@@ -366,7 +383,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         float Hst[32];
         {
             const float *h_in = prm.h_in;
-            if (h_in && full) {
+            if (h_in && kfull) {
                 const int64_t base = prm.nseg > 1
                     ? ((((int64_t)b * prm.nseg + seg) * H + h) * SP) * SN
                     : (((int64_t)b * H + h) * SP) * SN;
@@ -376,7 +393,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 #pragma unroll
                 for (int q = 0; q < 32; ++q) Hst[q] = 0.f;
             }
-            if (full) {
+            if (kfull && n_pre == 0) {
+                // bf16 copy of the state the first tile starts from
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     uint4 v = make_uint4(tc::pack_bf16x2(Hst[8 * ch + 0], Hst[8 * ch + 1]),
@@ -387,6 +405,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 tc::fence_proxy_async_smem();
                 tc::mbar_arrive(&hb->h_ready);
+            }
+            if (kfull) {
                 // blocks of M above the diagonal stay zero for the whole kernel
                 uint32_t zero[8];
 #pragma unroll
@@ -401,6 +421,9 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 
         for (int j = 0; j < ntiles; ++j) {
             const int sx = j & 1;
+            const bool full = SPLIT ? (kfull && j >= n_pre) : kfull;
+            const bool hb_next = SPLIT ? (kfull && j + 1 >= n_pre) : kfull;   // the next tile reads the bf16 state copy
+            const int jf = SPLIT ? j - n_pre : j;
             const uint8_t *s_x = s_head + sx * SLAB;
             // ---- per-token scalars: this row's cumulative log2 decay inside the tile (prefetched);
             // the weights of all rows and the block ends arrive in shared memory
@@ -446,7 +469,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 
             if (full) {
                 // ---- Y = exp(l_i) * (Ctilde Hprev^T), in place
-                tc::mbar_wait(&hb->yoff_full, j & 1, abort_flag, d_status);
+                tc::mbar_wait(&hb->yoff_full, jf & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 {
                     const float e_i = tc::ex2_approx(l2);
@@ -462,7 +485,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 }
                 // ---- decay mask: G (fp32, TMEM) -> M (bf16, TMEM); this thread owns row i and
                 // columns 16 hf .. 16 hf + 15 of every 32-column block
-                tc::mbar_wait(&bars->g_full, j & 1, abort_flag, d_status);
+                tc::mbar_wait(&bars->g_full, jf & 1, abort_flag, d_status);
                 tc::tc_fence_after();
                 const float r_i = tc::ex2_approx(l2 - Lw);
                 const uint32_t g_addr = tmem + lane_base + TM_G + 16 * hf;
@@ -535,7 +558,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 #pragma unroll
                 for (int q = 0; q < 16; ++q)
                     Hst[16 * hh + q] = fmaf(dec, Hst[16 * hh + q], __uint_as_float(dh[q]));
-                if (full) {
+                if (hb_next) {
 #pragma unroll
                     for (int c2 = 0; c2 < 2; ++c2) {
                         const int ch = 2 * hh + c2;
@@ -547,13 +570,14 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     }
                 }
             }
-            if (full) {
+            if (hb_next) {
                 tc::fence_proxy_async_smem();
                 tc::tc_fence_before();
                 tc::mbar_arrive(&hb->h_ready);
-
+            }
+            if (full) {
                 // ---- epilogue: y_i = Y_i + D x_i, staged in shared memory for the TMA store
-                tc::mbar_wait(&hb->yd_full, j & 1, abort_flag, d_status);
+                tc::mbar_wait(&hb->yd_full, jf & 1, abort_flag, d_status);
                 tc::tc_fence_after();
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
@@ -588,8 +612,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         }
 
         // ---- final state of the segment
-        if (full) {
-            if (prm.h_out && seg == prm.nseg - 1) {
+        if (kfull) {
+            if (prm.h_out && seg == prm.nseg - 1 && !head_part) {
                 float *dst = prm.h_out + (((int64_t)b * H + h) * SP) * SN;
 #pragma unroll
                 for (int q = 0; q < 32; ++q) dst[(int64_t)(p0 + q) * SN + i] = Hst[q];
@@ -701,6 +725,27 @@ ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bi
     return a;
 }
 
+// Split of a one-segment launch (see ssd_tiles_kernel): 0 when one CTA per (sequence, head pair)
+// already fills the GPU (or the segmented path applies), else the number of leading tiles a.  The
+// CTAs that walk the whole sequence (started first, one per SM) cost (n - a) full tiles plus a
+// state-only tiles at about 0.47 of a full one; the CTAs that produce y of the leading tiles run
+// on the SMs left over, in ceil(ctas / spare) rounds of a tiles.  a minimises the later of the two.
+static int ssd_split_tiles(int B, int L, int H, int G, int sm_count)
+{
+    const int64_t ctas = (int64_t)B * G * pairs_per_group(H, G);
+    const int n = ceil_div(L, ST);
+    if (2 * ctas <= sm_count || ctas >= sm_count || n < 4) return 0;
+    const int64_t spare = sm_count - ctas, rounds = ceil_div64(ctas, spare);
+    float best = (float)n;
+    int best_a = 0;
+    for (int a = 1; a < n; ++a) {
+        const float whole = (float)n - 0.53f * a, lead = (float)(rounds * a);
+        const float m = whole > lead ? whole : lead;
+        if (m < best) { best = m; best_a = a; }
+    }
+    return best < 0.93f * n ? best_a : 0;
+}
+
 int launch_ssd_scalars(LaunchCtx &ctx, const ScalarsArgs &sa)
 {
     if (scalars_units(sa) <= 0) return SWIMBA_OK;
@@ -733,7 +778,8 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         if (!encode_tmap_bf16(&tm_y, y, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
     }
     const size_t smem = ssd_smem_bytes();
-    if (cudaFuncSetAttribute(ssd_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(ssd_tiles_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(ssd_tiles_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return SWIMBA_ERR_CUDA;
 
     const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
@@ -754,17 +800,23 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     p.L = L; p.Lpad = Lpad; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
     p.d_status = ctx.d_status;
     dim3 grid((unsigned)nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
+    p.split_tiles = 0;
     if (nseg == 1) {
         p.h_in = h0; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
+        p.split_tiles = ssd_split_tiles(B, L, H, G, sm_count);
+        if (p.split_tiles > 0) grid = dim3((unsigned)B, (unsigned)(G * pairs_per_group(H, G)), 2u);
         ctx.begin(STAGE_SSD_TILES);
-        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        if (p.split_tiles > 0)
+            launch_kernel(ssd_tiles_kernel<true>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        else
+            launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     } else {
         float *states = (float *)seg_ws;
         float *decay = states + (size_t)B * nseg * H * SP * SN;
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
         ctx.begin(STAGE_SSD_TILES);
-        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
@@ -773,7 +825,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         ctx.end();
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
-        launch_kernel(ssd_tiles_kernel, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;

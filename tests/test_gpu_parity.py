@@ -61,6 +61,10 @@ CASES = [
     cfg_of("bf16", L=14420, B=2, H=2, F=200, E=16, k=2),
     cfg_of("bf16", L=28810, B=1, H=2, F=72, E=32, k=3),
     cfg_of("bf16", L=28900, B=1, H=2, F=128, E=64, k=8),
+    # between half an SM count and one SM count of (sequence, head pair) CTAs: every pair is worked by
+    # two CTAs (leading tiles / whole sequence with a state-only lead); even and odd head counts
+    cfg_of("bf16", L=700, B=40, H=4, h0_std=0.3),
+    cfg_of("bf16", L=650, B=45, H=3),
 ]
 
 
