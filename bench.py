@@ -38,7 +38,7 @@ NCU_TRAFFIC_BYTES = {
     # before a launch and part of a kernel's writes can still sit in L2 when it ends
     # (the router launch includes the SSD step sizes; the projection reads the cleared rows it adds to;
     # the slot-mix and stand-alone step-size kernels do not run in this workload: no capture)
-    "ssd_tiles": 79.649e6, "router_topk": 26.790e6, "expert_gemm": 36.987e6,
+    "ssd_tiles": 82.547e6, "router_topk": 26.790e6, "expert_gemm": 36.986e6,
     # decode workload (profiles/decode_update_kernel.md)
     "decode_update": 479.8e6,
 }

@@ -743,7 +743,7 @@ static int ssd_split_tiles(int B, int L, int H, int G, int sm_count)
         const float m = whole > lead ? whole : lead;
         if (m < best) { best = m; best_a = a; }
     }
-    return best < 0.93f * n ? best_a : 0;
+    return best < 0.95f * n ? best_a : 0;
 }
 
 int launch_ssd_scalars(LaunchCtx &ctx, const ScalarsArgs &sa)
