@@ -142,6 +142,37 @@ def test_forward_is_bitwise_reproducible():
     assert torch.equal(a["idx"], b["idx"])
 
 
+@pytest.mark.parametrize("shape", [dict(L=400), dict(L=700, B=40, H=4), dict(L=5000, B=1, H=2)])
+def test_calls_queued_back_to_back_do_not_disturb_each_other(shape):
+    """Three forwards on one handle, one workspace and one stream with no host synchronisation in
+    between (inputs A, B, A): the kernels of a call start under the tail of the kernel before them,
+    but never under an earlier call.  Each result must equal that of the same call made alone.
+    Shapes: one CTA per head pair, the split launch, the segmented launch."""
+    cfg = cfg_of("bf16", **shape)
+    ia = synth.make_inputs(cfg, seed=21)
+    ib = dict(synth.make_inputs(cfg, seed=22), **{n: ia[n] for n in ("W_r", "W_e", "A", "dt_bias", "D")})
+    alone = [hp.gpu_forward(cfg, ia), hp.gpu_forward(cfg, ib)]
+    h = hp.create_handle(cfg)
+    w, keep = hp.device_weights(ia)
+    dev_in = [{n: hp.dev(i[n]) for n in ("u", "x", "dt")} for i in (ia, ib)]
+    ws = torch.empty(sb.swimba_workspace_bytes(h, cfg.B, cfg.L), dtype=torch.uint8, device="cuda")
+    outs = []
+    for which in (0, 1, 0):
+        d = dev_in[which]
+        y = torch.full_like(d["x"], float("nan"))
+        hf = torch.full((cfg.B, cfg.H, cfg.P, cfg.N), float("nan"), device="cuda")
+        idx = torch.full((cfg.B, cfg.L, cfg.k), -1, dtype=torch.int32, device="cuda")
+        wt = torch.full((cfg.B, cfg.L, cfg.k), float("nan"), device="cuda")
+        sb.swimba_forward(h, w, d["u"], d["x"], d["dt"], None, cfg.B, cfg.L, y, hf, idx, wt, ws)
+        outs.append((y, hf, idx))
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    for (y, hf, idx), ref in zip(outs, (alone[0], alone[1], alone[0])):
+        assert torch.equal(y.cpu().view(torch.int16), ref["y"].view(torch.int16))
+        assert torch.equal(hf.cpu(), ref["h_final"])
+        assert torch.equal(idx.cpu(), ref["idx"])
+
+
 def test_theorem3_state_bound_holds_on_device():
     # ||h_T|| <= rho^T ||h_0|| + (1-rho^T)/(1-rho) U, per (head, channel), with the mixed streams
     cfg = cfg_of("fp32", L=256, B=1, N=32, P=16, H=2, h0_std=1.0)
