@@ -475,7 +475,7 @@ router_stream_kernel(const __grid_constant__ CUtensorMap tmap_u, const __nv_bflo
         }
         const uint4 *W4 = reinterpret_cast<const uint4 *>(W_r);
         const int vec_per_row = F >> 3, n_vec = E * vec_per_row;
-#pragma unroll 4
+#pragma unroll 8
         for (int i = tid; i < n_vec; i += RS_THREADS) {
             const int e = i / vec_per_row, v = i - e * vec_per_row;
             const uint4 val = W4[i];
