@@ -695,7 +695,8 @@ int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count)
     return seg_tiles * ST;
 }
 
-// Workspace: [Delta / log-decay pairs B*H*Lpad float2] [segment states] [segment decays].
+// Workspace: [log-decays B*H*Lpad float] [per-tile records B*H*(Lpad/128)] [segment states]
+// [segment decays].
 static size_t ssd_scalars_bytes(int B, int L, int H)
 {
     const size_t Lpad = (size_t)ceil_div(L, ST) * ST;
