@@ -65,6 +65,7 @@ CASES = [
     # two CTAs (leading tiles / whole sequence with a state-only lead); even and odd head counts
     cfg_of("bf16", L=700, B=40, H=4, h0_std=0.3),
     cfg_of("bf16", L=650, B=45, H=3),
+    cfg_of("bf16", L=520, B=40, H=4, G=2),                 # the same with two B/C groups
 ]
 
 
