@@ -1,17 +1,26 @@
 #!/usr/bin/env python
 """Benchmark of the Swimba token-mixer forward on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config small_lm] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config mid] [--impl ours|reference]
 
 One "step" is one pass of the whole hot path (router, top-k, expert projection, mix, SSD) over one
-batch of synthetic layer-shaped input.  Prints ONE JSON line on rank 0.  With N > 1 (torchrun)
-every rank runs an independent replica on its own batch: the path has no exchange step, so there
-is no collective on the data path (weak scaling).
+batch of synthetic layer-shaped input.  Prints ONE JSON line on rank 0.  The headline workload is
+`mid` (the largest single-GPU forward shape that is run beside the dense and separated
+comparators); `small_lm` and `long_seq` ride along as compact records under "workloads", the
+decode workload under "decode".  With N > 1 (torchrun) every rank runs an independent replica on
+its own batch: the path has no exchange step, so there is no collective on the data path (weak
+scaling).
+
+Timing.  The K-step timed region (barrier + synchronize on both sides, CUDA events on the launching
+stream, max over ranks) is repeated back to back until about 1.5 s have passed, so that the clock
+sampler sees the load; the reported step time is the median round's.
 """
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -29,19 +38,23 @@ from paper_2603_06938_b200 import replicas, synth
 
 METRIC = "swimba_layer_fwd_tokens_per_s"
 UNIT = "tokens/s"
-NSETS = 4   # rotating input sets: together several times the 126 MB L2
+L2_BYTES = 126e6
+TIMED_SECONDS = 1.5   # the K-step timed region is repeated until it has covered about this long
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of each kernel from the ncu
-# captures summarised under profiles/; None until a capture of that kernel exists.
+# captures summarised under profiles/, per workload; a (workload, kernel) pair without a capture of
+# the current kernel reports null.  ncu flushes caches before a launch, and part of a kernel's
+# writes can still sit in L2 when it ends.
 NCU_TRAFFIC_BYTES = {
-    # workload small_lm, one launch each (profiles/forward_small_lm_kernels.md); ncu flushes caches
-    # before a launch and part of a kernel's writes can still sit in L2 when it ends
-    # (the router launch includes the SSD step sizes; the projection reads the cleared rows it adds to;
-    # the slot-mix and stand-alone step-size kernels do not run in this workload: no capture)
-    "ssd_tiles": 82.547e6, "router_topk": 26.790e6, "expert_gemm": 36.986e6,
-    # decode workload (profiles/decode_update_kernel.md)
-    "decode_update": 479.8e6,
+    "small_lm": {},
+    "mid": {},
+    "long_seq": {},
+    "decode": {},
 }
+
+
+def ncu_traffic(workload, kernel):
+    return NCU_TRAFFIC_BYTES.get(workload, {}).get(kernel)
 
 
 def peaks():
@@ -79,9 +92,13 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self):
+    def mark(self):
+        return time.time()
+
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken between the two marks (all samples without marks)."""
         if self.proc is None:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
         time.sleep(0.15)
@@ -90,12 +107,15 @@ class ClockSampler:
             self.proc.wait(timeout=2)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for ts, r in self.rows:
+            if t_begin is not None and not (t_begin <= ts <= t_end + 0.05):
+                continue
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
+                pw.append(float(r[2]))
                 for n, v in zip(names, r[3:7]):
                     if v.lower().startswith("active"):
                         reasons.add(n)
@@ -103,11 +123,12 @@ class ClockSampler:
                 pass
         return dict(sm_mhz=statistics.median(sm) if sm else None,
                     sm_max_mhz=max(mx) if mx else None, reasons=sorted(reasons),
-                    samples=len(sm))
+                    samples=len(sm), power_w_max=max(pw) if pw else None,
+                    window="samples taken during the timed rounds of the headline workload")
 
 
-def algorithmic_work(cfg: synth.LayerConfig, sm_count: int = 148):
-    """Per-launch algorithmic work of each kernel for B x L tokens: bytes the method must move or
+def algorithmic_work(cfg: synth.LayerConfig, nseg: int = 1, sm_count: int = 148):
+    """Per-step algorithmic work of each kernel for B x L tokens: bytes the method must move or
     flops it must execute, not what a particular kernel happens to do."""
     T, F, S, E, k = cfg.tokens, cfg.F, cfg.S, cfg.E, cfg.k
     H, P, N, G, Q = cfg.H, cfg.P, cfg.N, cfg.G, cfg.Q
@@ -125,12 +146,13 @@ def algorithmic_work(cfg: synth.LayerConfig, sm_count: int = 148):
     ssd_bytes = T * (2 * H * P * es + S * es + H * 4) + cfg.B * H * P * N * 4
     w["ssd_tiles"] = dict(bound="tensor", work=ssd_flops, bytes=ssd_bytes)
     w["ssd_sequential"] = dict(bound="alu", work=4.0 * T * H * P * N, bytes=ssd_bytes)
-    w["segment_scan"] = dict(bound="hbm", work=0)
+    # the scan reads every segment's local end state and writes the state entering it
+    w["segment_scan"] = dict(bound="hbm", work=2 * nseg * cfg.B * H * P * N * 4)
     w["ssd_scalars"] = dict(bound="hbm", work=T * H * 12)
     return w
 
 
-def roofline_entry(name, avg_ms, work, pk):
+def roofline_entry(workload, name, avg_ms, work, pk):
     info = work.get(name)
     if info is None or avg_ms <= 0:
         return None
@@ -140,7 +162,7 @@ def roofline_entry(name, avg_ms, work, pk):
         t_tc = info["work"] / (pk["bf16_tflops"] * 1e12)
         ach_b = info["bytes"] / (avg_ms * 1e-3) / 1e9
         ach_f = info["work"] / (avg_ms * 1e-3) / 1e12
-        ent = dict(kernel=name, traffic=NCU_TRAFFIC_BYTES.get(name), peak_source=pk["source"],
+        ent = dict(kernel=name, traffic=ncu_traffic(workload, name), peak_source=pk["source"],
                    avg_ms=avg_ms, hbm_frac=ach_b / pk["hbm_gbs"], tensor_frac=ach_f / pk["bf16_tflops"])
         if t_hbm >= t_tc:
             ent.update(bound="hbm", achieved=ach_b, peak=pk["hbm_gbs"], unit="GB/s",
@@ -160,13 +182,12 @@ def roofline_entry(name, avg_ms, work, pk):
         ach = info["work"] / (avg_ms * 1e-3) / 1e12
         peak, unit = 148 * 128 * 2 * 1.965e9 / 1e12, "TFLOP/s"
     return dict(kernel=name, bound=info["bound"], achieved=ach, peak=peak, unit=unit,
-                frac=ach / peak, traffic=NCU_TRAFFIC_BYTES.get(name),
+                frac=ach / peak, traffic=ncu_traffic(workload, name),
                 peak_source=pk["source"], avg_ms=avg_ms)
 
 
 def time_oracle_sample(cfg: synth.LayerConfig, n_seq: int, seed: int = 0):
     """The CPU oracle, as it stands, on n_seq whole sequences of the workload."""
-    import dataclasses
     import oracle
     sub = dataclasses.replace(cfg, B=n_seq)
     inp = synth.make_inputs(sub, seed=seed)
@@ -179,54 +200,149 @@ def time_oracle_sample(cfg: synth.LayerConfig, n_seq: int, seed: int = 0):
                        f"{dt:.2f} s"), dt
 
 
-def time_layer(sb, cfg, steps, warmup, n_sets=2, seed0=5000, repeat=1):
-    """ms per forward of one layer configuration through swimba_forward (device-resident inputs)."""
-    dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
-    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
-    sets = [synth.make_inputs(cfg, seed=seed0 + i) for i in range(n_sets)]
-    wts = {n: sets[0][n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
-    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
-    dev = [dict(u=s_["u"].cuda(), x=s_["x"].cuda(), dt=s_["dt"].cuda()) for s_ in sets]
-    y = torch.empty_like(dev[0]["x"])
-    hf = torch.empty(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
-    ws = torch.empty(sb.swimba_workspace_bytes(h, cfg.B, cfg.L), dtype=torch.uint8, device="cuda")
+def input_sets_needed(cfg: synth.LayerConfig) -> int:
+    """Distinct input sets to rotate over so that together they are several times the L2."""
+    es = 2 if cfg.dtype == "bf16" else 4
+    per_set = cfg.tokens * (cfg.F * es + cfg.H * cfg.P * es + cfg.H * 4)
+    return max(2, min(8, math.ceil(4 * L2_BYTES / per_set)))
+
+
+class Layer:
+    """One layer configuration resident on the device: handle, weights, rotating inputs, outputs."""
+
+    def __init__(self, sb, cfg: synth.LayerConfig, rank: int = 0, seed0: int = 0, n_sets=None):
+        self.sb, self.cfg = sb, cfg
+        dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
+        self.h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
+        self.n_sets = n_sets or input_sets_needed(cfg)
+        self.host_sets = [synth.make_inputs(cfg, seed=seed0 + replicas.replica_seed(rank, i))
+                          for i in range(self.n_sets)]
+        s0 = self.host_sets[0]
+        self.wts = {n: s0[n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
+        self.w = sb.make_weights(*(self.wts[n] for n in ("W_r", "W_e", "A", "dt_bias", "D")))
+        self.dev = [dict(u=s["u"].cuda(), x=s["x"].cuda(), dt=s["dt"].cuda()) for s in self.host_sets]
+        self.y = torch.empty_like(self.dev[0]["x"])
+        self.hf = torch.empty(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
+        self.ws = torch.empty(sb.swimba_workspace_bytes(self.h, cfg.B, cfg.L), dtype=torch.uint8,
+                              device="cuda")
+
+    def step(self, i):
+        d = self.dev[i % self.n_sets]
+        c = self.cfg
+        self.sb.swimba_forward(self.h, self.w, d["u"], d["x"], d["dt"], None, c.B, c.L, self.y, self.hf,
+                               None, None, self.ws)
+
+    def check(self):
+        assert self.sb.swimba_status(self.h) == 0, self.sb.swimba_last_error(self.h)
+
+    def close(self):
+        self.sb.swimba_destroy(self.h)
+        self.dev = self.ws = self.y = self.hf = None
+
+
+def time_rounds(layer: Layer, steps: int, warmup: int, dist, min_seconds: float, repeat: int = 1):
+    """Warm-up, then rounds of exactly `steps` steps, each bracketed by a barrier and a device
+    synchronisation on both sides and timed with CUDA events on the launching stream; every
+    round's time is the maximum over ranks.  Returns (median ms per step, [ms per step of every
+    round], launches per step)."""
     stream = torch.cuda.current_stream()
 
-    def step(i):
-        d = dev[i % n_sets]
-        for _ in range(repeat):
-            sb.swimba_forward(h, w, d["u"], d["x"], d["dt"], None, cfg.B, cfg.L, y, hf, None, None, ws)
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
 
-    for i in range(warmup):
-        step(i)
-    torch.cuda.synchronize()
+    def run(n, base):
+        for i in range(n):
+            for _ in range(repeat):
+                layer.step(base + i)
+
+    run(warmup, 0)
+    layer.check()
+    launches = layer.sb.swimba_last_launch_count(layer.h)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
     e0.record(stream)
-    for i in range(steps):
-        step(i)
+    run(steps, 0)
     e1.record(stream)
-    torch.cuda.synchronize()
-    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
-    sb.swimba_destroy(h)
-    return e0.elapsed_time(e1) / steps
+    barrier()
+    first = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
+    rounds = [first / steps]
+    n_more = int(min(2000, max(0, math.ceil(min_seconds * 1e3 / max(first, 1e-3)) - 1)))
+    for r in range(n_more):
+        barrier()
+        e0.record(stream)
+        run(steps, (r + 1) * steps)
+        e1.record(stream)
+        barrier()
+        rounds.append(e0.elapsed_time(e1) / steps)
+    if dist is not None and len(rounds) > 1:
+        t = torch.tensor(rounds, dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        rounds = [float(v) for v in t.tolist()]
+    layer.check()
+    return statistics.median(rounds), rounds, launches
 
 
-def bench_comparators(sb, cfg, steps, warmup, ms_swimba):
+def kernel_breakdown(layer: Layer, n: int, pk, sm_count: int):
+    """Per-kernel durations, live, same launch configuration: CUDA events around every kernel
+    (swimba_profile), read from the second of two back-to-back calls, so that the call's first
+    kernel starts behind a busy GPU as in the timed loop."""
+    sb, cfg = layer.sb, layer.cfg
+    sb.swimba_profile(layer.h, True)
+    per = {}
+    for i in range(n):
+        layer.step(i)
+        layer.step(i + 1)
+        for name, ms in sb.swimba_profile_read(layer.h):
+            per.setdefault(name, []).append(ms)
+    sb.swimba_profile(layer.h, False)
+    nseg = sb.swimba_ssd_segments(layer.h, cfg.B, cfg.L)
+    work = algorithmic_work(cfg, nseg, sm_count)
+    tot = sum(sum(v) for v in per.values())
+    kernels = []
+    for name, v in per.items():
+        n_per_step = len(v) / n
+        # a kernel launched several times per step (the two SSD passes of segmented sequences) is
+        # rated on its time per step: the algorithmic work is per step
+        ms_per_step_k = sum(v) / n
+        ent = roofline_entry(cfg.name, name, ms_per_step_k, work, pk) or dict(kernel=name, avg_ms=ms_per_step_k)
+        ent["avg_ms"] = sum(v) / len(v)
+        ent["ms_per_step"] = ms_per_step_k
+        ent["share"] = sum(v) / tot if tot > 0 else 0.0
+        ent["launches_per_step"] = n_per_step
+        npos = int(round(n_per_step))
+        if npos > 1 and len(v) % npos == 0:
+            ent["per_launch_ms"] = [sum(v[i::npos]) / (len(v) // npos) for i in range(npos)]
+        kernels.append(ent)
+    kernels.sort(key=lambda e: -e["share"])
+    return kernels, nseg
+
+
+def dense_ratio(sb, cfg, steps, warmup, ms_swimba, with_separated: bool):
     """The same shape as (1) a dense Mamba-2 layer: the library with E = k = 1 (no router, one
     projection), and (2) E separated SSMs: every expert's streams projected for every token and E
     independent SSD evaluations with E states (the readout sum over the active experts is left
     out, so the figure is a lower bound of that design's cost)."""
-    import dataclasses
     dense = dataclasses.replace(cfg, name=cfg.name + "_dense", E=1, k=1)
-    ms_dense = time_layer(sb, dense, steps, warmup)
-    ms_sep = time_layer(sb, dense, steps, warmup, repeat=cfg.E)
-    return {
-        "dense_mamba2": {"ms_per_step": ms_dense, "swimba_over_dense": ms_swimba / ms_dense,
-                         "how": "same library, E = k = 1"},
-        "separated_ssm_E_fold": {"ms_per_step": ms_sep, "swimba_over_separated": ms_swimba / ms_sep,
-                                 "how": f"{cfg.E} dense-layer passes back to back (one projection "
-                                        f"and one SSD evaluation per expert), readout sum not counted"},
-    }
+    lay = Layer(sb, dense, seed0=5000, n_sets=2)
+    ms_dense, _, _ = time_rounds(lay, steps, warmup, None, 0.3)
+    out = {"dense_mamba2": {"ms_per_step": ms_dense, "swimba_over_dense": ms_swimba / ms_dense,
+                            "how": "same library, E = k = 1"}}
+    if with_separated:
+        ms_sep, _, _ = time_rounds(lay, steps, warmup, None, 0.0, repeat=cfg.E)
+        out["separated_ssm_E_fold"] = {
+            "ms_per_step": ms_sep, "swimba_over_separated": ms_swimba / ms_sep,
+            "how": f"{cfg.E} dense-layer passes back to back (one projection and one SSD "
+                   f"evaluation per expert), readout sum not counted"}
+    lay.close()
+    return out
+
+
+def compact_kernels(kernels):
+    keep = ("kernel", "bound", "frac", "hbm_frac", "tensor_frac", "ms_per_step", "share",
+            "launches_per_step", "per_launch_ms", "traffic")
+    return [{k_: e[k_] for k_ in keep if k_ in e} for e in kernels]
 
 
 def run_reference(args, cfg, rank, world):
@@ -244,37 +360,40 @@ def run_reference(args, cfg, rank, world):
     value = tok / (ms * 1e-3)
     cb = dict(vals[-1])
     cb["value"] = value
+    cb["sample"] = f"every step: {n_seq} of {cfg.B} sequences x {cfg.L} tokens of {cfg.name}, fp64"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": config_dict(cfg, sample=f"{n_seq} sequence(s) per step"),
+        "config": config_dict(cfg),
         "cpu_baseline": cb,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
 
-def config_dict(cfg, **extra):
-    d = {"workload": f"{cfg.name}: B={cfg.B} L={cfg.L} d_model={cfg.F} H={cfg.H} P={cfg.P} "
-                     f"N={cfg.N} G={cfg.G} E={cfg.E} top_k={cfg.k} chunk={cfg.Q} {cfg.dtype}",
-         "tokens_per_step_per_gpu": cfg.tokens,
-         "l2_policy": f"inputs rotate over {NSETS} distinct sets (> L2) between timed steps"}
-    d.update(extra)
-    return d
+def config_dict(cfg):
+    return {"workload": f"{cfg.name}: B={cfg.B} L={cfg.L} d_model={cfg.F} H={cfg.H} P={cfg.P} "
+                        f"N={cfg.N} G={cfg.G} E={cfg.E} top_k={cfg.k} chunk={cfg.Q} {cfg.dtype}",
+            "tokens_per_step_per_gpu": cfg.tokens,
+            "l2_policy": f"inputs rotate over {input_sets_needed(cfg)} distinct sets (> L2) between timed steps"}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", default="small_lm", choices=[c for c in synth.CONFIG_ORDER if c != "decode"])
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="mid", choices=[c for c in synth.CONFIG_ORDER if c != "decode"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seconds", type=float, default=TIMED_SECONDS,
+                    help="the K-step timed region is repeated until about this long has been timed")
     ap.add_argument("--no-decode", action="store_true")
     ap.add_argument("--decode-steps", type=int, default=512,
                     help="consecutive steps timed by the decode leg (the workload has 512)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-comparators", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="skip the compact records of the other forward workloads")
     ap.add_argument("--no-e2e", action="store_true",
                     help="skip the host-buffer leg (for profiler launch lists of the device-resident steps)")
     args = ap.parse_args()
@@ -293,126 +412,106 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
     pk = peaks()
-    dcode = sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
-    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, dcode)
-    sets = [synth.make_inputs(cfg, seed=replicas.replica_seed(rank, i)) for i in range(NSETS)]
-    wts = {n: sets[0][n].cuda() for n in ("W_r", "W_e", "A", "dt_bias", "D")}
-    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
-    dev_sets = [dict(u=s["u"].cuda(), x=s["x"].cuda(), dt=s["dt"].cuda()) for s in sets]
-    B, L = cfg.B, cfg.L
-    y = torch.empty_like(dev_sets[0]["x"])
-    hf = torch.empty(B, cfg.H, cfg.P, cfg.N, device="cuda")
-    ws = torch.empty(sb.swimba_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     stream = torch.cuda.current_stream()
 
-    def step(i):
-        s = dev_sets[i % NSETS]
-        sb.swimba_forward(h, w, s["u"], s["x"], s["dt"], None, B, L, y, hf, None, None, ws)
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
+    layer = Layer(sb, cfg, rank=rank)
     # the clock sampler is up before the warm-up, so that the warm-up steps run right in front of
     # the timed ones (no idle gap in which the GPU could leave its boost state)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.2)
-    for i in range(args.warmup):
-        step(i)
-    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
-    launches_per_step = sb.swimba_last_launch_count(h)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    barrier()
-    ms_total = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
-    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
-    ms_step = ms_total / args.steps
+    t_begin = sampler.mark()
+    ms_step, rounds, launches_per_step = time_rounds(layer, args.steps, args.warmup, dist, args.seconds)
+    t_end = sampler.mark()
     value = replicas.whole_job_throughput(world, cfg.tokens, ms_step)
+    kernels, nseg = kernel_breakdown(layer, max(args.steps, 20), pk, sm_count)
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
 
-    # per-kernel durations, live, same launch configuration (CUDA events around every kernel)
-    sb.swimba_profile(h, True)
-    per = {}
-    for i in range(args.steps):
-        # two calls back to back, the second one is read: its first kernel then starts behind a
-        # busy GPU, as in the timed loop, instead of absorbing the host's launch latency
-        step(i)
-        step(i + 1)
-        for name, ms in sb.swimba_profile_read(h):
-            per.setdefault(name, []).append(ms)
-    sb.swimba_profile(h, False)
-    clocks = sampler.stop() if rank == 0 else None
-
-    work = algorithmic_work(cfg, torch.cuda.get_device_properties(local).multi_processor_count)
-    tot = sum(sum(v) for v in per.values())
-    kernels = []
-    for name, v in per.items():
-        n_per_step = len(v) / args.steps
-        # a kernel launched several times per step (the two SSD passes of segmented sequences) is
-        # rated on its time per step: the algorithmic work is per step
-        ms_per_step_k = sum(v) / args.steps
-        ent = roofline_entry(name, ms_per_step_k, work, pk) or dict(kernel=name, avg_ms=ms_per_step_k)
-        ent["avg_ms"] = sum(v) / len(v)
-        ent["ms_per_step"] = ms_per_step_k
-        ent["share"] = sum(v) / tot if tot > 0 else 0.0
-        ent["launches_per_step"] = n_per_step
-        npos = int(round(n_per_step))
-        if npos > 1 and len(v) % npos == 0:
-            ent["per_launch_ms"] = [sum(v[i::npos]) / (len(v) // npos) for i in range(npos)]
-        kernels.append(ent)
-    kernels.sort(key=lambda e: -e["share"])
     dom = kernels[0] if kernels else None
     roofline = None
     if dom and "bound" in dom:
         roofline = {k_: dom[k_] for k_ in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
         roofline["kernel"] = dom["kernel"]
         roofline["peak_source"] = "of " + pk["source"]
+        for k_ in ("hbm_frac", "tensor_frac"):
+            if k_ in dom:
+                roofline[k_] = dom[k_]
 
     e2e = None
-    hws = None
     if not args.no_e2e:
         # end to end through the host-buffer entry point: pinned host inputs, H2D and D2H in the timed region
-        hws = torch.empty(sb.swimba_host_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+        B, L = cfg.B, cfg.L
+        hws = torch.empty(sb.swimba_host_workspace_bytes(layer.h, B, L), dtype=torch.uint8, device="cuda")
         host_sets = [dict(u=s["u"].pin_memory(), x=s["x"].pin_memory(), dt=s["dt"].pin_memory())
-                     for s in sets[:2]]
-        y_host = torch.empty_like(sets[0]["x"]).pin_memory()
-        for i in range(2):
+                     for s in layer.host_sets[:2]]
+        y_host = torch.empty_like(layer.host_sets[0]["x"]).pin_memory()
+
+        def host_step(i):
             s = host_sets[i % 2]
-            sb.swimba_forward_host(h, w, s["u"], s["x"], s["dt"], B, L, y_host, None, None, None, hws)
-        barrier()
+            sb.swimba_forward_host(layer.h, layer.w, s["u"], s["x"], s["dt"], B, L, y_host, None, None,
+                                   None, hws)
+
+        for i in range(3):
+            host_step(i)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for i in range(args.steps):
-            s = host_sets[i % 2]
-            sb.swimba_forward_host(h, w, s["u"], s["x"], s["dt"], B, L, y_host, None, None, None, hws)
+            host_step(i)
         e1.record(stream)
-        barrier()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
         e2e_ms = replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
+        layer.check()
         es = 2 if cfg.dtype == "bf16" else 4
         h2d = cfg.tokens * (cfg.F * es + cfg.H * cfg.P * es + cfg.H * 4)
         d2h = cfg.tokens * cfg.H * cfg.P * es
         e2e = {"value": replicas.whole_job_throughput(world, cfg.tokens, e2e_ms / args.steps), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-    sb.swimba_destroy(h)
-    del dev_sets, hws, ws, y, hf
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "how": "swimba_forward_host: pinned host u, x, dt in, y out, every step"}
+        del hws, host_sets, y_host
+    layer.close()
+    del layer
+    torch.cuda.empty_cache()
+
+    single = rank == 0 and world == 1
+    comparators = None
+    if single and not args.no_comparators:
+        comparators = dense_ratio(sb, cfg, args.steps, args.warmup, ms_step, with_separated=True)
+
+    workloads = None
+    if single and not args.no_workloads:
+        workloads = {}
+        for name in ("small_lm", "long_seq", "mid"):
+            if name == cfg.name:
+                continue
+            c2 = synth.CONFIGS[name]
+            lay = Layer(sb, c2)
+            ms2, r2, l2 = time_rounds(lay, args.steps, args.warmup, None, 0.5)
+            k2, nseg2 = kernel_breakdown(lay, max(args.steps, 20), pk, sm_count)
+            lay.close()
+            del lay
+            torch.cuda.empty_cache()
+            rec = {"workload": config_dict(c2)["workload"], "ms_per_step": ms2,
+                   "value": c2.tokens / (ms2 * 1e-3), "unit": UNIT, "rounds": len(r2),
+                   "launches_per_step": l2, "ssd_segments": nseg2, "kernels": compact_kernels(k2)}
+            if not args.no_comparators:
+                rec["swimba_over_dense"] = dense_ratio(sb, c2, args.steps, args.warmup, ms2, False)[
+                    "dense_mamba2"]["swimba_over_dense"]
+            workloads[name] = rec
 
     decode = None
-    if rank == 0 and world == 1 and not args.no_decode:
+    if single and not args.no_decode:
         decode = bench_decode(sb, pk, steps=args.decode_steps)
 
-    comparators = None
-    if rank == 0 and world == 1 and not args.no_comparators:
-        comparators = bench_comparators(sb, cfg, args.steps, args.warmup, ms_step)
-
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if single and not args.no_cpu_baseline:
         cpu, _ = time_oracle_sample(cfg, cfg.B)
 
     if rank == 0:
@@ -422,7 +521,13 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32",
             "data": "synthetic", "config": config_dict(cfg), "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "roofline": roofline,
-            "kernels": kernels, "decode": decode, "comparators": comparators, "cpu_baseline": cpu,
+            "timing": {"rounds": len(rounds), "steps_per_round": args.steps,
+                       "ms_per_step_median": ms_step, "ms_per_step_min": min(rounds),
+                       "ms_per_step_max": max(rounds),
+                       "how": "value is the median over rounds of exactly `steps` steps each"},
+            "ssd_segments": nseg,
+            "kernels": kernels, "comparators": comparators, "workloads": workloads,
+            "decode": decode, "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     if dist is not None:
@@ -481,7 +586,7 @@ def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
                      "achieved": state_bytes / (upd_us * 1e-6) / 1e9 if upd_us > 0 else None,
                      "peak": pk["hbm_gbs"], "unit": "GB/s",
                      "frac": state_bytes / (upd_us * 1e-6) / 1e9 / pk["hbm_gbs"] if upd_us > 0 else None,
-                     "traffic": NCU_TRAFFIC_BYTES.get("decode_update"),
+                     "traffic": ncu_traffic("decode", "decode_update"),
                      "whole_step_frac": state_bytes / (us * 1e-6) / 1e9 / pk["hbm_gbs"]},
     }
     sb.swimba_destroy(h)

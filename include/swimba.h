@@ -121,6 +121,14 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
                const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
+/* How many segments the SSD evaluation cuts every sequence of a B x L call into (Background,
+ * "Mamba-2 and SSD": a linear recurrence between blocks of tokens).  1: each sequence is walked
+ * once with the carried state kept on chip.  More than 1 (long sequences, few of them): a first
+ * pass computes every segment's end state, a scan chains them, a second pass produces y; the
+ * workspace then holds segments * B*H*P*N floats of segment states.  0 if B or L is not
+ * positive.  The result does not depend on the segmentation beyond rounding. */
+int32_t swimba_ssd_segments(const swimba_handle *h, int32_t B, int32_t L);
+
 /* Bytes of device workspace swimba_decode_step needs for B sequences. */
 size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B);
 
@@ -158,8 +166,10 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
  * workspace.
  *   - The array is SWIMBA_STATIC_SCRATCH_BYTES large and is held by every GPU that loads the
  *     library until the process exits.  Token counts whose scratch need exceeds it are rejected
- *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (with bf16, S = 256,
- *     E = 8 and k = 2 the limit is about 14000 tokens per call).
+ *     with SWIMBA_ERR_WORKSPACE_TOO_SMALL and a message naming both sizes (the need is 8 k bytes per
+ *     token for the routing outputs plus, on the bf16 tensor-core path, 4 E bytes per token of
+ *     per-expert lists and, for k > 2, 2 k S bytes of per-slot projections: about 170000 tokens
+ *     per call with E = 8, k = 2; about 5000 with S = 256, k = 3).
  *   - The first call on each device looks up the array's device address; make that first call
  *     outside any stream capture.  No call allocates or frees device memory.
  *   - All calls on a device share the one array, and it keeps the previous call's contents (the
@@ -172,7 +182,7 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router + grouping by
+ * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router + grouping by
  * expert (for fewer than about 28000 tokens the launch also computes the SSD step sizes), 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
  * tile kernel, 10 segment scan, 11 SSD step sizes and decays; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */

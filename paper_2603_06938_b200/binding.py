@@ -28,7 +28,7 @@ DTYPE_FP32 = 0
 DTYPE_BF16 = 1
 
 EXPORTS = [
-    "swimba_create", "swimba_workspace_bytes", "swimba_forward", "swimba_route_mix", "swimba_ssd",
+    "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
     "swimba_forward_host", "swimba_route_mix_static", "swimba_profile", "swimba_profile_read",
     "swimba_last_launch_count", "swimba_status", "swimba_last_error",
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
         L.swimba_create.restype = ctypes.c_int
         L.swimba_workspace_bytes.argtypes = [vp, i32, i32]
         L.swimba_workspace_bytes.restype = sz
+        L.swimba_ssd_segments.argtypes = [vp, i32, i32]
+        L.swimba_ssd_segments.restype = i32
         L.swimba_decode_workspace_bytes.argtypes = [vp, i32]
         L.swimba_decode_workspace_bytes.restype = sz
         L.swimba_host_workspace_bytes.argtypes = [vp, i32, i32]
@@ -160,6 +162,10 @@ def make_weights(W_router, W_expert, A, dt_bias, D) -> swimba_weights:
 
 def swimba_workspace_bytes(h: Handle, B: int, L: int) -> int:
     return int(lib().swimba_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_ssd_segments(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_ssd_segments(h.ptr, B, L))
 
 
 def swimba_decode_workspace_bytes(h: Handle, B: int) -> int:

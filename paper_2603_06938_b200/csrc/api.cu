@@ -217,6 +217,30 @@ int run_ssd(swimba_handle *h, LaunchCtx &ctx, const swimba_weights *w, const voi
     return SWIMBA_OK;
 }
 
+// The routing/projection stage with its scratch regions given one by one (idx_scratch / w_scratch
+// are used when the caller does not ask for the routing outputs).
+int route_mix_call(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T, void *BC,
+                   int32_t *topk_idx, float *topk_w, void *idx_scratch, void *w_scratch,
+                   void *gemm_ws, void *cuda_stream)
+{
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !BC) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC or workspace is NULL");
+    if (!aligned16(u) || !aligned16(BC) || !aligned16(idx_scratch) || !aligned16(w_scratch) ||
+        !aligned16(gemm_ws) || !aligned16(topk_idx) || !aligned16(topk_w))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    h->prof.n = 0;
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)idx_scratch;
+    float *wt = topk_w ? topk_w : (float *)w_scratch;
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, gemm_ws);
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -264,6 +288,15 @@ size_t swimba_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
     return fwd_layout(h->cfg, B, L, h->sm_count).total;
 }
 
+int32_t swimba_ssd_segments(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    const swimba_config &c = h->cfg;
+    if (!ssd_tiles_supported(c.dtype, c.head_dim, c.d_state)) return 1;
+    const int seg_len = ssd_segment_len(B, L, c.n_heads, c.n_groups, c.chunk, h->sm_count);
+    return (L + seg_len - 1) / seg_len;
+}
+
 size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B)
 {
     if (!h || B <= 0) return 0;
@@ -285,24 +318,11 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
     // (token, slot) entries are indexed with 32-bit integers
     if (T < 0 || T * h->cfg.top_k >= (int64_t)1 << 31)
         return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range (T * top_k must stay below 2^31)");
-    int rc = check_weights(h, w, true);
-    if (rc != SWIMBA_OK) return rc;
-    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
-    if (!u || !BC || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC or workspace is NULL");
-    if (!aligned16(u) || !aligned16(BC) || !aligned16(workspace) || !aligned16(topk_idx) || !aligned16(topk_w))
-        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    if (T > 0 && !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC or workspace is NULL");
     const FwdLayout l = fwd_layout(h->cfg, 1, (int)T, h->sm_count);
-    if (workspace_bytes < l.ssd) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
-    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    if (T > 0 && workspace_bytes < l.ssd) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
-    h->prof.n = 0;
-    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
-    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
-    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
-    h->last_stream = ctx.stream;
-    h->last_launches = ctx.launches;
-    return rc;
+    return route_mix_call(h, w, u, T, BC, topk_idx, topk_w, ws + l.idx, ws + l.w, ws + l.gemm, cuda_stream);
 }
 
 int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const void *BC,
@@ -461,7 +481,7 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
                             h_final_host ? (float *)(ws + l.hf + (size_t)b0 * seq_hf) : nullptr,
                             (int32_t *)(ws + l.idx + t0 * tok_k), (float *)(ws + l.w + t0 * tok_k),
                             ws + l.fwd, workspace_bytes - l.fwd, cuda_stream);
-        if (rc != SWIMBA_OK) return rc;
+        if (rc != SWIMBA_OK) break;
         launches += h->last_launches;
         ok = cudaEventRecord(h->ev_done[slice], st) == cudaSuccess &&
              cudaStreamWaitEvent(h->s_out, h->ev_done[slice], 0) == cudaSuccess &&
@@ -477,11 +497,16 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
             ok = cudaMemcpyAsync((char *)topk_w_host + t0 * tok_k, ws + l.w + t0 * tok_k, nt * tok_k,
                                  cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
     }
-    // the caller's stream ends after the last copy out: synchronising it is enough
-    ok = ok && cudaEventRecord(h->ev_out, h->s_out) == cudaSuccess &&
-         cudaStreamWaitEvent(st, h->ev_out, 0) == cudaSuccess;
+    // The caller's stream ends after the last copy in and the last copy out, on the error paths
+    // too (copies of earlier slices may still be in flight): synchronising it is enough before the
+    // host buffers are read, reused or freed.
+    const bool joined = cudaEventRecord(h->ev_out, h->s_out) == cudaSuccess &&
+                        cudaStreamWaitEvent(st, h->ev_out, 0) == cudaSuccess &&
+                        cudaEventRecord(h->ev_start, h->s_in) == cudaSuccess &&
+                        cudaStreamWaitEvent(st, h->ev_start, 0) == cudaSuccess;
     h->last_launches = launches;
-    if (!ok) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "a copy or an event of the host pipeline failed"); }
+    if (rc != SWIMBA_OK) return rc;             // (message set by the failing forward)
+    if (!ok || !joined) { cudaGetLastError(); return fail(h, SWIMBA_ERR_CUDA, "a copy or an event of the host pipeline failed"); }
     return SWIMBA_OK;
 }
 
@@ -587,13 +612,21 @@ extern "C" int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w
         }
         g_static_scratch_ptr[h->device] = p;
     }
-    const FwdLayout l = fwd_layout(h->cfg, 1, (int)T, h->sm_count);
-    if (l.ssd > (size_t)SWIMBA_STATIC_SCRATCH_BYTES) {
+    // Regions the stage really uses: routing outputs the caller did not ask for, then the grouped
+    // GEMM's scratch (histogram, per-expert lists, slot buffer when k > 2).  BC is the caller's.
+    const swimba_config &c = h->cfg;
+    const size_t off_idx = 0;
+    const size_t off_w = off_idx + align_up((size_t)T * c.top_k * sizeof(int32_t));
+    const size_t off_gemm = off_w + align_up((size_t)T * c.top_k * sizeof(float));
+    const size_t need = off_gemm +
+        (use_tensor_k1(c) ? align_up(expert_gemm_workspace_bytes(T, 2 * c.n_groups * c.d_state, c.n_experts, c.top_k)) : 0);
+    if (need > (size_t)SWIMBA_STATIC_SCRATCH_BYTES) {
         snprintf(h->err, sizeof(h->err),
                  "T = %lld tokens needs %zu bytes of scratch, the static scratch holds %d",
-                 (long long)T, l.ssd, (int)SWIMBA_STATIC_SCRATCH_BYTES);
+                 (long long)T, need, (int)SWIMBA_STATIC_SCRATCH_BYTES);
         return SWIMBA_ERR_WORKSPACE_TOO_SMALL;
     }
-    return swimba_route_mix(h, w, u, T, BC, topk_idx, topk_w, g_static_scratch_ptr[h->device],
-                            (size_t)SWIMBA_STATIC_SCRATCH_BYTES, cuda_stream);
+    char *ws = (char *)g_static_scratch_ptr[h->device];
+    return route_mix_call(h, w, u, T, BC, topk_idx, topk_w, ws + off_idx, ws + off_w, ws + off_gemm,
+                          cuda_stream);
 }

@@ -36,6 +36,8 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
 // K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
 bool ssd_tiles_supported(int dtype, int P, int N);
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);
+// Tokens per segment the tile path cuts a sequence into (a multiple of 128; >= L: one segment).
+int ssd_segment_len(int B, int L, int H, int G, int chunk, int sm_count);
 // scalars_done: the step sizes and tile log-decays (ssd_scalars_args over the same workspace) have
 // already been produced earlier in the stream (launch_router with scalars, or launch_ssd_scalars).
 ScalarsArgs ssd_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,

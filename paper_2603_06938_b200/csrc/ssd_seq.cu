@@ -52,11 +52,11 @@ ssd_sequential_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
             const int tt = i / P, pp = i % P;
             sx[tt * P + pp] = to_f32<T>(x[(((int64_t)b * L + t0 + tt) * H + h) * P + pp]);
         }
-        if (tid < nt) {
-            const float raw = dt ? dt[((int64_t)b * L + t0 + tid) * H + h] : 0.f;
+        for (int i = tid; i < nt; i += nthr) {        // (blocks may have fewer than SEQ_TS threads)
+            const float raw = dt ? dt[((int64_t)b * L + t0 + i) * H + h] : 0.f;
             const float delta = softplus_f(raw + bias);
-            sdl[tid] = delta;
-            sa[tid] = expf(delta * Ah);
+            sdl[i] = delta;
+            sa[i] = expf(delta * Ah);
         }
         __syncthreads();
         for (int tt = 0; tt < nt; ++tt) {

@@ -75,6 +75,91 @@ def max_rel(got, ref) -> float:
     return float(np.max(np.abs(got - ref)) / (den if den > 0 else 1.0))
 
 
+def _head_max(a, head_axis):
+    """max |a| per (sequence, head): a is [B, ..., H, ...] with the head index at head_axis."""
+    axes = tuple(i for i in range(a.ndim) if i not in (0, head_axis))
+    return np.max(np.abs(a), axis=axes)
+
+
+def per_head_rel(got, ref, head_axis) -> float:
+    """max over (sequence, head) of max|got - ref| / max|ref|, both maxima taken inside that
+    (sequence, head).  Heads differ by orders of magnitude in step size and decay, so one scale
+    for the whole tensor would hide the small ones.  A (sequence, head) whose reference is
+    identically zero must be reproduced as zero."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    err = _head_max(got - ref, head_axis)
+    den = _head_max(ref, head_axis)
+    rel = np.where(den > 0, err / np.where(den > 0, den, 1.0), np.where(err > 0, np.inf, 0.0))
+    return float(rel.max())
+
+
+def elementwise_rel(got, ref):
+    """(max, 99.9th percentile) of |got - ref| / (|ref| + 1e-3 rms(ref)) over all elements."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    r = np.abs(got - ref) / (np.abs(ref) + 1e-3 * rms + 1e-300)
+    return float(r.max()), float(np.percentile(r, 99.9))
+
+
+BF16_EPS = 2.0 ** -8      # unit roundoff of a bf16 store
+FP32_EPS = 2.0 ** -22     # the skip product and the final sum, each rounded once to fp32
+
+
+def check_outputs(cfg: synth.LayerConfig, inp, got_y, got_h, ref, tol_y, tol_h):
+    """y and final state against the oracle at the resolution of one (sequence, head).
+
+    Final state: per (sequence, head) max-norm relative error <= tol_h.
+    y, call without skip term (D is None): y is the readout Ctilde^T h alone; per (sequence, head)
+    max-norm relative error <= tol_y.
+    y, call with a skip term: y is dominated by D x, so the whole-tensor measure alone could not
+    see the readout.  Here every element must satisfy
+        |y - yref| <= tol_y * max_{(b,h)} |Ctilde^T h| + eps_out * |yref|
+    i.e. the readout part is held to tol_y of its own per-head scale, and the only extra slack is
+    the rounding of the stored y (eps_out = 2^-8 for bf16 outputs, 2^-22 for fp32: D x and the
+    final sum are each rounded once).
+    Sequences shorter than one 128-token tile are the one place where the readout of a whole
+    (sequence, head) can nearly cancel (with a single token, y is one 128-term dot product
+    Ctilde . Btilde of streams that are stored in bf16, times Delta x): there the per-head scale
+    is floored by 1/16 of the same readout evaluated on absolute values, the scale a forward
+    error bound is relative to.
+    Also returned (not asserted): the elementwise measure |y - yref| / (|yref| + 1e-3 rms), its
+    maximum and 99.9th percentile (the largest over sequences).  got_y / got_h: torch tensors."""
+    D = inp.get("D")
+    Dv = None if D is None else synth.f64(D)[None, :, None]
+    eps_out = BF16_EPS if cfg.dtype == "bf16" else FP32_EPS
+    floor = None
+    if ref["y"].shape[1] < 128 and "BC" in ref:
+        h0 = inp.get("h0")
+        y_abs, _ = oracle.ssm_recurrence(np.abs(synth.f64(inp["x"])), np.abs(ref["BC"]), synth.f64(inp["dt"]),
+                                         synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), None,
+                                         None if h0 is None else np.abs(synth.f64(h0)), G=cfg.G)
+        floor = np.max(np.abs(y_abs), axis=(1, 3)) / 16.0                   # [B,H]
+    eh = per_head_rel(got_h.double().numpy(), ref["h_final"], 1)
+    y_den = float(np.max(np.abs(ref["y"])))
+    ey, ey_whole, emax, e999 = 0.0, 0.0, 0.0, 0.0
+    for b in range(ref["y"].shape[0]):           # one sequence at a time keeps the temporaries small
+        gy = got_y[b].double().numpy()           # [L,H,P]
+        ry = ref["y"][b]
+        diff = np.abs(gy - ry)
+        ey_whole = max(ey_whole, float(diff.max()) / (y_den if y_den > 0 else 1.0))
+        ssm = ry if Dv is None else ry - Dv * synth.f64(inp["x"][b])
+        scale = np.max(np.abs(ssm), axis=(0, 2))                          # [H]
+        if floor is not None:
+            scale = np.maximum(scale, floor[b])
+        scale = scale[None, :, None]
+        room = diff - (eps_out * np.abs(ry) if Dv is not None else 0.0)
+        rel = np.where(scale > 0, room / np.where(scale > 0, scale, 1.0), np.where(room > 0, np.inf, 0.0))
+        ey = max(ey, float(rel.max()))
+        m, p = elementwise_rel(gy, ry)
+        emax, e999 = max(emax, m), max(e999, p)
+    assert ey_whole <= tol_y, f"y whole-tensor max-rel error {ey_whole:.3e} > {tol_y}"
+    assert ey <= tol_y, f"y per-(sequence, head) error {ey:.3e} > {tol_y}"
+    assert eh <= tol_h, f"h_final per-(sequence, head) error {eh:.3e} > {tol_h}"
+    return dict(err_y=ey, err_y_whole=ey_whole, err_h=eh, err_y_elem_max=emax, err_y_elem_p999=e999)
+
+
 def check_routing(cfg: synth.LayerConfig, inp, idx_gpu, w_gpu, require_all_certified=False):
     """Certified tokens must match exactly; returns (#uncertified tokens, oracle router output).
     r["mismatch"] counts the tokens (necessarily uncertified) whose routing differs from the
@@ -117,11 +202,9 @@ def compare_forward(cfg: synth.LayerConfig, inp, got, tol_y, tol_h, h0=None,
         ref = oracle_forward(cfg, inp, h0=h0, forced_idx=forced_idx, forced_w=forced_w)
     else:
         ref = oracle_forward(cfg, inp, h0=h0)
-    ey = max_rel(got["y"].double().numpy(), ref["y"])
-    eh = max_rel(got["h_final"].double().numpy(), ref["h_final"])
-    assert ey <= tol_y, f"y max-rel error {ey:.3e} > {tol_y}"
-    assert eh <= tol_h, f"h_final max-rel error {eh:.3e} > {tol_h}"
-    return dict(err_y=ey, err_h=eh, ambiguous=n_amb, mismatch=r0["mismatch"], ref=ref)
+    res = check_outputs(cfg, inp, got["y"], got["h_final"], ref, tol_y, tol_h)
+    res.update(ambiguous=n_amb, mismatch=r0["mismatch"], ref=ref)
+    return res
 
 
 def tolerances(cfg: synth.LayerConfig):

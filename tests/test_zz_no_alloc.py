@@ -9,6 +9,8 @@ previous call's contents in the array.  This file is collected last on purpose.
 import pytest
 import torch
 
+import oracle
+
 from paper_2603_06938_b200 import binding as sb
 from paper_2603_06938_b200 import synth
 
@@ -36,20 +38,41 @@ def run_both(cfg, seed):
         assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
         outs.append((BC.float().cpu(), idx.cpu(), wt.cpu()))
     sb.swimba_destroy(h)
-    return outs
+    return inp, outs
 
 
-def test_static_scratch_entry_point_matches_regular_one_twice_in_a_row():
-    # two calls in a row: the second (different size, different routing) finds the first one's
-    # histogram, tile table and slot buffer still in the shared array
-    first = synth.LayerConfig("noalloc_a", "bf16", 2, 700, 128, 4, 64, 128, 1, 8, 2, 128)
-    second = synth.LayerConfig("noalloc_b", "bf16", 1, 333, 128, 4, 64, 128, 1, 8, 2, 128)
+def lc(name, dtype, B, L, E, k):
+    return synth.LayerConfig(name, dtype, B, L, 128, 4, 64, 128, 1, E, k, 128)
+
+
+# two calls in a row per case: the second (different size, different routing) finds the first one's
+# histogram, per-expert lists (and, for k > 2, slot buffer) still in the shared array
+@pytest.mark.parametrize("first,second", [
+    (lc("noalloc_a", "bf16", 2, 700, 8, 2), lc("noalloc_b", "bf16", 1, 333, 8, 2)),    # rows added in place
+    (lc("noalloc_c", "bf16", 2, 500, 8, 3), lc("noalloc_d", "bf16", 1, 777, 8, 3)),    # slot buffer + slot sum
+    (lc("noalloc_e", "fp32", 1, 300, 4, 2), lc("noalloc_f", "fp32", 2, 150, 4, 2)),    # fp32 path: routing scratch only
+], ids=["bf16_k2", "bf16_k3", "fp32"])
+def test_static_scratch_entry_point_matches_regular_one_twice_in_a_row(first, second):
     for cfg, seed in ((first, 51), (second, 52)):
-        (bc_ref, idx_ref, w_ref), (bc, idx, w) = run_both(cfg, seed)
+        inp, ((bc_ref, idx_ref, w_ref), (bc, idx, w)) = run_both(cfg, seed)
         assert torch.equal(idx, idx_ref)
         assert torch.equal(w, w_ref)
         assert hp.max_rel(bc.numpy(), bc_ref.numpy()) <= 1e-2     # same kernels: identical in practice
         assert torch.equal(bc, bc_ref)
+        # and against the CPU oracle: routing under the margin protocol, mixed streams given that routing
+        hp.check_routing(cfg, inp, idx, w)
+        T = cfg.B * cfg.L
+        ref_bc = oracle.mix_topk(synth.f64(inp["u"]).reshape(T, -1), synth.f64(inp["W_e"]),
+                                 idx.numpy().reshape(T, -1), w.double().numpy().reshape(T, -1))
+        tol = 1e-2 if cfg.dtype == "bf16" else 1e-4
+        assert hp.max_rel(bc.double().numpy(), ref_bc) <= tol
+
+
+def test_static_scratch_serves_the_documented_token_count():
+    # 100 000 tokens at E = 8, k = 2 need 4.8 MB of the 8 MiB array
+    cfg = synth.LayerConfig("noalloc_many", "bf16", 1, 100000, 64, 2, 64, 128, 1, 8, 2, 128)
+    inp, ((bc_ref, idx_ref, w_ref), (bc, idx, w)) = run_both(cfg, 54)
+    assert torch.equal(idx, idx_ref) and torch.equal(w, w_ref) and torch.equal(bc, bc_ref)
 
 
 def test_static_scratch_rejects_sizes_beyond_its_capacity():
@@ -57,7 +80,7 @@ def test_static_scratch_rejects_sizes_beyond_its_capacity():
     inp = synth.make_inputs(cfg, seed=53)
     h = hp.create_handle(cfg)
     w, keep = hp.device_weights(inp)
-    T = 1 << 20                                   # needs far more than the 8 MiB array
+    T = 1 << 20                                   # 48 bytes of scratch per token: 48 MiB
     rc = sb.swimba_route_mix_static(h, w, hp.dev(inp["u"]), T, hp.dev(inp["u"]), None, None, check=False)
     assert rc == sb.ERR_WORKSPACE_TOO_SMALL
     assert "static scratch" in sb.swimba_last_error(h)
