@@ -51,6 +51,12 @@ extern "C" {
 #define SWIMBA_DTYPE_FP32 0
 #define SWIMBA_DTYPE_BF16 1
 
+/* Debug aid (no counterpart in the paper): kernels validate every index they read back from
+ * device memory (expert indices, per-expert token lists and their lengths) before using it as an
+ * address.  A bad value is skipped -- nothing is read or written through it -- and
+ * SWIMBA_ERR_DEVICE_BOUNDS is recorded for swimba_status.  Costs one comparison per row. */
+#define SWIMBA_FLAG_CHECK_INDICES 1
+
 #define SWIMBA_MAX_EXPERTS 64
 #define SWIMBA_MAX_TOPK 8
 
@@ -66,7 +72,7 @@ typedef struct {
     int32_t top_k;     /* k, 1..min(E, SWIMBA_MAX_TOPK); k == E is dense routing               */
     int32_t chunk;     /* Q in {64,128,256}: SSD chunk length (results do not depend on it)    */
     int32_t dtype;     /* SWIMBA_DTYPE_*                                                       */
-    int32_t flags;     /* reserved, must be 0                                                  */
+    int32_t flags;     /* 0 or SWIMBA_FLAG_CHECK_INDICES; other bits are reserved              */
 } swimba_config;
 
 typedef struct {
@@ -80,7 +86,12 @@ typedef struct {
 /* Create a layer handle.  Validates the configuration (Section "MoE-parameterized SSM":
  * E experts, k active, one shared transition) against what the kernels support:
  * F % 8 == 0, N % 16 == 0 and N <= 256, P <= 256, (N/16 rounded up to a power of two) * P <= 1024.
- * Uses the current CUDA device.  *out is set only on success. */
+ * Uses the current CUDA device.  *out is set only on success.
+ * Which kernels serve a configuration: with SWIMBA_DTYPE_BF16, P == 64 and N == 128 the SSD runs
+ * on the tensor cores in 128-token tiles; every other shape, and SWIMBA_DTYPE_FP32, evaluates the
+ * recurrence token by token with one block per (sequence, head), which is exact in fp32 but
+ * serial over L (orders of magnitude slower on long sequences).  The expert projection uses the
+ * tensor cores for SWIMBA_DTYPE_BF16 with F >= 64 and S % 32 == 0. */
 int swimba_create(const swimba_config *cfg, swimba_handle **out);
 
 /* Bytes of device workspace swimba_forward / swimba_route_mix / swimba_ssd need for B
@@ -188,6 +199,18 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);
+
+/* Self-test of the failure path (no counterpart in the paper).  Every device-side wait in the
+ * tensor-core kernels is bounded: when it runs out, the kernel records
+ * SWIMBA_ERR_DEVICE_TIMEOUT, makes its later waits return at once and runs to its normal exit.
+ * This call exercises exactly that code on a barrier that nothing signals: one warp waits for
+ * limit_cycles SM cycles (1e3 .. 1e8), gives up, and waits once more.  Afterwards swimba_status
+ * returns SWIMBA_ERR_DEVICE_TIMEOUT (and clears it), and the handle stays usable.
+ *   result_host  HOST array of 3, may be NULL; when given the call synchronises the stream and
+ *                returns {first wait gave up (1/0), second wait gave up (1/0), cycles the second
+ *                wait took}. */
+int swimba_selftest_wait(swimba_handle *h, int64_t limit_cycles, int64_t *result_host,
+                         void *cuda_stream);
 
 /* Number of kernels the most recent forward/route_mix/ssd/decode call on this handle enqueued. */
 int swimba_last_launch_count(const swimba_handle *h);

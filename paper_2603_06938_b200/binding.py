@@ -26,12 +26,13 @@ ERR_DEVICE_TIMEOUT = -7
 ERR_DEVICE_BOUNDS = -8
 DTYPE_FP32 = 0
 DTYPE_BF16 = 1
+FLAG_CHECK_INDICES = 1
 
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
     "swimba_forward_host", "swimba_route_mix_static", "swimba_profile", "swimba_profile_read",
-    "swimba_last_launch_count", "swimba_status", "swimba_last_error",
+    "swimba_selftest_wait", "swimba_last_launch_count", "swimba_status", "swimba_last_error",
     "swimba_destroy",
 ]
 
@@ -96,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.swimba_profile.restype = ctypes.c_int
         L.swimba_profile_read.argtypes = [vp, vp, vp, i32]
         L.swimba_profile_read.restype = ctypes.c_int
+        L.swimba_selftest_wait.argtypes = [vp, i64, vp, vp]
+        L.swimba_selftest_wait.restype = ctypes.c_int
         L.swimba_last_launch_count.argtypes = [vp]
         L.swimba_last_launch_count.restype = ctypes.c_int
         L.swimba_status.argtypes = [vp]
@@ -269,6 +272,16 @@ def swimba_profile_read(h: Handle):
     if n < 0:
         h._raise(n)
     return [(KERNEL_NAMES.get(ids[i], str(ids[i])), float(ms[i])) for i in range(n)]
+
+
+def swimba_selftest_wait(h: Handle, limit_cycles: int, stream=None, check: bool = True):
+    """Runs the bounded-wait self-test; returns (rc, [first gave up, second gave up, cycles])."""
+    res = (ctypes.c_int64 * 3)()
+    rc = lib().swimba_selftest_wait(h.ptr, limit_cycles, ctypes.cast(res, ctypes.c_void_p),
+                                    _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc, [int(v) for v in res]
 
 
 def swimba_last_launch_count(h: Handle) -> int:

@@ -4,6 +4,7 @@
 #include <new>
 
 #include "internal.h"
+#include "tc05.cuh"
 
 using namespace swimba;
 
@@ -15,6 +16,7 @@ struct swimba_handle {
     cudaStream_t last_stream;
     int last_launches;
     Profiler prof;
+    TmapCache tmaps;        // tensor maps encoded so far (same buffers call after call: encoded once)
     // host-buffer entry point: copy streams and events of its batch-slice pipeline
     cudaStream_t s_in, s_out;
     cudaEvent_t ev_start, ev_out, ev_in[8], ev_done[8];
@@ -231,7 +233,7 @@ int route_mix_call(swimba_handle *h, const swimba_weights *w, const void *u, int
         !aligned16(gemm_ws) || !aligned16(topk_idx) || !aligned16(topk_w))
         return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (h->cfg.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
     h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)idx_scratch;
     float *wt = topk_w ? topk_w : (float *)w_scratch;
@@ -257,7 +259,7 @@ int swimba_create(const swimba_config *cfg, swimba_handle **out)
         return SWIMBA_ERR_BAD_CONFIG;
     if (c.chunk != 64 && c.chunk != 128 && c.chunk != 256) return SWIMBA_ERR_BAD_CONFIG;
     if (c.dtype != SWIMBA_DTYPE_FP32 && c.dtype != SWIMBA_DTYPE_BF16) return SWIMBA_ERR_BAD_CONFIG;
-    if (c.flags != 0) return SWIMBA_ERR_BAD_CONFIG;
+    if ((c.flags & ~SWIMBA_FLAG_CHECK_INDICES) != 0) return SWIMBA_ERR_BAD_CONFIG;
     if (c.d_model % 8 != 0 || c.d_state % 16 != 0 || c.d_state > 256 || c.head_dim > 256)
         return SWIMBA_ERR_UNSUPPORTED_SHAPE;
     int ns = 1;
@@ -343,7 +345,7 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
     const FwdLayout l = fwd_layout(h->cfg, B, L, h->sm_count);
     if (!workspace || workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (h->cfg.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
     h->prof.n = 0;
     rc = run_ssd(h, ctx, w, x, BC, dt, h0, B, L, y, h_final, (char *)workspace + l.ssd);
     h->last_stream = ctx.stream;
@@ -374,7 +376,7 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (h->cfg.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
     h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
@@ -410,7 +412,7 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
     if ((rc = set_device(h)) != SWIMBA_OK) return rc;
     const swimba_config &c = h->cfg;
     char *ws = (char *)workspace;
-    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof};
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (h->cfg.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
     h->prof.n = 0;
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
@@ -534,6 +536,31 @@ int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_
             return fail(h, SWIMBA_ERR_CUDA, "cudaEventElapsedTime failed");
     }
     return n;
+}
+
+int swimba_selftest_wait(swimba_handle *h, int64_t limit_cycles, int64_t *result_host, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (limit_cycles < 1000 || limit_cycles > 100000000)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "limit_cycles must lie in [1e3, 1e8]");
+    int rc = set_device(h);
+    if (rc != SWIMBA_OK) return rc;
+    // the three result words live behind the status word in the handle's 64-byte device block
+    long long *out_dev = (long long *)(h->d_status + 4);
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, nullptr};
+    rc = launch_wait_selftest(ctx, (long long)limit_cycles, out_dev);
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    if (rc != SWIMBA_OK) return fail(h, rc, "self-test launch failed");
+    if (result_host) {
+        long long tmp[3];
+        if (cudaStreamSynchronize(ctx.stream) != cudaSuccess ||
+            cudaMemcpy(tmp, out_dev, sizeof(tmp), cudaMemcpyDeviceToHost) != cudaSuccess)
+            return fail(h, SWIMBA_ERR_CUDA, "reading the self-test result failed");
+        for (int i = 0; i < 3; ++i) result_host[i] = (int64_t)tmp[i];
+    }
+    return SWIMBA_OK;
 }
 
 int swimba_last_launch_count(const swimba_handle *h) { return h ? h->last_launches : 0; }

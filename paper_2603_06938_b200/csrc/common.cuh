@@ -9,6 +9,8 @@
 
 namespace swimba {
 
+struct TmapCache;
+
 // Kernel ids reported by the optional per-kernel timing (swimba_profile_read).
 enum Stage {
     STAGE_ROUTER = 1, STAGE_EXPERT_GEMM = 4,
@@ -29,6 +31,8 @@ struct LaunchCtx {
     int *d_status;   // device status word (0 = ok, else a SWIMBA_ERR_* code)
     int launches;    // kernels enqueued through this context
     Profiler *prof;  // optional CUDA-event bracket around every kernel
+    bool check_indices = false;   // SWIMBA_FLAG_CHECK_INDICES: kernels validate indices they read from memory
+    struct TmapCache *tmaps = nullptr;   // the handle's tensor-map cache (may be null)
     void begin(int stage) {
         if (prof && prof->on && prof->n < PROF_MAX) {
             prof->stage[prof->n] = stage;

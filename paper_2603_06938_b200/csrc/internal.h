@@ -48,6 +48,10 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
                      int chunk, int sm_count, void *y, float *h_final, void *workspace,
                      bool scalars_done);
 
+// One warp waiting on a barrier nobody signals, with the given limit (see swimba_selftest_wait).
+// out_dev: three 64-bit words on the device.
+int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev);
+
 // Per-timestep SIMT evaluation of the recurrence (fp32 state in registers).
 int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
                           const float *dt, const float *A, const float *dt_bias, const float *D,

@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(GM_THREADS, 1)
 expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat16 *__restrict__ u,
                    const int *__restrict__ perm, int64_t cap, const float *__restrict__ w_slot,
                    const int *__restrict__ counts, int E, int F, int S, int k, int add_rows,
-                   __nv_bfloat16 *__restrict__ out, int *d_status)
+                   __nv_bfloat16 *__restrict__ out, int *d_status, int check)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     constexpr int STAGES = gm_stages(BN);
@@ -78,7 +78,11 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     {
         int before = 0;
         for (int base = 0; base < E && e < 0; base += 32) {
-            const int c = (base + lane < E) ? counts[base + lane] : 0;
+            int c = (base + lane < E) ? counts[base + lane] : 0;
+            if (check && (c < 0 || c > cap)) {          // a list cannot be longer than its capacity
+                atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
+                c = 0;
+            }
             const int nt = (c + GM_BM - 1) / GM_BM;
             int incl = nt;
 #pragma unroll
@@ -105,6 +109,12 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     for (int r = tid; r < GM_BM; r += GM_THREADS) {
         if (r < nrows) {
             const int entry = perm[row0 + r];
+            if (check && (entry < 0 || entry >= cap * k)) {  // entries are t * k + j with t < cap tokens
+                atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
+                row_src[r] = -1;
+                row_dst[r] = 0;
+                continue;
+            }
             row_src[r] = entry / k;
             row_dst[r] = add_rows ? entry / k : entry;      // token row, or slot row
         } else {
@@ -130,7 +140,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
             const int row = hf * 128 + warp * 32 + lane;
-            wr2[hf] = row < nrows ? w_slot[perm[row0 + row]] : 0.f;
+            wr2[hf] = (row < nrows && row_src[row] >= 0) ? w_slot[perm[row0 + row]] : 0.f;
         }
         int tsrc[16];
 #pragma unroll
@@ -191,7 +201,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
             }
             if (add_rows) {
                 tc::fence_proxy_async_smem();
-                if (row < nrows)
+                if (row < nrows && row_src[row] >= 0)
                     tc::bulk_reduce_add_bf16(out + (int64_t)row_dst[row] * S + n0, srow, BN * 2);
                 tc::bulk_commit_group();
             }
@@ -204,7 +214,7 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
 #pragma unroll 4
             for (int r0 = 0; r0 < 32; r0 += RPI) {
                 const int row = hf * 128 + warp * 32 + r0 + sub;
-                if (row < nrows) {
+                if (row < nrows && row_src[row] >= 0) {
                     const uint4 v = *reinterpret_cast<const uint4 *>(smem + (uint32_t)row * ROW_STRIDE + piece * 16);
                     __nv_bfloat16 *dst = out + (int64_t)row_dst[row] * S + n0 + piece * 8;
                     *reinterpret_cast<uint4 *>(dst) = v;
@@ -335,19 +345,18 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
     const uint64_t dims[3] = {(uint64_t)F, (uint64_t)S, (uint64_t)E};
     const uint64_t strides[2] = {(uint64_t)F * 2, (uint64_t)S * F * 2};
     const uint32_t box[3] = {(uint32_t)GM_BK, (uint32_t)BN, 1};
-    if (!encode_tmap_bf16(&tmap, W_e, 3, dims, strides, box)) return SWIMBA_ERR_CUDA;
+    if (!encode_tmap_bf16_cached(ctx.tmaps, &tmap, W_e, 3, dims, strides, box)) return SWIMBA_ERR_CUDA;
 
     const size_t smem = gemm_smem_bytes(BN);
     dim3 grid((unsigned)max_tiles, (unsigned)(S / BN));
 #define SWIMBA_GEMM_CASE(BNV)                                                                   \
     do {                                                                                        \
         auto kern = expert_gemm_kernel<BNV>;                                                    \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != \
-            cudaSuccess)                                                                        \
-            return SWIMBA_ERR_CUDA;                                                             \
+        if (!ensure_dynamic_smem((const void *)kern, smem)) return SWIMBA_ERR_CUDA;             \
         launch_kernel(kern, grid, dim3(GM_THREADS), smem, ctx.stream, true, tmap,               \
                       (const __nv_bfloat16 *)u, (const int *)perm, (int64_t)T, (const float *)w, \
-                      (const int *)counts, E, F, S, k, add_rows, slots, ctx.d_status);          \
+                      (const int *)counts, E, F, S, k, add_rows, slots, ctx.d_status,           \
+                      ctx.check_indices ? 1 : 0);                                               \
     } while (0)
     ctx.begin(STAGE_EXPERT_GEMM);
     if (BN == 256) SWIMBA_GEMM_CASE(256);

@@ -671,7 +671,7 @@ static int launch_router_stream(LaunchCtx &ctx, const __nv_bfloat16 *u, const __
     const uint64_t dims[2] = {(uint64_t)F, (uint64_t)Ttok};
     const uint64_t strides[1] = {(uint64_t)F * 2};
     const uint32_t box[2] = {(uint32_t)RS_BOX, 16u};
-    if (!encode_tmap_bf16(&tmap, u, 2, dims, strides, box)) return SWIMBA_ERR_CUDA;
+    if (!encode_tmap_bf16_cached(ctx.tmaps, &tmap, u, 2, dims, strides, box)) return SWIMBA_ERR_CUDA;
     const int64_t ntiles = ceil_div64(Ttok, RS_TOK);
     int64_t ctas = (int64_t)sm_count * per_sm;
     if (ctas > ntiles) ctas = ntiles;
@@ -679,8 +679,8 @@ static int launch_router_stream(LaunchCtx &ctx, const __nv_bfloat16 *u, const __
 #define SWIMBA_ROUTER_STREAM_CASE(NTV)                                                          \
     do {                                                                                        \
         auto kern = router_stream_kernel<NTV>;                                                  \
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,             \
-                                 (int)smem) != cudaSuccess)                                     \
+        if (!ensure_dynamic_smem((const void *)kern,             \
+                                 smem))                                     \
             return SWIMBA_ERR_CUDA;                                                             \
         launch_kernel(kern, dim3((unsigned)ctas), dim3(RS_THREADS), smem, ctx.stream, behind_scalars, tmap, \
                       W_r, Ttok, F, E, k, idx, w, counts, perm, cap, (uint4 *)zero_out,         \
@@ -715,8 +715,8 @@ static int launch_router_mma(LaunchCtx &ctx, const __nv_bfloat16 *u, const __nv_
     do {                                                                                        \
         auto kern = router_mma_kernel<NTV>;                                                     \
         if (smem > 32 * 1024 &&  /* static shared memory counts toward the 48 KB default */     \
-            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,             \
-                                 (int)smem) != cudaSuccess)                                     \
+            !ensure_dynamic_smem((const void *)kern,             \
+                                 smem))                                     \
             return SWIMBA_ERR_CUDA;                                                             \
         launch_kernel(kern, dim3((unsigned)(extra + blocks)), dim3(256), smem, ctx.stream, false, \
                       u, W_r, Ttok, F, E, k, idx, w, counts, perm, cap, stage_w, chunk,         \
@@ -776,8 +776,8 @@ static int launch_router_t(LaunchCtx &ctx, const T *u, const T *W_r, int64_t Tto
     do {                                                                                       \
         auto kern = router_topk_kernel<T, EPV, TPWV>;                                          \
         if (smem > 32 * 1024 &&  /* static shared memory counts toward the 48 KB default */    \
-            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
-                                 (int)smem) != cudaSuccess)                                    \
+            !ensure_dynamic_smem((const void *)kern,            \
+                                 smem))                                    \
             return SWIMBA_ERR_CUDA;                                                            \
         int64_t blocks = ceil_div64(Ttok, chunk);                                              \
         const int64_t cap_blocks = (int64_t)sm_count * (smem > 40 * 1024 ? 2 : 4);             \
@@ -816,7 +816,7 @@ template <typename T, typename TO, int RW>
 __global__ void __launch_bounds__(256)
 project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
                         const int32_t *__restrict__ idx, const float *__restrict__ w, int64_t Ttok,
-                        int F, int S, int k, TO *__restrict__ BC)
+                        int F, int S, int k, TO *__restrict__ BC, int E, int check, int *d_status)
 {
     const int lane = threadIdx.x & 31;
     const int nblk = ceil_div(S, RW);
@@ -830,6 +830,11 @@ project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
     for (int j = 0; j < SWIMBA_MAX_TOPK; ++j) {
         ej[j] = (j < k) ? idx[t * k + j] : 0;
         wj[j] = (j < k) ? w[t * k + j] : 0.f;
+        if (check && (ej[j] < 0 || ej[j] >= E)) {      // a bad expert index is skipped, not followed
+            if (lane == 0) atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
+            ej[j] = 0;
+            wj[j] = 0.f;
+        }
     }
     float acc[RW];
 #pragma unroll
@@ -868,7 +873,7 @@ project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
 
 template <typename T, typename TO>
 static int launch_pm(LaunchCtx &ctx, const void *u, const void *W_e, const int32_t *idx,
-                     const float *w, int64_t T_, int F, int S, int k, void *BC)
+                     const float *w, int64_t T_, int F, int S, int E, int k, void *BC)
 {
     constexpr int RW = 16;
     const int warps = 8;
@@ -876,7 +881,7 @@ static int launch_pm(LaunchCtx &ctx, const void *u, const void *W_e, const int32
     dim3 grid((unsigned)ceil_div64(nw, warps)), block(warps * 32);
     ctx.begin(STAGE_PROJECT_SIMT);
     project_mix_simt_kernel<T, TO, RW><<<grid, block, 0, ctx.stream>>>(
-        (const T *)u, (const T *)W_e, idx, w, T_, F, S, k, (TO *)BC);
+        (const T *)u, (const T *)W_e, idx, w, T_, F, S, k, (TO *)BC, E, ctx.check_indices ? 1 : 0, ctx.d_status);
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
@@ -885,11 +890,10 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
                             const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
                             int k, void *BC, bool bc_fp32)
 {
-    (void)E;
     if (T <= 0) return SWIMBA_OK;
-    if (dtype == SWIMBA_DTYPE_FP32) return launch_pm<float, float>(ctx, u, W_e, idx, w, T, F, S, k, BC);
-    if (bc_fp32) return launch_pm<__nv_bfloat16, float>(ctx, u, W_e, idx, w, T, F, S, k, BC);
-    return launch_pm<__nv_bfloat16, __nv_bfloat16>(ctx, u, W_e, idx, w, T, F, S, k, BC);
+    if (dtype == SWIMBA_DTYPE_FP32) return launch_pm<float, float>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
+    if (bc_fp32) return launch_pm<__nv_bfloat16, float>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
+    return launch_pm<__nv_bfloat16, __nv_bfloat16>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
 }
 
 }  // namespace swimba

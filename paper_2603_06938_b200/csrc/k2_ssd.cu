@@ -107,6 +107,73 @@ ssd_scalars_kernel(const ScalarsArgs args)
     ssd_scalars_block(args, blockIdx.x);
 }
 
+// Self-test of the bounded wait every tensor-core kernel here relies on: one warp waits, with the
+// given cycle limit, on a barrier that nothing ever signals.  The wait must give up, record
+// SWIMBA_ERR_DEVICE_TIMEOUT and raise the CTA's abort flag; a second wait must then return at once.
+// out[0] = 1 if the first wait reported failure, out[1] = 1 if the second did, out[2] = cycles the
+// second wait took.
+__global__ void __launch_bounds__(32)
+wait_selftest_kernel(int *d_status, long long limit_cycles, long long *out)
+{
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        abort_flag = 0;
+        tc::fence_mbar_init();
+    }
+    __syncwarp();
+    const bool first = tc::mbar_wait(&bar, 0, &abort_flag, d_status, limit_cycles);
+    __syncwarp();
+    const long long t0 = clock64();
+    const bool second = tc::mbar_wait(&bar, 0, &abort_flag, d_status, limit_cycles);
+    const long long t1 = clock64();
+    if (threadIdx.x == 0) {
+        out[0] = first ? 0 : 1;
+        out[1] = second ? 0 : 1;
+        out[2] = t1 - t0;
+    }
+}
+
+int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev)
+{
+    wait_selftest_kernel<<<1, 32, 0, ctx.stream>>>(ctx.d_status, limit_cycles, out_dev);
+    ctx.launches++;
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
+// w . X for units [UB, UE) of one lane's 16 (row block, 16-byte chunk) units of its half of the
+// head dim: x' = w x with the weight given as a two-term bf16 sum (rounded once).  The unit range
+// is known at compile time, so that all loads are issued before the first use.
+template <int UB, int UE>
+__device__ __forceinline__ void scale_units(const uint8_t *s_x, uint8_t *s_xp, const uint32_t *s_wp, int lane, int hf)
+{
+    uint4 xr[UE - UB];
+    uint32_t wp[UE - UB];
+#pragma unroll
+    for (int un = UB; un < UE; ++un) {
+        const int r = (un >> 2) * 32 + lane;
+        wp[un - UB] = s_wp[r];
+        xr[un - UB] = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(r, 4 * hf + (un & 3)));
+    }
+#pragma unroll
+    for (int un = UB; un < UE; ++un) {
+        const int r = (un >> 2) * 32 + lane;
+        const uint32_t hi_u = __byte_perm(wp[un - UB], 0, 0x1010), lo_u = __byte_perm(wp[un - UB], 0, 0x3232);
+        const __nv_bfloat162 w_hi2 = *reinterpret_cast<const __nv_bfloat162 *>(&hi_u);
+        const __nv_bfloat162 w_lo2 = *reinterpret_cast<const __nv_bfloat162 *>(&lo_u);
+        const uint32_t wv[4] = {xr[un - UB].x, xr[un - UB].y, xr[un - UB].z, xr[un - UB].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
+            const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
+            o[q] = *reinterpret_cast<const uint32_t *>(&pr);
+        }
+        *reinterpret_cast<uint4 *>(s_xp + tc::sw128_offset(r, 4 * hf + (un & 3))) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 template <bool SPLIT>
 __global__ void __launch_bounds__(SSD_THREADS, 1)
 ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
@@ -441,28 +508,16 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             // to row blocks 0 .. 3 instead of 4 each; a foreign row's weight is read from shared
             // memory.
             tc::mbar_wait(&hb->x_full[sx], (j >> 1) & 1, abort_flag, d_status);
-            {
-                const int ubeg = full ? (wq == 0 ? 0 : (wq == 1 ? 6 : (wq == 2 ? 11 : 14))) : 4 * wq;
-                const int uend = full ? (wq == 0 ? 6 : (wq == 1 ? 11 : (wq == 2 ? 14 : 16))) : 4 * wq + 4;
-#pragma unroll 1
-                for (int un = ubeg; un < uend; ++un) {
-                    const int r = (un >> 2) * 32 + lane;
-                    const uint32_t wp = s_wp[r];
-                    const uint32_t hi_u = __byte_perm(wp, 0, 0x1010), lo_u = __byte_perm(wp, 0, 0x3232);
-                    const __nv_bfloat162 w_hi2 = *reinterpret_cast<const __nv_bfloat162 *>(&hi_u);
-                    const __nv_bfloat162 w_lo2 = *reinterpret_cast<const __nv_bfloat162 *>(&lo_u);
-                    const uint32_t off = tc::sw128_offset(r, 4 * hf + (un & 3));
-                    const uint4 xr = *reinterpret_cast<const uint4 *>(s_x + off);
-                    const uint32_t wv[4] = {xr.x, xr.y, xr.z, xr.w};
-                    uint32_t o[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
-                        const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
-                        o[q] = *reinterpret_cast<const uint32_t *>(&pr);
-                    }
-                    *reinterpret_cast<uint4 *>(s_xp + off) = make_uint4(o[0], o[1], o[2], o[3]);
-                }
+            if (full) {
+                if (wq == 0) scale_units<0, 6>(s_x, s_xp, s_wp, lane, hf);
+                else if (wq == 1) scale_units<6, 11>(s_x, s_xp, s_wp, lane, hf);
+                else if (wq == 2) scale_units<11, 14>(s_x, s_xp, s_wp, lane, hf);
+                else scale_units<14, 16>(s_x, s_xp, s_wp, lane, hf);
+            } else {
+                if (wq == 0) scale_units<0, 4>(s_x, s_xp, s_wp, lane, hf);
+                else if (wq == 1) scale_units<4, 8>(s_x, s_xp, s_wp, lane, hf);
+                else if (wq == 2) scale_units<8, 12>(s_x, s_xp, s_wp, lane, hf);
+                else scale_units<12, 16>(s_x, s_xp, s_wp, lane, hf);
             }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&hb->xp_full);
@@ -769,18 +824,18 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         const uint64_t dims[3] = {(uint64_t)S, (uint64_t)L, (uint64_t)B};
         const uint64_t str[2] = {(uint64_t)S * 2, (uint64_t)L * S * 2};
         const uint32_t box[3] = {64, ST, 1};
-        if (!encode_tmap_bf16(&tm_bc, BC, 3, dims, str, box)) return SWIMBA_ERR_CUDA;
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_bc, BC, 3, dims, str, box)) return SWIMBA_ERR_CUDA;
     }
     {
         const uint64_t dims[4] = {(uint64_t)SP, (uint64_t)H, (uint64_t)L, (uint64_t)B};
         const uint64_t str[3] = {(uint64_t)SP * 2, (uint64_t)H * SP * 2, (uint64_t)L * H * SP * 2};
         const uint32_t box[4] = {SP, 1, ST, 1};
-        if (!encode_tmap_bf16(&tm_x, x, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
-        if (!encode_tmap_bf16(&tm_y, y, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_x, x, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_y, y, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
     }
     const size_t smem = ssd_smem_bytes();
-    if (cudaFuncSetAttribute(ssd_tiles_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(ssd_tiles_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (!ensure_dynamic_smem((const void *)ssd_tiles_kernel<false>, smem) ||
+        !ensure_dynamic_smem((const void *)ssd_tiles_kernel<true>, smem))
         return SWIMBA_ERR_CUDA;
 
     const int seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);

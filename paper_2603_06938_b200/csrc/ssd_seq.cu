@@ -2,6 +2,7 @@
 // the channelwise convention; Theorem 1) with the state held in registers: the fp32 path of the
 // forward, and K4, the one-token decode update.
 #include "internal.h"
+#include "tc05.cuh"
 
 namespace swimba {
 
@@ -105,10 +106,7 @@ static int launch_seq_t(LaunchCtx &ctx, const void *x, const void *BC, const flo
     const int NS = seq_ns(N);
     const size_t smem = sizeof(float) * (size_t)(2 * SEQ_TS * N + 2 * SEQ_TS * P + 2 * SEQ_TS);
     auto kern = ssd_sequential_kernel<T, TBC>;
-    if (smem > 48 * 1024 &&
-        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
-        return SWIMBA_ERR_CUDA;
+    if (smem > 48 * 1024 && !ensure_dynamic_smem((const void *)kern, smem)) return SWIMBA_ERR_CUDA;
     ctx.begin(STAGE_SSD_SEQUENTIAL);
     kern<<<B * H, P * NS, smem, ctx.stream>>>((const T *)x, (const TBC *)BC, dt, A, dt_bias, D, h0,
                                              L, H, P, N, G, NS, (T *)y, h_final);

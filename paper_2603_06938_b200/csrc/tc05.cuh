@@ -59,13 +59,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 }
 // Bounded wait on phase `parity`.  `abort_flag` is a CTA-shared int, zero-initialised.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag,
-                                          int *d_status) {
+                                          int *d_status, long long limit_cycles = WAIT_LIMIT_CYCLES) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();             // the SM's own cycle counter: cheap to read
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
             atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_TIMEOUT);
             return false;
@@ -313,6 +313,25 @@ __device__ __forceinline__ void named_bar_sync(int id, int n) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory");
 }
 
+// Re-deal of the CTA's registers between warpgroups (all four warps of a warpgroup execute the
+// same call): the issuing warps give up what they do not need, the compute warpgroups take it.
+template <int N> __device__ __forceinline__ void reg_alloc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_dealloc() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// Packed fp32 pairs (one instruction for two lanes of arithmetic): (a, b) <- (a, b) * (x, y) on the
+// raw 32-bit images of two floats.
+__device__ __forceinline__ void mul2(uint32_t &a, uint32_t &b, float x, float y) {
+    asm("{\n\t.reg .b64 ra, rb, rc;\n\t"
+        "mov.b64 ra, {%0, %1};\n\tmov.b64 rb, {%2, %3};\n\t"
+        "mul.rn.f32x2 rc, ra, rb;\n\tmov.b64 {%0, %1}, rc;\n\t}"
+        : "+r"(a), "+r"(b)
+        : "f"(x), "f"(y));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits)
     return *reinterpret_cast<const uint32_t *>(&v);
@@ -325,5 +344,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // strides[i] is the byte stride of dimension i+1.  Returns false on failure.
 bool encode_tmap_bf16(CUtensorMap *out, const void *base, int rank, const uint64_t *dims,
                       const uint64_t *strides_bytes, const uint32_t *box);
+
+// A handle's memory of the tensor maps it has encoded, keyed by base pointer, extents, strides and
+// box: callers that pass the same buffers call after call (a layer inside a model does) pay for
+// the driver's encoding once.  A small ring; the oldest entry is replaced.
+struct TmapCache {
+    static constexpr int N = 16;
+    struct Entry {
+        const void *base;
+        int rank;
+        uint64_t dims[5], strides[4];
+        uint32_t box[5];
+        alignas(64) CUtensorMap map;
+    };
+    Entry e[N];
+    int used, next;
+};
+// As encode_tmap_bf16, through the cache when one is given.
+bool encode_tmap_bf16_cached(TmapCache *cache, CUtensorMap *out, const void *base, int rank,
+                             const uint64_t *dims, const uint64_t *strides_bytes, const uint32_t *box);
+
+// Raises a kernel's dynamic shared-memory limit to `bytes` on the current device; the runtime call
+// is made only the first time (or when a larger size is asked for).
+bool ensure_dynamic_smem(const void *func, size_t bytes);
 
 }  // namespace swimba

@@ -22,9 +22,30 @@ def dtype_code(cfg: synth.LayerConfig) -> int:
     return sb.DTYPE_FP32 if cfg.dtype == "fp32" else sb.DTYPE_BF16
 
 
-def create_handle(cfg: synth.LayerConfig, chunk=None) -> sb.Handle:
+def create_handle(cfg: synth.LayerConfig, chunk=None, flags: int = 0) -> sb.Handle:
     return sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k,
-                            chunk if chunk is not None else cfg.Q, dtype_code(cfg))
+                            chunk if chunk is not None else cfg.Q, dtype_code(cfg), flags)
+
+
+CANARY_BYTES = 1024
+
+
+def with_canary(shape, dtype, fill):
+    """A device tensor of the given shape followed in memory by CANARY_BYTES of a fixed pattern:
+    returns (tensor view, whole byte buffer).  A kernel that writes past the end of its output or
+    workspace damages the pattern."""
+    n = 1
+    for d in shape:
+        n *= d
+    es = torch.empty((), dtype=dtype).element_size()
+    raw = torch.full((n * es + CANARY_BYTES,), 0xA5, dtype=torch.uint8, device="cuda")
+    view = raw[:n * es].view(dtype).view(*shape)
+    view.fill_(fill)
+    return view, raw
+
+
+def canary_intact(raw) -> bool:
+    return bool((raw[-CANARY_BYTES:] == 0xA5).all())
 
 
 def dev(t):
@@ -36,22 +57,26 @@ def device_weights(inp):
     return sb.make_weights(keep["W_r"], keep["W_e"], keep["A"], keep["dt_bias"], keep["D"]), keep
 
 
-def gpu_forward(cfg: synth.LayerConfig, inp, chunk=None, h0=None, want_topk=True):
-    """Runs swimba_forward; returns host tensors dict(y, h_final, idx, w)."""
-    h = create_handle(cfg, chunk)
+def gpu_forward(cfg: synth.LayerConfig, inp, chunk=None, h0=None, want_topk=True, flags: int = 0):
+    """Runs swimba_forward; returns host tensors dict(y, h_final, idx, w).  Outputs and workspace
+    are followed by canary bytes, which must come back untouched."""
+    h = create_handle(cfg, chunk, flags)
     try:
         B, L = inp["u"].shape[0], inp["u"].shape[1]
         w, keep = device_weights(inp)
         u, x, dt = dev(inp["u"]), dev(inp["x"]), dev(inp["dt"])
         h0d = dev(h0 if h0 is not None else inp.get("h0"))
-        y = torch.full_like(x, float("nan"))
-        hf = torch.full((B, cfg.H, cfg.P, cfg.N), float("nan"), device="cuda")
+        y, y_raw = with_canary(x.shape, x.dtype, float("nan"))
+        hf, hf_raw = with_canary((B, cfg.H, cfg.P, cfg.N), torch.float32, float("nan"))
         idx = torch.full((B, L, cfg.k), -1, dtype=torch.int32, device="cuda") if want_topk else None
         wt = torch.full((B, L, cfg.k), float("nan"), device="cuda") if want_topk else None
-        ws = torch.empty(max(sb.swimba_workspace_bytes(h, B, L), 16), dtype=torch.uint8, device="cuda")
+        nws = max(sb.swimba_workspace_bytes(h, B, L), 16)
+        ws, ws_raw = with_canary((nws,), torch.uint8, 0)
         sb.swimba_forward(h, w, u, x, dt, h0d, B, L, y, hf, idx, wt, ws)
         rc = sb.swimba_status(h)
         assert rc == 0, sb.swimba_last_error(h)
+        assert canary_intact(y_raw) and canary_intact(hf_raw) and canary_intact(ws_raw), \
+            "a kernel wrote past the end of y, h_final or the workspace"
         launches = sb.swimba_last_launch_count(h)
         return dict(y=y.cpu(), h_final=hf.cpu(), idx=None if idx is None else idx.cpu(),
                     w=None if wt is None else wt.cpu(), launches=launches)

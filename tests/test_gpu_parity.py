@@ -286,6 +286,44 @@ def test_decode_steps_match_oracle_and_forward(dtype):
     sb.swimba_destroy(h)
 
 
+# ------------------------------------------------------------------- device-detected errors
+def test_bounded_wait_runs_out_and_the_handle_stays_usable():
+    """The failure path of the tensor-core kernels' waits, exercised on a barrier nothing signals:
+    the wait gives up after its cycle limit, the status word carries DEVICE_TIMEOUT, later waits of
+    the same block return at once, the kernel exits normally, and a forward on the same handle
+    afterwards is correct."""
+    cfg = cfg_of("bf16", L=300)
+    h = hp.create_handle(cfg)
+    rc, (first, second, cycles2) = sb.swimba_selftest_wait(h, 2000000)      # about 1 ms
+    assert rc == 0 and first == 1 and second == 1
+    assert cycles2 < 200000, "the second wait must not spin for the limit again"
+    assert sb.swimba_status(h) == sb.ERR_DEVICE_TIMEOUT
+    assert "device reported error" in sb.swimba_last_error(h)
+    assert sb.swimba_status(h) == 0                      # reading the status cleared it
+    assert sb.swimba_selftest_wait(h, 10, check=False)[0] == sb.ERR_UNSUPPORTED_SHAPE
+    sb.swimba_destroy(h)
+    inp = synth.make_inputs(cfg, seed=71)
+    got = hp.gpu_forward(cfg, inp)
+    hp.compare_forward(cfg, inp, got, *hp.tolerances(cfg))
+
+
+@pytest.mark.parametrize("dtype,k", [("bf16", 2), ("bf16", 3), ("fp32", 2)])
+def test_index_checks_stay_silent_on_valid_calls(dtype, k):
+    # SWIMBA_FLAG_CHECK_INDICES: the kernels validate expert indices and per-expert lists before
+    # following them; on a healthy call nothing fires and the results are unchanged
+    cfg = cfg_of(dtype, L=400, E=8, k=k, N=64 if dtype == "fp32" else 128)
+    inp = synth.make_inputs(cfg, seed=72)
+    plain = hp.gpu_forward(cfg, inp)
+    checked = hp.gpu_forward(cfg, inp, flags=sb.FLAG_CHECK_INDICES)
+    assert torch.equal(plain["idx"], checked["idx"])
+    assert torch.equal(plain["y"].float(), checked["y"].float())
+    assert torch.equal(plain["h_final"], checked["h_final"])
+    hp.compare_forward(cfg, inp, checked, *hp.tolerances(cfg))
+    with pytest.raises(sb.SwimbaError) as e:
+        sb.swimba_create(64, 4, 64, 128, 1, 4, 2, 128, sb.DTYPE_BF16, 2)    # reserved flag bit
+    assert e.value.code == sb.ERR_BAD_CONFIG
+
+
 # ------------------------------------------------------------------- host-detected errors
 def test_host_side_errors_leave_outputs_untouched():
     cfg = cfg_of("bf16", L=64)
