@@ -174,6 +174,31 @@ __device__ __forceinline__ void scale_units(const uint8_t *s_x, uint8_t *s_xp, c
     }
 }
 
+// The same for the four units of the thread's own row (state-only tiles), with the row's weight
+// multiplied by `f` first: w' = w f is split again into two bf16 terms.
+__device__ __forceinline__ void scale_own_row(const uint8_t *s_x, uint8_t *s_xp, uint32_t wp, float f, int i, int hf)
+{
+    const float w = (__uint_as_float(wp << 16) + __uint_as_float(wp & 0xffff0000u)) * f;
+    const __nv_bfloat16 w_hi = __float2bfloat16_rn(w);
+    const __nv_bfloat16 w_lo = __float2bfloat16_rn(w - __bfloat162float(w_hi));
+    const __nv_bfloat162 w_hi2 = __halves2bfloat162(w_hi, w_hi), w_lo2 = __halves2bfloat162(w_lo, w_lo);
+    uint4 xr[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) xr[c] = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(i, 4 * hf + c));
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t wv[4] = {xr[c].x, xr[c].y, xr[c].z, xr[c].w};
+        uint32_t o[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
+            const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
+            o[q] = *reinterpret_cast<const uint32_t *>(&pr);
+        }
+        *reinterpret_cast<uint4 *>(s_xp + tc::sw128_offset(i, 4 * hf + c)) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+}
+
 template <bool SPLIT>
 __global__ void __launch_bounds__(SSD_THREADS, 1)
 ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
@@ -392,9 +417,9 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     tc::tc_fence_after();
                     if (leader) {
 #pragma unroll
-                        for (int kk = 0; kk < 8; ++kk)
+                        for (int kk = 0; kk < 8; ++kk)     // (the tiles of a state-only run accumulate)
                             tc::mma_ss(tmem_u + TM_DH, tc::smem_desc_advance(dBt, kk * 2048),
-                                       tc::smem_desc_advance(dXp, kk * 2048), id_hn, kk > 0);
+                                       tc::smem_desc_advance(dXp, kk * 2048), id_hn, (kk > 0) || (!full && j > 0));
                         for (int q = 0; q < nh; ++q) tc::mma_commit(&bars->hd[q].dh_full);
                         tc::mma_commit(&bars->cb_empty);     // C and B tiles are no longer needed
                     }
@@ -485,6 +510,18 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         float seg_l2 = 0.f;      // log2 of the product of a_t over the tiles done so far
         const float *l2p = prm.l2 + ((int64_t)b * H + h) * prm.Lpad + t_begin;
         float l2_next = l2p[i];
+        // A run of state-only tiles (a whole segment in the state-only pass, the lead of a split
+        // launch) is one long contraction: with every token weighted by its decay up to the END OF
+        // THE RUN (exponent <= 0), Btilde^T (w . X) accumulates over all tiles of the run in tensor
+        // memory and the state is touched once, at the run's last tile:
+        //   H_end = 2^(sum of l_last over the run) H_in + sum_tiles Btilde^T (w' . X).
+        const int run_end = kfull ? n_pre : ntiles;
+        float run_total = 0.f;   // log2 decay over the whole run
+        {
+            const TileScalars *rec0 = prm.rec + ((int64_t)b * H + h) * (prm.Lpad / ST) + t_begin / ST;
+            for (int jr = 0; jr < run_end; ++jr) run_total += rec0[jr].ends[3];
+        }
+        float run_done = 0.f;    // ... over the tiles of the run up to and including the current one
 
         for (int j = 0; j < ntiles; ++j) {
             const int sx = j & 1;
@@ -514,10 +551,11 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 else if (wq == 2) scale_units<11, 14>(s_x, s_xp, s_wp, lane, hf);
                 else scale_units<14, 16>(s_x, s_xp, s_wp, lane, hf);
             } else {
-                if (wq == 0) scale_units<0, 4>(s_x, s_xp, s_wp, lane, hf);
-                else if (wq == 1) scale_units<4, 8>(s_x, s_xp, s_wp, lane, hf);
-                else if (wq == 2) scale_units<8, 12>(s_x, s_xp, s_wp, lane, hf);
-                else scale_units<12, 16>(s_x, s_xp, s_wp, lane, hf);
+                // a tile of a run: the X' slab is free once the previous tile's product has read it
+                run_done += l2_last;
+                const uint32_t wp = s_wp[i];
+                if (j > 0) tc::mbar_wait(&hb->dh_full, (j - 1) & 1, abort_flag, d_status);
+                scale_own_row(s_x, s_xp, wp, tc::ex2_approx(run_total - run_done), i, hf);
             }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&hb->xp_full);
@@ -600,11 +638,13 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 tc::mbar_arrive(&hb->m_full);
             }
 
-            // ---- state: H = exp(l_last) H + dH  (thread owns state index n = i, 32 channels)
+            // ---- state: H = exp(l_last) H + dH  (thread owns state index n = i, 32 channels); inside a
+            // run of state-only tiles only at its last tile, with the decay of the whole run
+            seg_l2 += l2_last;
+            if (full || j == run_end - 1) {
             tc::mbar_wait(&hb->dh_full, j & 1, abort_flag, d_status);
             tc::tc_fence_after();
-            const float dec = tc::ex2_approx(l2_last);
-            seg_l2 += l2_last;
+            const float dec = tc::ex2_approx(full ? l2_last : run_total);
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh) {
                 uint32_t dh[16];
@@ -629,6 +669,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 tc::fence_proxy_async_smem();
                 tc::tc_fence_before();
                 tc::mbar_arrive(&hb->h_ready);
+            }
             }
             if (full) {
                 // ---- epilogue: y_i = Y_i + D x_i, staged in shared memory for the TMA store
