@@ -140,6 +140,33 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
  * positive.  The result does not depend on the segmentation beyond rounding. */
 int32_t swimba_ssd_segments(const swimba_handle *h, int32_t B, int32_t L);
 
+/* The general form of the layer, with expert-specific SSM inputs (the state equation of Section
+ * "MoE-parameterized SSM" as printed: h_t = A h_{t-1} + sum_{e in K_t} pi_{t,e} B_t^(e) X_t^(e)^T,
+ * Y_t = (sum_{e in K_t} pi_{t,e} C_t^(e))^T h_t).  The caller's experts produce X^(e) themselves (in
+ * the paper they are in-projection layers), so the work is cut in two calls around that step:
+ *
+ * swimba_route_project_slots: router + projection WITHOUT the mix.
+ *   u [T,F] dtype -> BC_slots [T,k,S] dtype: row (t, j) = pi_{t,e} [B_t^(e) ; C_t^(e)] for the j-th
+ *   active expert e = topk_idx[t,j] (weight already applied), topk_idx [T,k], topk_w [T,k] (may be
+ *   NULL).  Workspace as for swimba_route_mix.
+ *
+ * swimba_ssd_slots: the single recurrence on those streams.
+ *   x_slots  [k,B,L,H,P] dtype  slot j holds, for every token, X^(e) of its j-th active expert
+ *   BC_slots [B*L,k,S]   dtype  as produced above
+ *   dt, h0, y, h_final as in swimba_forward; there is no skip term (w->D is not read).
+ * The injection is linear in (B^(e), X^(e)), so the call evaluates k ordinary chunked recurrences
+ * (one per slot, each with its own injection stream and the readout stream mixed over all slots)
+ * and adds them; cost is k times swimba_ssd plus two streaming passes per extra slot, and the state
+ * stays [B,H,P,N] whatever E is (Theorem 1).  Workspace: swimba_ssd_slots_workspace_bytes. */
+int swimba_route_project_slots(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
+                               void *BC_slots, int32_t *topk_idx, float *topk_w, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream);
+size_t swimba_ssd_slots_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+int swimba_ssd_slots(swimba_handle *h, const swimba_weights *w, const void *x_slots,
+                     const void *BC_slots, const float *dt, const float *h0, int32_t B, int32_t L,
+                     void *y, float *h_final, void *workspace, size_t workspace_bytes,
+                     void *cuda_stream);
+
 /* Bytes of device workspace swimba_decode_step needs for B sequences. */
 size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B);
 
@@ -193,9 +220,9 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..11 (1 router + grouping by
+ * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..13 (1 router + grouping by
  * expert (for fewer than about 28000 tokens the launch also computes the SSD step sizes), 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
- * tile kernel, 10 segment scan, 11 SSD step sizes and decays; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
+ * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);

@@ -30,6 +30,7 @@ FLAG_CHECK_INDICES = 1
 
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
+    "swimba_route_project_slots", "swimba_ssd_slots_workspace_bytes", "swimba_ssd_slots",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
     "swimba_forward_host", "swimba_route_mix_static", "swimba_profile", "swimba_profile_read",
     "swimba_selftest_wait", "swimba_last_launch_count", "swimba_status", "swimba_last_error",
@@ -84,6 +85,14 @@ def lib() -> ctypes.CDLL:
         L.swimba_ssd.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32, vp,
                                  vp, vp, sz, vp]
         L.swimba_ssd.restype = ctypes.c_int
+        L.swimba_route_project_slots.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, i64, vp, vp, vp,
+                                                 vp, sz, vp]
+        L.swimba_route_project_slots.restype = ctypes.c_int
+        L.swimba_ssd_slots_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_ssd_slots_workspace_bytes.restype = sz
+        L.swimba_ssd_slots.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32, vp,
+                                       vp, vp, sz, vp]
+        L.swimba_ssd_slots.restype = ctypes.c_int
         L.swimba_decode_step.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32,
                                          vp, vp, vp, vp, sz, vp]
         L.swimba_decode_step.restype = ctypes.c_int
@@ -218,6 +227,30 @@ def swimba_route_mix_static(h: Handle, w: swimba_weights, u, T: int, BC, topk_id
     return rc
 
 
+def swimba_route_project_slots(h: Handle, w: swimba_weights, u, T: int, BC_slots, topk_idx, topk_w,
+                               workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_route_project_slots(h.ptr, ctypes.byref(w), _ptr(u), T, _ptr(BC_slots),
+                                          _ptr(topk_idx), _ptr(topk_w), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_ssd_slots_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_ssd_slots_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_ssd_slots(h: Handle, w: swimba_weights, x_slots, BC_slots, dt, h0, B: int, L: int, y,
+                     h_final, workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_ssd_slots(h.ptr, ctypes.byref(w), _ptr(x_slots), _ptr(BC_slots), _ptr(dt),
+                                _ptr(h0), B, L, _ptr(y), _ptr(h_final), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
 def swimba_ssd(h: Handle, w: swimba_weights, x, BC, dt, h0, B: int, L: int, y, h_final, workspace,
                stream=None, check: bool = True) -> int:
     wp, wb = _ws(workspace)
@@ -254,7 +287,8 @@ def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B
 
 KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
-                9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars"}
+                9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars", 12: "slot_streams",
+                13: "slot_sum"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

@@ -327,6 +327,118 @@ int swimba_route_mix(swimba_handle *h, const swimba_weights *w, const void *u, i
     return route_mix_call(h, w, u, T, BC, topk_idx, topk_w, ws + l.idx, ws + l.w, ws + l.gemm, cuda_stream);
 }
 
+int swimba_route_project_slots(swimba_handle *h, const swimba_weights *w, const void *u, int64_t T,
+                               void *BC_slots, int32_t *topk_idx, float *topk_w, void *workspace,
+                               size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (T < 0 || T * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "T out of range (T * top_k must stay below 2^31)");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !BC_slots || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, BC_slots or workspace is NULL");
+    if (!aligned16(u) || !aligned16(BC_slots) || !aligned16(workspace) || !aligned16(topk_idx) || !aligned16(topk_w))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const swimba_config &c = h->cfg;
+    const FwdLayout l = fwd_layout(c, 1, (int)T, h->sm_count);
+    if (workspace_bytes < l.ssd) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    const int S = 2 * c.n_groups * c.d_state;
+    const void *Wr = w->W_router ? w->W_router : w->W_expert;
+    const bool tensor = use_tensor_k1(c);
+    int *counts = nullptr, *perm = nullptr;
+    if (tensor) {
+        counts = expert_gemm_counts(ws + l.gemm);
+        perm = expert_gemm_perm(ws + l.gemm);
+        if (cudaMemsetAsync(counts, 0, sizeof(int) * SWIMBA_MAX_EXPERTS, ctx.stream) != cudaSuccess)
+            return fail(h, SWIMBA_ERR_CUDA, "clearing the expert histogram failed");
+    }
+    rc = launch_router(ctx, c.dtype, u, Wr, T, c.d_model, c.n_experts, c.top_k, idx, wt, counts, perm, T,
+                       h->sm_count, nullptr, S * 2, ScalarsArgs{});
+    if (rc != SWIMBA_OK) return fail(h, rc, "router launch failed");
+    if (tensor)
+        rc = launch_expert_gemm(ctx, u, w->W_expert, wt, T, c.d_model, S, c.n_experts, c.top_k, h->sm_count,
+                                nullptr, ws + l.gemm, BC_slots);
+    else
+        rc = launch_project_slots_simt(ctx, c.dtype, u, w->W_expert, idx, wt, T, c.d_model, S, c.n_experts,
+                                       c.top_k, BC_slots);
+    if (rc != SWIMBA_OK) fail(h, rc, "projection launch failed");
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+size_t swimba_ssd_slots_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    const swimba_config &c = h->cfg;
+    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const size_t S = 2u * c.n_groups * c.d_state, HP = (size_t)c.n_heads * c.head_dim;
+    // [forward workspace | BC of one slot | y of one slot | end state of one slot]
+    return fwd_layout(c, B, L, h->sm_count).total + align_up(T * S * es) + align_up(T * HP * es) +
+           align_up((size_t)B * HP * c.d_state * sizeof(float));
+}
+
+int swimba_ssd_slots(swimba_handle *h, const swimba_weights *w, const void *x_slots, const void *BC_slots,
+                     const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
+                     void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
+    int rc = check_weights(h, w, false);
+    if (rc != SWIMBA_OK) return rc;
+    if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!x_slots || !BC_slots || !y || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "x_slots, BC_slots, y or workspace is NULL");
+    if (!aligned16(x_slots) || !aligned16(BC_slots) || !aligned16(y) || !aligned16(dt) || !aligned16(h0) ||
+        !aligned16(h_final) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    if (workspace_bytes < swimba_ssd_slots_workspace_bytes(h, B, L))
+        return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    const swimba_config &c = h->cfg;
+    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const int S = 2 * c.n_groups * c.d_state, k = c.top_k;
+    const size_t HP = (size_t)c.n_heads * c.head_dim;
+    const FwdLayout l = fwd_layout(c, B, L, h->sm_count);
+    char *ws = (char *)workspace;
+    char *bcj = ws + l.total;
+    char *ytmp = bcj + align_up(T * S * es);
+    float *htmp = (float *)(ytmp + align_up(T * HP * es));
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    // The injection is linear in (B^(e), X^(e)): the layer is the sum over the k slots of one
+    // ordinary evaluation each, with slot j's own injection stream and input and the readout stream
+    // mixed over all slots; the initial state enters through slot 0 only.  No skip term: the
+    // paper's output equation has none, and with expert-specific inputs there is no single x.
+    swimba_weights wj = *w;
+    wj.D = nullptr;
+    for (int j = 0; j < k && rc == SWIMBA_OK; ++j) {
+        rc = launch_assemble_slot_streams(ctx, c.dtype, BC_slots, (int64_t)T, S, k, j, bcj);
+        if (rc != SWIMBA_OK) { fail(h, rc, "slot stream launch failed"); break; }
+        const char *xj = (const char *)x_slots + (size_t)j * T * HP * es;
+        rc = run_ssd(h, ctx, &wj, xj, bcj, dt, j == 0 ? h0 : nullptr, B, L, j == 0 ? y : (void *)ytmp,
+                     h_final ? (j == 0 ? h_final : htmp) : nullptr, ws + l.ssd);
+        if (rc != SWIMBA_OK) break;
+        if (j > 0) {
+            rc = launch_accumulate(ctx, c.dtype, y, ytmp, (int64_t)(T * HP), h_final, h_final ? htmp : nullptr,
+                                   (int64_t)B * HP * c.d_state);
+            if (rc != SWIMBA_OK) fail(h, rc, "slot sum launch failed");
+        }
+    }
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const void *BC,
                const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
                void *workspace, size_t workspace_bytes, void *cuda_stream)

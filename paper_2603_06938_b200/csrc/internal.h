@@ -24,14 +24,29 @@ bool expert_gemm_supported(int F, int S);
 bool expert_gemm_adds_rows(int k);   // true: BC must be zero before launch_expert_gemm runs
 int *expert_gemm_counts(void *workspace);
 int *expert_gemm_perm(void *workspace);
+// slots_out (may be NULL): [T*k, S] bf16; when given, the projection of (token t, slot j), scaled by
+// its router weight, is stored in row t*k + j and nothing is mixed (BC is not touched).
 int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const float *w, int64_t T,
-                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace);
+                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace,
+                       void *slots_out = nullptr);
 
 // K1b (SIMT): project the k selected experts and mix.  BC is written in `dtype`, or as float
 // per slot-sum when bc_fp32 is set.
 int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void *W_e,
                             const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
                             int k, void *BC, bool bc_fp32);
+// The same without the mix: row t*k + j of slots_out (dtype) = w[t,j] * W_e[idx[t,j]] u_t.
+int launch_project_slots_simt(LaunchCtx &ctx, int dtype, const void *u, const void *W_e,
+                              const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
+                              int k, void *slots_out);
+
+// General injection (expert-specific SSM inputs) helpers, all dtype-generic streaming kernels:
+//   assemble: BCj[t, :] = [ slots[t*k + j, 0:GN] | sum_j' slots[t*k + j', GN:2GN] ]
+//   accumulate: y += y_add (dtype, fp32 sum), h += h_add (float); either pair may be NULL
+int launch_assemble_slot_streams(LaunchCtx &ctx, int dtype, const void *slots, int64_t T, int S, int k,
+                                 int j, void *BCj);
+int launch_accumulate(LaunchCtx &ctx, int dtype, void *y, const void *y_add, int64_t ny, float *h,
+                      const float *h_add, int64_t nh);
 
 // K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
 bool ssd_tiles_supported(int dtype, int P, int N);

@@ -324,14 +324,17 @@ bool expert_gemm_supported(int F, int S)
 }
 
 int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const float *w, int64_t T,
-                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace)
+                       int F, int S, int E, int k, int sm_count, void *BC, void *workspace,
+                       void *slots_out)
 {
     if (T <= 0) return SWIMBA_OK;
     const int max_tiles = (int)ceil_div64(T * k, GM_BM) + E;
     int *counts = expert_gemm_counts(workspace);
     int *perm = expert_gemm_perm(workspace);
-    const int add_rows = expert_gemm_adds_rows(k) ? 1 : 0;
-    __nv_bfloat16 *slots = (k > 1 && !add_rows)
+    // slots_out given: every (token, slot) projection goes to its own row there and nothing is mixed
+    const int add_rows = (!slots_out && expert_gemm_adds_rows(k)) ? 1 : 0;
+    __nv_bfloat16 *slots = slots_out ? (__nv_bfloat16 *)slots_out
+        : (k > 1 && !add_rows)
         ? (__nv_bfloat16 *)((char *)perm + gemm_ws_up((size_t)E * T * sizeof(int)))
         : (__nv_bfloat16 *)BC;
 
@@ -365,7 +368,7 @@ int launch_expert_gemm(LaunchCtx &ctx, const void *u, const void *W_e, const flo
     else SWIMBA_GEMM_CASE(32);
 #undef SWIMBA_GEMM_CASE
     ctx.end();
-    if (k > 1 && !add_rows) {
+    if (k > 1 && !add_rows && !slots_out) {
         const int64_t nvec = T * (S / 8);
         int64_t blocks = ceil_div64(nvec, 256);
         if (blocks > (int64_t)sm_count * 16) blocks = (int64_t)sm_count * 16;

@@ -816,8 +816,11 @@ template <typename T, typename TO, int RW>
 __global__ void __launch_bounds__(256)
 project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
                         const int32_t *__restrict__ idx, const float *__restrict__ w, int64_t Ttok,
-                        int F, int S, int k, TO *__restrict__ BC, int E, int check, int *d_status)
+                        int F, int S, int k, TO *__restrict__ BC, int E, int check, int *d_status,
+                        int kst, int joff)
 {
+    // (kst, joff): the k experts of token t are entries t*kst + joff .. + k - 1 of idx / w and the
+    // output row is t*(kst/k) + joff/k ... used with k = 1, joff = j to write unmixed slots
     const int lane = threadIdx.x & 31;
     const int nblk = ceil_div(S, RW);
     const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -828,8 +831,8 @@ project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
     float wj[SWIMBA_MAX_TOPK];
 #pragma unroll
     for (int j = 0; j < SWIMBA_MAX_TOPK; ++j) {
-        ej[j] = (j < k) ? idx[t * k + j] : 0;
-        wj[j] = (j < k) ? w[t * k + j] : 0.f;
+        ej[j] = (j < k) ? idx[t * kst + joff + j] : 0;
+        wj[j] = (j < k) ? w[t * kst + joff + j] : 0.f;
         if (check && (ej[j] < 0 || ej[j] >= E)) {      // a bad expert index is skipped, not followed
             if (lane == 0) atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
             ej[j] = 0;
@@ -868,20 +871,24 @@ project_mix_simt_kernel(const T *__restrict__ u, const T *__restrict__ W_e,
         const float s = warp_sum(acc[r]);
         if (lane == r) mine = s;
     }
-    if (lane < RW && r0 + lane < S) BC[t * S + r0 + lane] = from_f32<TO>(mine);
+    const int64_t orow = (kst == k) ? t : t * kst + joff;
+    if (lane < RW && r0 + lane < S) BC[orow * S + r0 + lane] = from_f32<TO>(mine);
 }
 
 template <typename T, typename TO>
 static int launch_pm(LaunchCtx &ctx, const void *u, const void *W_e, const int32_t *idx,
-                     const float *w, int64_t T_, int F, int S, int E, int k, void *BC)
+                     const float *w, int64_t T_, int F, int S, int E, int k, void *BC, int kst = -1,
+                     int joff = 0)
 {
+    if (kst < 0) kst = k;
     constexpr int RW = 16;
     const int warps = 8;
     const int64_t nw = T_ * ceil_div(S, RW);
     dim3 grid((unsigned)ceil_div64(nw, warps)), block(warps * 32);
     ctx.begin(STAGE_PROJECT_SIMT);
     project_mix_simt_kernel<T, TO, RW><<<grid, block, 0, ctx.stream>>>(
-        (const T *)u, (const T *)W_e, idx, w, T_, F, S, k, (TO *)BC, E, ctx.check_indices ? 1 : 0, ctx.d_status);
+        (const T *)u, (const T *)W_e, idx, w, T_, F, S, k, (TO *)BC, E, ctx.check_indices ? 1 : 0, ctx.d_status,
+        kst, joff);
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
@@ -894,6 +901,88 @@ int launch_project_mix_simt(LaunchCtx &ctx, int dtype, const void *u, const void
     if (dtype == SWIMBA_DTYPE_FP32) return launch_pm<float, float>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
     if (bc_fp32) return launch_pm<__nv_bfloat16, float>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
     return launch_pm<__nv_bfloat16, __nv_bfloat16>(ctx, u, W_e, idx, w, T, F, S, E, k, BC);
+}
+
+int launch_project_slots_simt(LaunchCtx &ctx, int dtype, const void *u, const void *W_e,
+                              const int32_t *idx, const float *w, int64_t T, int F, int S, int E,
+                              int k, void *slots_out)
+{
+    if (T <= 0) return SWIMBA_OK;
+    for (int j = 0; j < k; ++j) {
+        const int rc = dtype == SWIMBA_DTYPE_FP32
+            ? launch_pm<float, float>(ctx, u, W_e, idx, w, T, F, S, E, 1, slots_out, k, j)
+            : launch_pm<__nv_bfloat16, __nv_bfloat16>(ctx, u, W_e, idx, w, T, F, S, E, 1, slots_out, k, j);
+        if (rc != SWIMBA_OK) return rc;
+    }
+    return SWIMBA_OK;
+}
+
+// BCj[t, :] = [ slots[t*k + j, 0:half] | sum_j' slots[t*k + j', half:S] ]: slot j's own injection
+// stream beside the readout stream mixed over all slots (the slots already carry their weights).
+template <typename T>
+__global__ void __launch_bounds__(256)
+assemble_slot_streams_kernel(const T *__restrict__ slots, int64_t Ttok, int S, int k, int j, T *__restrict__ BCj)
+{
+    const int half = S >> 1;
+    const int64_t n = Ttok * S;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t t = i / S;
+        const int c = (int)(i % S);
+        float v;
+        if (c < half) {
+            v = to_f32<T>(slots[(t * k + j) * S + c]);
+        } else {
+            v = 0.f;
+            for (int q = 0; q < k; ++q) v += to_f32<T>(slots[(t * k + q) * S + c]);
+        }
+        BCj[i] = from_f32<T>(v);
+    }
+}
+
+int launch_assemble_slot_streams(LaunchCtx &ctx, int dtype, const void *slots, int64_t T, int S, int k,
+                                 int j, void *BCj)
+{
+    if (T <= 0) return SWIMBA_OK;
+    int64_t blocks = ceil_div64(T * S, 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    ctx.begin(STAGE_SLOT_STREAMS);
+    if (dtype == SWIMBA_DTYPE_FP32)
+        assemble_slot_streams_kernel<float><<<(unsigned)blocks, 256, 0, ctx.stream>>>((const float *)slots, T, S, k, j, (float *)BCj);
+    else
+        assemble_slot_streams_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, ctx.stream>>>(
+            (const __nv_bfloat16 *)slots, T, S, k, j, (__nv_bfloat16 *)BCj);
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
+// y += y_add (sum in fp32, stored in T), h += h_add
+template <typename T>
+__global__ void __launch_bounds__(256)
+accumulate_kernel(T *__restrict__ y, const T *__restrict__ y_add, int64_t ny, float *__restrict__ h,
+                  const float *__restrict__ h_add, int64_t nh)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x, i0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (y && y_add)
+        for (int64_t i = i0; i < ny; i += stride) y[i] = from_f32<T>(to_f32<T>(y[i]) + to_f32<T>(y_add[i]));
+    if (h && h_add)
+        for (int64_t i = i0; i < nh; i += stride) h[i] += h_add[i];
+}
+
+int launch_accumulate(LaunchCtx &ctx, int dtype, void *y, const void *y_add, int64_t ny, float *h,
+                      const float *h_add, int64_t nh)
+{
+    const int64_t n = ny > nh ? ny : nh;
+    if (n <= 0) return SWIMBA_OK;
+    int64_t blocks = ceil_div64(n, 256);
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    ctx.begin(STAGE_SLOT_SUM);
+    if (dtype == SWIMBA_DTYPE_FP32)
+        accumulate_kernel<float><<<(unsigned)blocks, 256, 0, ctx.stream>>>((float *)y, (const float *)y_add, ny, h, h_add, nh);
+    else
+        accumulate_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, ctx.stream>>>(
+            (__nv_bfloat16 *)y, (const __nv_bfloat16 *)y_add, ny, h, h_add, nh);
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
 }  // namespace swimba
