@@ -288,7 +288,7 @@ def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B
 KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
                 9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars", 12: "slot_streams",
-                13: "slot_sum"}
+                13: "slot_sum", 14: "project_small"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

@@ -529,8 +529,18 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
     int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
     float *wt = topk_w ? topk_w : (float *)(ws + l.w);
     void *BC = ws + l.bc;
-    const bool tensor = use_tensor_k1(c);   // bf16 streams from the grouped GEMM, else fp32 from SIMT
-    rc = run_route_mix(h, ctx, w, u, B, BC, !tensor, idx, wt, tensor ? ws + l.gemm : nullptr);
+    const int S = 2 * c.n_groups * c.d_state;
+    // a handful of tokens: the two-kernel front end (fp32 streams); else bf16 streams from the
+    // grouped GEMM, or fp32 from the SIMT projection
+    const bool small = front_small_supported(c.dtype, B, c.d_model, S, c.n_experts, c.top_k);
+    const bool tensor = !small && use_tensor_k1(c);
+    if (small) {
+        rc = launch_front_small(ctx, u, w->W_router ? w->W_router : w->W_expert, w->W_expert, B, c.d_model, S,
+                                c.n_experts, c.top_k, idx, wt, (float *)BC);
+        if (rc != SWIMBA_OK) fail(h, rc, "routing / projection launch failed");
+    } else {
+        rc = run_route_mix(h, ctx, w, u, B, BC, !tensor, idx, wt, tensor ? ws + l.gemm : nullptr);
+    }
     if (rc == SWIMBA_OK) {
         rc = launch_decode_update(ctx, c.dtype, x, BC, !tensor, dt, w->A, w->dt_bias, w->D, state, B,
                                   c.n_heads, c.head_dim, c.d_state, c.n_groups, h->sm_count, y);

@@ -16,7 +16,7 @@ enum Stage {
     STAGE_ROUTER = 1, STAGE_EXPERT_GEMM = 4,
     STAGE_MIX_SLOTS = 5, STAGE_PROJECT_SIMT = 6, STAGE_SSD_SEQUENTIAL = 7, STAGE_DECODE_UPDATE = 8,
     STAGE_SSD_TILES = 9, STAGE_SEGMENT_SCAN = 10, STAGE_SSD_SCALARS = 11, STAGE_SLOT_STREAMS = 12,
-    STAGE_SLOT_SUM = 13,
+    STAGE_SLOT_SUM = 13, STAGE_PROJECT_SMALL = 14,
 };
 
 constexpr int PROF_MAX = 64;

@@ -48,6 +48,12 @@ int launch_assemble_slot_streams(LaunchCtx &ctx, int dtype, const void *slots, i
 int launch_accumulate(LaunchCtx &ctx, int dtype, void *y, const void *y_add, int64_t ny, float *h,
                       const float *h_add, int64_t nh);
 
+// K1 for at most a few hundred tokens (decode): two short kernels, no lists in global memory.
+// idx [T,k], w [T,k] and the fp32 mixed streams BC [T,S] are written.
+bool front_small_supported(int dtype, int64_t T, int F, int S, int E, int k);
+int launch_front_small(LaunchCtx &ctx, const void *u, const void *W_r, const void *W_e, int64_t T, int F,
+                       int S, int E, int k, int32_t *idx, float *w, float *BC);
+
 // K2/K3 (tensor cores): tiled SSD with the carried state kept on chip; bf16, P == 64, N == 128.
 bool ssd_tiles_supported(int dtype, int P, int N);
 size_t ssd_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);

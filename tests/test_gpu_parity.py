@@ -250,9 +250,12 @@ def test_route_mix_and_ssd_entry_points():
 
 
 # -------------------------------------------------------------------------------- decode
-@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-def test_decode_steps_match_oracle_and_forward(dtype):
-    cfg = cfg_of(dtype, B=5, L=40, H=4, P=64, N=128 if dtype == "bf16" else 32, E=8, k=2, F=128,
+# F = 128: grouped GEMM (bf16) / SIMT (fp32) front end; F a multiple of 256 with k <= 2 and E <= 16:
+# the two-kernel front end for a handful of tokens (ragged token tiles, k = 1, E = 16, several passes)
+@pytest.mark.parametrize("dtype,F,k,B,E", [("fp32", 128, 2, 5, 8), ("bf16", 128, 2, 5, 8), ("bf16", 256, 2, 5, 8),
+                                           ("bf16", 512, 1, 37, 16), ("bf16", 256, 2, 150, 4)])
+def test_decode_steps_match_oracle_and_forward(dtype, F, k, B, E):
+    cfg = cfg_of(dtype, B=B, L=40 if B < 100 else 12, H=4, P=64, N=128 if dtype == "bf16" else 32, E=E, k=k, F=F,
                  h0_std=0.1)
     inp = synth.make_inputs(cfg, seed=21)
     B, L = cfg.B, cfg.L
@@ -260,7 +263,7 @@ def test_decode_steps_match_oracle_and_forward(dtype):
     w, keep = hp.device_weights(inp)
     state = hp.dev(inp["h0"]).clone()
     ws = torch.empty(sb.swimba_decode_workspace_bytes(h, B), dtype=torch.uint8, device="cuda")
-    ys, idxs = [], []
+    ys, idxs, wts = [], [], []
     for t in range(L):
         u = hp.dev(inp["u"][:, t])
         x = hp.dev(inp["x"][:, t])
@@ -271,18 +274,22 @@ def test_decode_steps_match_oracle_and_forward(dtype):
         sb.swimba_decode_step(h, w, u, x, dt, state, B, y, idx, wt, ws)
         ys.append(y.cpu())
         idxs.append(idx.cpu())
+        wts.append(wt.cpu())
     assert sb.swimba_status(h) == 0
     y_dec = torch.stack(ys, 1)
     idx_dec = torch.stack(idxs, 1)
     ty, th = hp.tolerances(cfg)
     # (a) against the oracle's decode loop == oracle forward (pinned on the CPU side)
-    fwd = hp.gpu_forward(cfg, inp)
-    res = hp.compare_forward(cfg, inp, dict(y=y_dec, h_final=state.cpu(), idx=idx_dec, w=fwd["w"]),
+    res = hp.compare_forward(cfg, inp, dict(y=y_dec, h_final=state.cpu(), idx=idx_dec, w=torch.stack(wts, 1)),
                              ty, th)
-    # (b) against the library's own forward over the same L tokens
-    assert torch.equal(idx_dec, fwd["idx"])
-    assert hp.max_rel(y_dec.double().numpy(), fwd["y"].double().numpy()) <= ty
-    assert hp.max_rel(state.cpu().numpy(), fwd["h_final"].numpy()) <= th
+    # (b) against the library's own forward over the same L tokens (the two paths may use different
+    # router kernels: only tokens too close to a tie to be certified may be routed differently)
+    fwd = hp.gpu_forward(cfg, inp)
+    differ = int((idx_dec != fwd["idx"]).any(-1).sum())
+    assert differ <= res["ambiguous"]
+    if differ == 0:
+        assert hp.max_rel(y_dec.double().numpy(), fwd["y"].double().numpy()) <= ty
+        assert hp.max_rel(state.cpu().numpy(), fwd["h_final"].numpy()) <= th
     sb.swimba_destroy(h)
 
 
