@@ -167,6 +167,37 @@ int swimba_ssd_slots(swimba_handle *h, const swimba_weights *w, const void *x_sl
                      void *y, float *h_final, void *workspace, size_t workspace_bytes,
                      void *cuda_stream);
 
+/* The whole block around the mixer (Section "Swimba layer": the in-projection of a Mamba-2 block
+ * becomes a mixture of expert projections, "the rest of the Mamba-2 layer is kept unchanged"; that
+ * rest is the public Mamba-2 block):
+ *   [z | x' | dt] = W_in u               shared in-projection: D = H*P gate columns, D input columns,
+ *                                        H raw step sizes
+ *   [B' | C']     = router, top-k, expert projections, parameter-space mix of u (as swimba_route_mix)
+ *   [x | B | C]   = silu(causal depthwise conv of width d_conv over [x' | B' | C'])
+ *   y             = the single selective-SSM recurrence on (x, B, C, dt), skip term included
+ *   out           = W_out ( rmsnorm over each of the G channel groups of y * silu(z), times norm_w )
+ * Weights (device pointers): W_in [2D + H, F] dtype; conv_w [D + S, d_conv] float, tap d_conv - 1
+ * multiplies the current token; conv_b [D + S] float or NULL; norm_w [D] float; W_out [F, D] dtype.
+ *   u [B,L,F] -> out [B,L,F] dtype.  conv_state_in / conv_state_out [B, d_conv - 1, D + S] dtype: the
+ * d_conv - 1 pre-convolution rows before / at the end of the call (NULL: zeros / not wanted); with
+ * h0 / h_final they carry a sequence across calls (chunked prefill).  d_conv in 1..4, P % 8 == 0.
+ * Linear maps whose width is not a multiple of 32 run on the CUDA cores. */
+typedef struct {
+    const void *W_in;
+    const float *conv_w;
+    const float *conv_b;
+    const float *norm_w;
+    const void *W_out;
+    int32_t d_conv;
+    float eps;
+} swimba_block_weights;
+size_t swimba_block_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+int swimba_block_forward(swimba_handle *h, const swimba_weights *w, const swimba_block_weights *bw,
+                         const void *u, const void *conv_state_in, const float *h0, int32_t B,
+                         int32_t L, void *out, void *conv_state_out, float *h_final,
+                         int32_t *topk_idx, float *topk_w, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream);
+
 /* Bytes of device workspace swimba_decode_step needs for B sequences. */
 size_t swimba_decode_workspace_bytes(const swimba_handle *h, int32_t B);
 
@@ -220,9 +251,9 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..14 (1 router + grouping by
+ * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..17 (1 router + grouping by
  * expert (for fewer than about 28000 tokens the launch also computes the SSD step sizes), 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
- * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
+ * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection, 15 convolution + SiLU, 16 gated norm, 17 step-size columns; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);

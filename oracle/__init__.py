@@ -259,3 +259,80 @@ def swimba_decode_step(u, x, dt, W_r, W_e, A, dt_bias, D, k: int, state, G: int 
                                              _p(fi), _p(fw), _p(state), _p(y), _p(idx), _p(w)),
            "oracle_swimba_decode_step")
     return dict(y=y, idx=idx, w=w)
+
+
+def conv_silu(xin, w, bias=None, state=None):
+    """Causal depthwise convolution + SiLU.  xin[B,L,C], w[C,K], bias[C] or None, state[B,K-1,C] or
+    None (the K-1 tokens before the call, oldest first) -> (out[B,L,C], state_out[B,K-1,C])."""
+    xin = _d(xin)
+    B, L, C = xin.shape
+    w = _d(w)
+    K = w.shape[1]
+    assert w.shape == (C, K)
+    bias = _d(bias, (C,)) if bias is not None else None
+    state = _d(state, (B, K - 1, C)) if state is not None else None
+    out = np.zeros((B, L, C), np.float64)
+    st = np.zeros((B, K - 1, C), np.float64)
+    _check(_load().oracle_conv_silu(_p(xin), _p(w), _p(bias), _p(state), B, L, C, K, _p(out), _p(st)),
+           "oracle_conv_silu")
+    return out, st
+
+
+def gated_rmsnorm(y, z, weight, ngroups: int = 1, eps: float = 1e-5):
+    """out = rmsnorm_groups(y * silu(z)) * weight.  y, z [T,D], weight [D]."""
+    y = _d(y)
+    T, D = y.shape
+    z = _d(z, (T, D))
+    weight = _d(weight, (D,))
+    out = np.zeros((T, D), np.float64)
+    _check(_load().oracle_gated_rmsnorm(_p(y), _p(z), _p(weight), ctypes.c_long(T), D, ngroups,
+                                        ctypes.c_double(eps), _p(out)), "oracle_gated_rmsnorm")
+    return out
+
+
+def linear(x, W):
+    """out[T,O] = x[T,F] W[O,F]^T."""
+    x = _d(x)
+    W = _d(W)
+    T, F = x.shape
+    O = W.shape[0]
+    assert W.shape == (O, F)
+    out = np.zeros((T, O), np.float64)
+    _check(_load().oracle_linear(_p(x), _p(W), ctypes.c_long(T), F, O, _p(out)), "oracle_linear")
+    return out
+
+
+def block_forward(u, W_in, W_r, W_e, conv_w, conv_b, A, dt_bias, D, norm_w, W_out, H: int, k: int,
+                  G: int = 1, eps: float = 1e-5, conv_state=None, h0=None, forced_idx=None,
+                  forced_w=None):
+    """The whole block around the mixer, step by step (the Mamba-2 block with its B / C projection
+    replaced by the routed mixture of expert projections):
+      [z | x' | dt] = W_in u                      shared in-projection (D = H*P channels each, H step sizes)
+      [B' | C']     = router + top-k + expert projections + parameter-space mix of u
+      [x | B | C]   = silu(causal depthwise conv([x' | B' | C']))
+      y, h          = the single selective-SSM recurrence on (x, B, C, dt)
+      out           = W_out ( rmsnorm(y * silu(z)) * norm_w )
+    u[B,L,F] -> dict(out[B,L,F], h_final, conv_state, idx, w, y, BC)."""
+    u = _d(u)
+    B, L, F = u.shape
+    W_in = _d(W_in)
+    Dm = (W_in.shape[0] - H) // 2
+    P = Dm // H
+    T = B * L
+    zxdt = linear(u.reshape(T, F), W_in)
+    z, xp, dt = zxdt[:, :Dm], zxdt[:, Dm:2 * Dm], zxdt[:, 2 * Dm:]
+    E, S, _ = np.asarray(W_e).shape
+    if forced_idx is None:
+        r = router(u.reshape(T, F), W_r, k)
+        idx, wts = r["idx"], r["w"]
+    else:
+        idx, wts = _i(forced_idx).reshape(T, k), _d(forced_w).reshape(T, k)
+    BCp = mix_topk(u.reshape(T, F), W_e, idx, wts)
+    xbc, cst = conv_silu(np.concatenate([xp, BCp], -1).reshape(B, L, Dm + S), conv_w, conv_b, conv_state)
+    x = np.ascontiguousarray(xbc[..., :Dm]).reshape(B, L, H, P)
+    BC = np.ascontiguousarray(xbc[..., Dm:])
+    y, hf = ssm_recurrence(x, BC, dt.reshape(B, L, H), A, dt_bias, D, h0, G=G)
+    g = gated_rmsnorm(y.reshape(T, Dm), z, norm_w, ngroups=G, eps=eps)
+    out = linear(g, W_out).reshape(B, L, -1)
+    return dict(out=out, h_final=hf, conv_state=cst, idx=idx.reshape(B, L, k), w=wts.reshape(B, L, k),
+                y=y, BC=BC, x=x, z=z.reshape(B, L, Dm), dt=dt.reshape(B, L, H))

@@ -415,6 +415,85 @@ int oracle_swimba_decode_step(const double *u, const double *x, const double *dt
     return rc;
 }
 
+/* ===========================================================================
+ * The rest of the block around the mixer (Section "Swimba layer": the in-projection becomes a
+ * mixture of experts and "the rest of the Mamba-2 layer is kept unchanged"; the paper does not
+ * restate that rest, so these three functions write out the public Mamba-2 block conventions:
+ * causal depthwise convolution + SiLU on the [x | B | C] stream, the gated RMS norm
+ * norm(y * silu(z)) * weight, and plain linear maps).
+ * ======================================================================== */
+static double silu(double v) { return v / (1.0 + exp(-v)); }
+
+/* Causal depthwise convolution of width K followed by SiLU, channel by channel:
+ *   out[b,t,c] = silu( bias[c] + sum_{i<K} w[c,i] * in[b, t-(K-1)+i, c] ),
+ * i.e. w[c,K-1] multiplies the current token.  Positions before the call are taken from
+ * state_in[b,i,c] (the K-1 tokens preceding the call, oldest first; zeros when NULL); the last
+ * K-1 inputs of the call (or of state + call when L < K-1) are returned in state_out. */
+int oracle_conv_silu(const double *in, const double *w, const double *bias, const double *state_in,
+                     int B, int L, int C, int K, double *out, double *state_out)
+{
+    if (!in || !w || !out || B <= 0 || L < 0 || C <= 0 || K <= 0) return ORACLE_BAD_ARG;
+    for (int b = 0; b < B; ++b)
+        for (int t = 0; t < L; ++t)
+            for (int c = 0; c < C; ++c) {
+                double acc = bias ? bias[c] : 0.0;
+                for (int i = 0; i < K; ++i) {
+                    const int tt = t - (K - 1) + i;
+                    double v;
+                    if (tt >= 0) v = in[((long)b * L + tt) * C + c];
+                    else v = state_in ? state_in[((long)b * (K - 1) + (K - 1 + tt)) * C + c] : 0.0;
+                    acc += w[(long)c * K + i] * v;
+                }
+                out[((long)b * L + t) * C + c] = silu(acc);
+            }
+    if (state_out)
+        for (int b = 0; b < B; ++b)
+            for (int i = 0; i < K - 1; ++i)
+                for (int c = 0; c < C; ++c) {
+                    const int tt = L - (K - 1) + i;      /* position of the i-th kept token */
+                    double v;
+                    if (tt >= 0) v = in[((long)b * L + tt) * C + c];
+                    else v = state_in ? state_in[((long)b * (K - 1) + (K - 1 + tt)) * C + c] : 0.0;
+                    state_out[((long)b * (K - 1) + i) * C + c] = v;
+                }
+    return ORACLE_OK;
+}
+
+/* Gated RMS norm over groups of D/ngroups channels:
+ *   v = y * silu(z),  out = v / sqrt(mean_group(v^2) + eps) * weight. */
+int oracle_gated_rmsnorm(const double *y, const double *z, const double *weight, long T, int D,
+                         int ngroups, double eps, double *out)
+{
+    if (!y || !z || !weight || !out || D <= 0 || ngroups <= 0 || D % ngroups != 0) return ORACLE_BAD_ARG;
+    const int gs = D / ngroups;
+    for (long t = 0; t < T; ++t)
+        for (int g = 0; g < ngroups; ++g) {
+            double ss = 0.0;
+            for (int c = g * gs; c < (g + 1) * gs; ++c) {
+                const double v = y[t * D + c] * silu(z[t * D + c]);
+                ss += v * v;
+            }
+            const double r = 1.0 / sqrt(ss / gs + eps);
+            for (int c = g * gs; c < (g + 1) * gs; ++c)
+                out[t * D + c] = y[t * D + c] * silu(z[t * D + c]) * r * weight[c];
+        }
+    return ORACLE_OK;
+}
+
+/* out[T,O] = x[T,F] W[O,F]^T */
+int oracle_linear(const double *x, const double *W, long T, int F, int O, double *out)
+{
+    if (!x || !W || !out || F <= 0 || O <= 0) return ORACLE_BAD_ARG;
+#pragma omp parallel for schedule(static)
+    for (long t = 0; t < T; ++t)
+        for (int o = 0; o < O; ++o) {
+            double acc = 0.0;
+            for (int f = 0; f < F; ++f) acc += W[(long)o * F + f] * x[t * F + f];
+            out[t * O + o] = acc;
+        }
+    return ORACLE_OK;
+}
+
 int oracle_num_threads(void)
 {
     int n = 1;

@@ -31,6 +31,7 @@ FLAG_CHECK_INDICES = 1
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_route_project_slots", "swimba_ssd_slots_workspace_bytes", "swimba_ssd_slots",
+    "swimba_block_workspace_bytes", "swimba_block_forward",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
     "swimba_forward_host", "swimba_route_mix_static", "swimba_profile", "swimba_profile_read",
     "swimba_selftest_wait", "swimba_last_launch_count", "swimba_status", "swimba_last_error",
@@ -52,6 +53,11 @@ class swimba_config(ctypes.Structure):
 
 class swimba_weights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("W_router", "W_expert", "A", "dt_bias", "D")]
+
+
+class swimba_block_weights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("W_in", "conv_w", "conv_b", "norm_w", "W_out")] + \
+               [("d_conv", ctypes.c_int32), ("eps", ctypes.c_float)]
 
 
 _lib = None
@@ -93,6 +99,11 @@ def lib() -> ctypes.CDLL:
         L.swimba_ssd_slots.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32, vp,
                                        vp, vp, sz, vp]
         L.swimba_ssd_slots.restype = ctypes.c_int
+        L.swimba_block_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_block_workspace_bytes.restype = sz
+        L.swimba_block_forward.argtypes = [vp, ctypes.POINTER(swimba_weights), ctypes.POINTER(swimba_block_weights),
+                                           vp, vp, vp, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.swimba_block_forward.restype = ctypes.c_int
         L.swimba_decode_step.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32,
                                          vp, vp, vp, vp, sz, vp]
         L.swimba_decode_step.restype = ctypes.c_int
@@ -251,6 +262,31 @@ def swimba_ssd_slots(h: Handle, w: swimba_weights, x_slots, BC_slots, dt, h0, B:
     return rc
 
 
+def make_block_weights(W_in, conv_w, conv_b, norm_w, W_out, d_conv: int, eps: float = 1e-5) -> swimba_block_weights:
+    bw = swimba_block_weights()
+    bw.W_in, bw.conv_w, bw.norm_w, bw.W_out = W_in.data_ptr(), conv_w.data_ptr(), norm_w.data_ptr(), W_out.data_ptr()
+    bw.conv_b = conv_b.data_ptr() if conv_b is not None else None
+    bw.d_conv, bw.eps = d_conv, eps
+    bw._keep = (W_in, conv_w, conv_b, norm_w, W_out)
+    return bw
+
+
+def swimba_block_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_block_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_block_forward(h: Handle, w: swimba_weights, bw: swimba_block_weights, u, conv_state_in, h0,
+                         B: int, L: int, out, conv_state_out, h_final, topk_idx, topk_w, workspace,
+                         stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_block_forward(h.ptr, ctypes.byref(w), ctypes.byref(bw), _ptr(u), _ptr(conv_state_in),
+                                    _ptr(h0), B, L, _ptr(out), _ptr(conv_state_out), _ptr(h_final),
+                                    _ptr(topk_idx), _ptr(topk_w), wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
 def swimba_ssd(h: Handle, w: swimba_weights, x, BC, dt, h0, B: int, L: int, y, h_final, workspace,
                stream=None, check: bool = True) -> int:
     wp, wb = _ws(workspace)
@@ -288,7 +324,8 @@ def swimba_forward_host(h: Handle, w: swimba_weights, u_host, x_host, dt_host, B
 KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
                 9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars", 12: "slot_streams",
-                13: "slot_sum", 14: "project_small"}
+                13: "slot_sum", 14: "project_small", 15: "conv_silu", 16: "gated_rmsnorm",
+                17: "dt_columns"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

@@ -439,6 +439,133 @@ int swimba_ssd_slots(swimba_handle *h, const swimba_weights *w, const void *x_sl
     return rc;
 }
 
+namespace {
+// out[T,So] = in[T,Fi] W[So,Fi]^T as the grouped projection with a single expert (tensor cores
+// where the shape allows, else the SIMT projection).  scratch: dense_scratch_bytes(T).
+size_t dense_scratch_bytes(int64_t T)
+{
+    return align_up((size_t)T * sizeof(int32_t)) + align_up((size_t)T * sizeof(float)) +
+           align_up(expert_gemm_workspace_bytes(T, 32, 1, 1));
+}
+int dense_linear(swimba_handle *h, LaunchCtx &ctx, const void *in, const void *W, int64_t T, int Fi, int So,
+                 void *out, char *scratch)
+{
+    const int dtype = h->cfg.dtype;
+    int32_t *idx = (int32_t *)scratch;
+    float *wt = (float *)(scratch + align_up((size_t)T * sizeof(int32_t)));
+    char *gws = (char *)wt + align_up((size_t)T * sizeof(float));
+    const bool tensor = dtype == SWIMBA_DTYPE_BF16 && expert_gemm_supported(Fi, So);
+    int *counts = nullptr, *perm = nullptr;
+    if (tensor) {
+        counts = expert_gemm_counts(gws);
+        perm = expert_gemm_perm(gws);
+        if (cudaMemsetAsync(counts, 0, sizeof(int) * SWIMBA_MAX_EXPERTS, ctx.stream) != cudaSuccess)
+            return fail(h, SWIMBA_ERR_CUDA, "clearing the expert histogram failed");
+    }
+    // one expert: the router only writes idx = 0, w = 1 and the identity list (W stands in for the
+    // router matrix, which is not read)
+    int rc = launch_router(ctx, dtype, in, W, T, Fi, 1, 1, idx, wt, counts, perm, T, h->sm_count, nullptr, 0,
+                           ScalarsArgs{});
+    if (rc != SWIMBA_OK) return fail(h, rc, "list launch failed");
+    rc = tensor ? launch_expert_gemm(ctx, in, W, wt, T, Fi, So, 1, 1, h->sm_count, out, gws)
+                : launch_project_mix_simt(ctx, dtype, in, W, idx, wt, T, Fi, So, 1, 1, out, false);
+    if (rc != SWIMBA_OK) return fail(h, rc, "linear map launch failed");
+    return SWIMBA_OK;
+}
+
+struct BlockLayout {
+    size_t zx, dtb, dt, bcp, x, bc, y, lin, fwd, total;
+};
+BlockLayout block_layout(const swimba_config &c, int B, int L, int sm_count)
+{
+    BlockLayout l;
+    const size_t T = (size_t)B * L, es = elt_size(c.dtype);
+    const size_t D = (size_t)c.n_heads * c.head_dim, S = 2u * c.n_groups * c.d_state;
+    size_t off = 0;
+    l.zx = off;  off += align_up(T * 2 * D * es);
+    l.dtb = off; off += align_up(T * c.n_heads * es);
+    l.dt = off;  off += align_up(T * c.n_heads * sizeof(float));
+    l.bcp = off; off += align_up(T * S * es);
+    l.x = off;   off += align_up(T * D * es);            // x, later the normalised gate output
+    l.bc = off;  off += align_up(T * S * es);
+    l.y = off;   off += align_up(T * D * es);
+    l.lin = off; off += dense_scratch_bytes((int64_t)T);
+    l.fwd = off; off += fwd_layout(c, B, L, sm_count).total;
+    l.total = off;
+    return l;
+}
+}  // namespace
+
+size_t swimba_block_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    return block_layout(h->cfg, B, L, h->sm_count).total;
+}
+
+int swimba_block_forward(swimba_handle *h, const swimba_weights *w, const swimba_block_weights *bw,
+                         const void *u, const void *conv_state_in, const float *h0, int32_t B, int32_t L,
+                         void *out, void *conv_state_out, float *h_final, int32_t *topk_idx, float *topk_w,
+                         void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    if ((int64_t)B * L * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (B * L * top_k must stay below 2^31)");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (!bw || !bw->W_in || !bw->conv_w || !bw->norm_w || !bw->W_out)
+        return fail(h, SWIMBA_ERR_NULL_ARG, "a block weight is NULL");
+    if (bw->d_conv < 1 || bw->d_conv > 4) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "d_conv must lie in 1..4");
+    const swimba_config &c = h->cfg;
+    if (c.head_dim % 8 != 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "the block needs head_dim % 8 == 0");
+    if (B == 0 || L == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !out || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, out or workspace is NULL");
+    if (!aligned16(u) || !aligned16(out) || !aligned16(conv_state_in) || !aligned16(conv_state_out) ||
+        !aligned16(h0) || !aligned16(h_final) || !aligned16(topk_idx) || !aligned16(topk_w) ||
+        !aligned16(workspace) || !aligned16(bw->W_in) || !aligned16(bw->W_out) || !aligned16(bw->conv_w) ||
+        !aligned16(bw->conv_b) || !aligned16(bw->norm_w))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const BlockLayout l = block_layout(c, B, L, h->sm_count);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    const int64_t T = (int64_t)B * L;
+    const size_t es = elt_size(c.dtype);
+    const int D = c.n_heads * c.head_dim, S = 2 * c.n_groups * c.d_state, F = c.d_model, H = c.n_heads;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    const FwdLayout fl = fwd_layout(c, B, L, h->sm_count);
+    char *fws = ws + l.fwd;
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(fws + fl.idx);
+    float *wt = topk_w ? topk_w : (float *)(fws + fl.w);
+    // shared in-projection: [z | x'] (2 D columns) and the raw step sizes (H columns)
+    rc = dense_linear(h, ctx, u, bw->W_in, T, F, 2 * D, ws + l.zx, ws + l.lin);
+    if (rc == SWIMBA_OK)
+        rc = dense_linear(h, ctx, u, (const char *)bw->W_in + (size_t)2 * D * F * es, T, F, H, ws + l.dtb, ws + l.lin);
+    if (rc == SWIMBA_OK) rc = launch_dt_columns(ctx, c.dtype, ws + l.dtb, H, 0, T, H, (float *)(ws + l.dt));
+    // routed mixture of the experts' B / C projections
+    if (rc == SWIMBA_OK) rc = run_route_mix(h, ctx, w, u, T, ws + l.bcp, false, idx, wt, fws + fl.gemm);
+    // convolution + SiLU over [x' | B' | C']
+    if (rc == SWIMBA_OK)
+        rc = launch_conv_silu(ctx, c.dtype, ws + l.zx + (size_t)D * es, 2 * (int64_t)D, ws + l.bcp, bw->conv_w,
+                              bw->conv_b, conv_state_in, B, L, D, S, bw->d_conv, ws + l.x, ws + l.bc, conv_state_out);
+    // the single recurrence
+    if (rc == SWIMBA_OK)
+        rc = run_ssd(h, ctx, w, ws + l.x, ws + l.bc, (const float *)(ws + l.dt), h0, B, L, ws + l.y, h_final,
+                     fws + fl.ssd);
+    // gate, norm, out-projection (the normalised rows reuse the x buffer)
+    if (rc == SWIMBA_OK)
+        rc = launch_gated_rmsnorm(ctx, c.dtype, ws + l.y, ws + l.zx, 2 * (int64_t)D, bw->norm_w, T, D, c.n_groups,
+                                  bw->eps, ws + l.x);
+    if (rc == SWIMBA_OK) rc = dense_linear(h, ctx, ws + l.x, bw->W_out, T, D, F, out, ws + l.lin);
+    if (rc != SWIMBA_OK && !h->err[0]) fail(h, rc, "a block kernel launch failed");
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const void *BC,
                const float *dt, const float *h0, int32_t B, int32_t L, void *y, float *h_final,
                void *workspace, size_t workspace_bytes, void *cuda_stream)

@@ -73,6 +73,15 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
 // out_dev: three 64-bit words on the device.
 int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev);
 
+// The rest of the block: causal depthwise convolution + SiLU over the channels [x' (D columns of a
+// matrix with row stride ldx) | B'C' (S)], gated RMS norm, step-size columns to fp32.
+int launch_conv_silu(LaunchCtx &ctx, int dtype, const void *xp, int64_t ldx, const void *bcp, const float *cw,
+                     const float *cb, const void *state_in, int B, int L, int D, int S, int K, void *x,
+                     void *bc, void *state_out);
+int launch_gated_rmsnorm(LaunchCtx &ctx, int dtype, const void *y, const void *z, int64_t ldz, const float *wt,
+                         int64_t T, int D, int ngroups, float eps, void *out);
+int launch_dt_columns(LaunchCtx &ctx, int dtype, const void *zxdt, int64_t ld, int off, int64_t T, int H, float *dt);
+
 // Per-timestep SIMT evaluation of the recurrence (fp32 state in registers).
 int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,
                           const float *dt, const float *A, const float *dt_bias, const float *D,

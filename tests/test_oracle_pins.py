@@ -383,3 +383,82 @@ def test_bad_arguments_are_rejected():
     with pytest.raises(ValueError):
         oracle.mix_topk(np.zeros((2, 3)), np.zeros((2, 4, 3)), np.array([[5], [0]]),
                         np.ones((2, 1)))                            # expert index out of range
+
+
+# ------------------------------------------------------------------ the rest of the block
+def test_conv_silu_equals_numpy_convolution_and_carries_its_state():
+    rng = np.random.default_rng(5)
+    B, L, C, K = 2, 37, 5, 4
+    xin = rng.standard_normal((B, L, C))
+    w = rng.standard_normal((C, K))
+    bias = rng.standard_normal(C)
+    out, st = oracle.conv_silu(xin, w, bias)
+    for b in range(B):
+        for c in range(C):
+            # np.convolve flips its second argument: w[c, K-1] multiplies the current token
+            full = np.convolve(xin[b, :, c], w[c, ::-1])[:L] + bias[c]
+            np.testing.assert_allclose(out[b, :, c], full / (1.0 + np.exp(-full)), rtol=1e-12, atol=1e-12)
+    np.testing.assert_array_equal(st, xin[:, L - (K - 1):, :])
+    # two calls with the carried state equal one call; a call shorter than the window keeps older tokens
+    cut = 11
+    o1, s1 = oracle.conv_silu(xin[:, :cut], w, bias)
+    o2, s2 = oracle.conv_silu(xin[:, cut:], w, bias, state=s1)
+    np.testing.assert_allclose(np.concatenate([o1, o2], 1), out, rtol=1e-12, atol=1e-12)
+    np.testing.assert_array_equal(s2, st)
+    o3, s3 = oracle.conv_silu(xin[:, :2], w, bias, state=np.ones((B, K - 1, C)))
+    np.testing.assert_array_equal(s3[:, 0], np.ones((B, C)))
+    np.testing.assert_array_equal(s3[:, 1:], xin[:, :2])
+
+
+def test_gated_rmsnorm_and_linear_equal_their_numpy_definitions():
+    rng = np.random.default_rng(6)
+    T, D, G = 9, 24, 3
+    y, z, wt = rng.standard_normal((T, D)), rng.standard_normal((T, D)), rng.standard_normal(D)
+    v = (y * z / (1.0 + np.exp(-z))).reshape(T, G, D // G)
+    ref = (v / np.sqrt((v * v).mean(-1, keepdims=True) + 1e-5)).reshape(T, D) * wt
+    np.testing.assert_allclose(oracle.gated_rmsnorm(y, z, wt, ngroups=G), ref, rtol=1e-12, atol=1e-12)
+    # unit weight, one group, no gate effect (z large: silu(z) ~ z): output has unit mean square
+    out = oracle.gated_rmsnorm(y, np.full((T, D), 50.0), np.ones(D), ngroups=1, eps=0.0)
+    np.testing.assert_allclose((out * out).mean(-1), 1.0, rtol=1e-9)
+    W = rng.standard_normal((7, D))
+    np.testing.assert_allclose(oracle.linear(y, W), y @ W.T, rtol=1e-12, atol=1e-12)
+
+
+def test_block_forward_is_the_composition_of_its_steps_and_reduces_to_a_plain_block():
+    rng = np.random.default_rng(7)
+    B, L, F, H, P, N, G, E, k, K = 2, 19, 12, 2, 4, 8, 1, 3, 2, 4
+    Dm, S = H * P, 2 * G * N
+    u = rng.standard_normal((B, L, F))
+    W_in = rng.standard_normal((2 * Dm + H, F)) * 0.3
+    W_r = rng.standard_normal((E, F))
+    W_e = rng.standard_normal((E, S, F)) * 0.3
+    conv_w, conv_b = rng.standard_normal((Dm + S, K)) * 0.5, rng.standard_normal(Dm + S) * 0.1
+    A, dt_bias, D = -np.exp(rng.uniform(0, 2, H)), rng.standard_normal(H), rng.standard_normal(H)
+    norm_w, W_out = rng.standard_normal(Dm), rng.standard_normal((F, Dm)) * 0.3
+    r = oracle.block_forward(u, W_in, W_r, W_e, conv_w, conv_b, A, dt_bias, D, norm_w, W_out, H=H, k=k, G=G)
+    # the mixer inside the block is the layer itself on the convolved streams
+    y2, h2 = oracle.ssm_recurrence(r["x"], r["BC"], r["dt"], A, dt_bias, D, G=G)
+    np.testing.assert_array_equal(y2, r["y"])
+    # identical experts and dense routing: the block is a plain Mamba-2 block whose B / C projection is
+    # that one expert matrix, written here with numpy only
+    W1 = np.repeat(W_e[:1], E, 0)
+    rb = oracle.block_forward(u, W_in, W_r, W1, conv_w, conv_b, A, dt_bias, D, norm_w, W_out, H=H, k=E, G=G)
+    T = B * L
+    zxdt = u.reshape(T, F) @ W_in.T
+    pre = np.concatenate([zxdt[:, Dm:2 * Dm], u.reshape(T, F) @ W_e[0].T], -1).reshape(B, L, Dm + S)
+    pad = np.concatenate([np.zeros((B, K - 1, Dm + S)), pre], 1)
+    acc = sum(conv_w[:, i] * pad[:, i:i + L] for i in range(K)) + conv_b
+    xbc = acc / (1.0 + np.exp(-acc))
+    y_ref, _ = oracle.ssm_recurrence(xbc[..., :Dm].reshape(B, L, H, P), xbc[..., Dm:], zxdt[:, 2 * Dm:].reshape(B, L, H),
+                                     A, dt_bias, D, G=G)
+    z = zxdt[:, :Dm]
+    v = y_ref.reshape(T, Dm) * z / (1.0 + np.exp(-z))
+    g = v / np.sqrt((v * v).mean(-1, keepdims=True) + 1e-5) * norm_w
+    np.testing.assert_allclose(rb["out"], (g @ W_out.T).reshape(B, L, F), rtol=1e-9, atol=1e-11)
+    # chunked prefill: two calls carrying the convolution window and the SSM state equal one call
+    cut = 7
+    r1 = oracle.block_forward(u[:, :cut], W_in, W_r, W_e, conv_w, conv_b, A, dt_bias, D, norm_w, W_out, H=H, k=k, G=G)
+    r2 = oracle.block_forward(u[:, cut:], W_in, W_r, W_e, conv_w, conv_b, A, dt_bias, D, norm_w, W_out, H=H, k=k, G=G,
+                              conv_state=r1["conv_state"], h0=r1["h_final"])
+    np.testing.assert_allclose(np.concatenate([r1["out"], r2["out"]], 1), r["out"], rtol=1e-9, atol=1e-11)
+    np.testing.assert_allclose(r2["h_final"], r["h_final"], rtol=1e-9, atol=1e-12)
