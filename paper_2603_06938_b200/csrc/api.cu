@@ -822,12 +822,18 @@ int swimba_status(swimba_handle *h)
                  cudaGetErrorString(cudaGetLastError()));
         return SWIMBA_ERR_CUDA;
     }
-    int code = 0;
-    if (cudaMemcpy(&code, h->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    int word[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(word, h->d_status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess)
         return fail(h, SWIMBA_ERR_CUDA, "reading the device status word failed");
+    const int code = word[0];
     if (code != 0) {
         cudaMemset(h->d_status, 0, 64);
-        snprintf(h->err, sizeof(h->err), "device reported error %d", code);
+        if (code == SWIMBA_ERR_DEVICE_TIMEOUT)
+            snprintf(h->err, sizeof(h->err),
+                     "device reported error %d (a wait ran out: barrier at shared address 0x%x, parity %d, block %d, thread %d)",
+                     code, (unsigned)word[1], word[2], word[3] >> 12, word[3] & 0xfff);
+        else
+            snprintf(h->err, sizeof(h->err), "device reported error %d", code);
     }
     return code;
 }

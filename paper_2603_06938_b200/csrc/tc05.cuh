@@ -67,7 +67,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         if (*abort_flag) return false;
         if (clock64() - t0 > limit_cycles) {
             *abort_flag = 1;
-            atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_TIMEOUT);
+            // the first wait to run out also leaves where it was: barrier (shared-memory address),
+            // phase parity, block and thread
+            if (atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_TIMEOUT) == 0) {
+                d_status[1] = (int)smem_u32(bar);
+                d_status[2] = (int)parity;
+                d_status[3] = (int)((blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z)) << 12 | threadIdx.x);
+            }
             return false;
         }
     }
