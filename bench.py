@@ -399,6 +399,8 @@ def main():
     ap.add_argument("--no-comparators", action="store_true")
     ap.add_argument("--no-workloads", action="store_true",
                     help="skip the compact records of the other forward workloads")
+    ap.add_argument("--no-serving", action="store_true",
+                    help="skip the batch x input-length sweep of packed prefill and decode")
     ap.add_argument("--no-e2e", action="store_true",
                     help="skip the host-buffer leg (for profiler launch lists of the device-resident steps)")
     args = ap.parse_args()
@@ -515,6 +517,10 @@ def main():
     if single and not args.no_decode:
         decode = bench_decode(sb, pk, steps=args.decode_steps)
 
+    serving = None
+    if single and not args.no_serving:
+        serving = bench_serving(sb)
+
     cpu = None
     if single and not args.no_cpu_baseline:
         cpu, _ = time_oracle_sample(cfg, cfg.B)
@@ -532,7 +538,7 @@ def main():
                        "how": "value is the median over rounds of exactly `steps` steps each"},
             "ssd_segments": nseg,
             "kernels": kernels, "comparators": comparators, "workloads": workloads,
-            "decode": decode, "cpu_baseline": cpu,
+            "decode": decode, "serving": serving, "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     if dist is not None:
@@ -596,6 +602,82 @@ def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
     }
     sb.swimba_destroy(h)
     return out
+
+
+def bench_serving(sb, steps: int = 10, warmup: int = 3):
+    """Serving-shaped batches on the `mid` layer shape: packed prefill (swimba_forward_packed) over a
+    sweep of batch size x input length plus one batch of mixed lengths, and the decode step over a
+    sweep of batch sizes.  Device-resident inputs, CUDA events on the launching stream."""
+    base = synth.CONFIGS["mid"]
+    h = sb.swimba_create(base.F, base.H, base.P, base.N, base.G, base.E, base.k, base.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(9)
+    wts = {n: v.cuda() for n, v in synth.make_weights(base, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    stream = torch.cuda.current_stream()
+    dgen = torch.Generator(device="cuda")
+    dgen.manual_seed(10)
+    Tmax = 32768
+    # two input sets, together above L2
+    sets = [dict(u=torch.randn(Tmax, base.F, generator=dgen, device="cuda").bfloat16(),
+                 x=torch.randn(Tmax, base.H, base.P, generator=dgen, device="cuda").bfloat16(),
+                 dt=0.5 * torch.randn(Tmax, base.H, generator=dgen, device="cuda")) for _ in range(2)]
+    y = torch.empty_like(sets[0]["x"])
+
+    def timed(fn):
+        for i in range(warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            fn(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    prefill = []
+    mixes = [("B=%d L=%d" % (b, l), [l] * b) for b in (1, 8, 64) for l in (128, 1024, 4096) if b * l <= Tmax]
+    lg = torch.Generator().manual_seed(11)
+    mixed = [int(v) for v in torch.exp(torch.rand(48, generator=lg) * (math.log(4096) - math.log(16)) + math.log(16))]
+    while sum(mixed) > Tmax:
+        mixed.pop()
+    mixes.append(("%d sequences, lengths log-uniform in [16, 4096]" % len(mixed), mixed))
+    mixes.append(("one 16384-token prompt among 64 single-token sequences", [16384] + [1] * 64))
+    for name, lens in mixes:
+        cu = [0]
+        for v in lens:
+            cu.append(cu[-1] + v)
+        T = cu[-1]
+        assert T <= Tmax, "the batch does not fit the input arrays"
+        hf = torch.empty(len(lens), base.H, base.P, base.N, device="cuda")
+        ws = torch.empty(sb.swimba_packed_workspace_bytes(h, cu), dtype=torch.uint8, device="cuda")
+
+        def step(i, cu=cu, hf=hf, ws=ws):
+            s_ = sets[i % 2]
+            sb.swimba_forward_packed(h, w, s_["u"], s_["x"], s_["dt"], None, cu, y, hf, None, None, ws)
+
+        ms = timed(step)
+        prefill.append({"batch": name, "tokens": T, "ms": ms, "tokens_per_s": T / (ms * 1e-3),
+                        "segments": sb.swimba_packed_segments(h, cu)})
+        del hf, ws
+    decode = []
+    for B in (1, 8, 32, 128):
+        state = 0.1 * torch.randn(B, base.H, base.P, base.N, device="cuda")
+        ws = torch.empty(sb.swimba_decode_workspace_bytes(h, B), dtype=torch.uint8, device="cuda")
+        yd = torch.empty(B, base.H, base.P, dtype=torch.bfloat16, device="cuda")
+
+        def dstep(i, B=B, state=state, ws=ws, yd=yd):
+            s_ = sets[i % 2]
+            sb.swimba_decode_step(h, w, s_["u"][:B], s_["x"][:B], s_["dt"][:B], state, B, yd, None, None, ws)
+
+        ms = timed(dstep)
+        decode.append({"batch": B, "us_per_step": ms * 1e3, "tokens_per_s": B / (ms * 1e-3)})
+        del state, ws, yd
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    return {"layer": f"d_model={base.F} H={base.H} P={base.P} N={base.N} E={base.E} top_k={base.k} bf16",
+            "steps": steps, "prefill_packed": prefill, "decode": decode}
 
 
 if __name__ == "__main__":

@@ -140,6 +140,30 @@ int swimba_ssd(swimba_handle *h, const swimba_weights *w, const void *x, const v
  * positive.  The result does not depend on the segmentation beyond rounding. */
 int32_t swimba_ssd_segments(const swimba_handle *h, int32_t B, int32_t L);
 
+/* The layer forward over a PACKED batch of sequences of different lengths (serving-shaped
+ * batches: Section "Efficiency" measures prefill and decoding over mixes of batch size and input
+ * length).  Sequence b of nseq holds tokens cu_seqlens[b] .. cu_seqlens[b+1]-1 of the packed arrays
+ *   u [T, F] dtype, x [T, H, P] dtype, dt [T, H] fp32 or NULL, y [T, H, P] dtype out,
+ *   topk_idx / topk_w [T, k] out (may be NULL),   T = cu_seqlens[nseq];
+ * every sequence runs its own recurrence (Theorem 1) from h0[b] (h0 [nseq, H, P, N] fp32 or NULL =>
+ * zeros) and leaves its end state in h_final[b] (may be NULL); a sequence of length 0 passes its
+ * state through.  Routing, projection and mix are per token and see the batch as one run of T
+ * tokens.  cu_seqlens is a HOST array of nseq + 1 non-decreasing offsets starting at 0; it is read
+ * (and small tables derived from it are copied to the device, in stream order) before the call
+ * returns, and may be freed then.  Everything else: device pointers, caller-owned, 16-byte aligned,
+ * enqueued on cuda_stream.  The workspace must hold swimba_packed_workspace_bytes(h, cu_seqlens,
+ * nseq) bytes (0 for invalid offsets or T == 0).  A sequence much longer than the batch's per-SM
+ * share of tokens is cut into segments as in swimba_ssd_segments; swimba_packed_segments returns
+ * the number of segments over the whole batch (nseq when nothing is cut).
+ * Errors: as swimba_forward; SWIMBA_ERR_UNSUPPORTED_SHAPE for offsets that do not start at 0 or
+ * decrease.  Rows of y outside every sequence do not exist; no byte outside y[0 .. T) is written. */
+size_t swimba_packed_workspace_bytes(const swimba_handle *h, const int32_t *cu_seqlens, int32_t nseq);
+int32_t swimba_packed_segments(const swimba_handle *h, const int32_t *cu_seqlens, int32_t nseq);
+int swimba_forward_packed(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                          const float *dt, const float *h0, const int32_t *cu_seqlens, int32_t nseq,
+                          void *y, float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream);
+
 /* The general form of the layer, with expert-specific SSM inputs (the state equation of Section
  * "MoE-parameterized SSM" as printed: h_t = A h_{t-1} + sum_{e in K_t} pi_{t,e} B_t^(e) X_t^(e)^T,
  * Y_t = (sum_{e in K_t} pi_{t,e} C_t^(e))^T h_t).  The caller's experts produce X^(e) themselves (in

@@ -30,6 +30,7 @@ FLAG_CHECK_INDICES = 1
 
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
+    "swimba_packed_workspace_bytes", "swimba_packed_segments", "swimba_forward_packed",
     "swimba_route_project_slots", "swimba_ssd_slots_workspace_bytes", "swimba_ssd_slots",
     "swimba_block_workspace_bytes", "swimba_block_forward",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
@@ -85,6 +86,13 @@ def lib() -> ctypes.CDLL:
         L.swimba_forward.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32,
                                      vp, vp, vp, vp, vp, sz, vp]
         L.swimba_forward.restype = ctypes.c_int
+        L.swimba_packed_workspace_bytes.argtypes = [vp, ctypes.POINTER(i32), i32]
+        L.swimba_packed_workspace_bytes.restype = sz
+        L.swimba_packed_segments.argtypes = [vp, ctypes.POINTER(i32), i32]
+        L.swimba_packed_segments.restype = i32
+        L.swimba_forward_packed.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp,
+                                            ctypes.POINTER(i32), i32, vp, vp, vp, vp, vp, sz, vp]
+        L.swimba_forward_packed.restype = ctypes.c_int
         L.swimba_route_mix.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, i64, vp, vp, vp, vp,
                                        sz, vp]
         L.swimba_route_mix.restype = ctypes.c_int
@@ -211,6 +219,34 @@ def swimba_forward(h: Handle, w: swimba_weights, u, x, dt, h0, B: int, L: int, y
     rc = lib().swimba_forward(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), B, L,
                               _ptr(y), _ptr(h_final), _ptr(topk_idx), _ptr(topk_w), wp, wb,
                               _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def _offsets(cu_seqlens):
+    """Host offsets (a sequence of ints) as a C array of nseq + 1 int32."""
+    n = len(cu_seqlens)
+    return (ctypes.c_int32 * n)(*[int(v) for v in cu_seqlens]), n - 1
+
+
+def swimba_packed_workspace_bytes(h: Handle, cu_seqlens) -> int:
+    arr, nseq = _offsets(cu_seqlens)
+    return int(lib().swimba_packed_workspace_bytes(h.ptr, arr, nseq))
+
+
+def swimba_packed_segments(h: Handle, cu_seqlens) -> int:
+    arr, nseq = _offsets(cu_seqlens)
+    return int(lib().swimba_packed_segments(h.ptr, arr, nseq))
+
+
+def swimba_forward_packed(h: Handle, w: swimba_weights, u, x, dt, h0, cu_seqlens, y, h_final,
+                          topk_idx, topk_w, workspace, stream=None, check: bool = True) -> int:
+    arr, nseq = _offsets(cu_seqlens)
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_forward_packed(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), arr,
+                                     nseq, _ptr(y), _ptr(h_final), _ptr(topk_idx), _ptr(topk_w), wp, wb,
+                                     _stream(stream))
     if check and rc != OK:
         h._raise(rc)
     return rc

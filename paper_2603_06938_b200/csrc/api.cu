@@ -631,6 +631,122 @@ int swimba_forward(swimba_handle *h, const swimba_weights *w, const void *u, con
     return rc;
 }
 
+namespace {
+// Workspace of the packed forward: the forward's regions for T tokens, with the SSD region sized for
+// the packed batch.
+FwdLayout packed_fwd_layout(const swimba_config &c, const int32_t *cu, int nseq, int sm_count)
+{
+    const int64_t T = cu[nseq];
+    FwdLayout l = fwd_layout(c, 1, (int)(T > 0 ? T : 1), sm_count);
+    size_t off = l.ssd;
+    if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+        off += align_up(ssd_packed_workspace_bytes(cu, nseq, c.n_heads, c.n_groups, c.chunk, sm_count));
+    l.total = off;
+    return l;
+}
+bool packed_offsets_ok(const int32_t *cu, int nseq)
+{
+    if (!cu || nseq < 0 || cu[0] != 0) return false;
+    for (int b = 0; b < nseq; ++b)
+        if (cu[b + 1] < cu[b]) return false;
+    return true;
+}
+}  // namespace
+
+size_t swimba_packed_workspace_bytes(const swimba_handle *h, const int32_t *cu_seqlens, int32_t nseq)
+{
+    if (!h || nseq <= 0 || !packed_offsets_ok(cu_seqlens, nseq) || cu_seqlens[nseq] <= 0) return 0;
+    return packed_fwd_layout(h->cfg, cu_seqlens, nseq, h->sm_count).total;
+}
+
+int32_t swimba_packed_segments(const swimba_handle *h, const int32_t *cu_seqlens, int32_t nseq)
+{
+    if (!h || nseq <= 0 || !packed_offsets_ok(cu_seqlens, nseq)) return 0;
+    const swimba_config &c = h->cfg;
+    if (!ssd_tiles_supported(c.dtype, c.head_dim, c.d_state)) return nseq;
+    return ssd_packed_segments(cu_seqlens, nseq, c.n_heads, c.n_groups, c.chunk, h->sm_count);
+}
+
+int swimba_forward_packed(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                          const float *dt, const float *h0, const int32_t *cu_seqlens, int32_t nseq,
+                          void *y, float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,
+                          size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    if (nseq < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative number of sequences");
+    if (nseq > 0 && !cu_seqlens) return fail(h, SWIMBA_ERR_NULL_ARG, "cu_seqlens is NULL");
+    if (nseq > 0 && !packed_offsets_ok(cu_seqlens, nseq))
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "cu_seqlens must start at 0 and never decrease");
+    const int64_t T = nseq > 0 ? cu_seqlens[nseq] : 0;
+    if (T * h->cfg.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (T * top_k must stay below 2^31)");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (nseq == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (T > 0 && (!u || !x || !y || !workspace)) return fail(h, SWIMBA_ERR_NULL_ARG, "u, x, y or workspace is NULL");
+    if (!aligned16(u) || !aligned16(x) || !aligned16(y) || !aligned16(dt) || !aligned16(h0) ||
+        !aligned16(h_final) || !aligned16(topk_idx) || !aligned16(topk_w) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const swimba_config &c = h->cfg;
+    const FwdLayout l = packed_fwd_layout(c, cu_seqlens, nseq, h->sm_count);
+    if (T > 0 && workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    const size_t PN = (size_t)c.n_heads * c.head_dim * c.d_state;
+    if (T == 0) {
+        // nothing but empty sequences: every state passes through
+        if (h_final) {
+            const cudaError_t e = h0 ? cudaMemcpyAsync(h_final, h0, (size_t)nseq * PN * sizeof(float), cudaMemcpyDeviceToDevice, ctx.stream)
+                                     : cudaMemsetAsync(h_final, 0, (size_t)nseq * PN * sizeof(float), ctx.stream);
+            if (e != cudaSuccess) return fail(h, SWIMBA_ERR_CUDA, "copying the states failed");
+        }
+        h->last_stream = ctx.stream;
+        h->last_launches = 0;
+        return SWIMBA_OK;
+    }
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    void *BC = ws + l.bc;
+    // routing, projection and mix are per token: the packed batch is one run of T tokens
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.gemm);
+    if (rc == SWIMBA_OK) {
+        if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state)) {
+            rc = launch_ssd_tiles_packed(ctx, x, BC, dt, w->A, w->dt_bias, w->D, h0, cu_seqlens, nseq, c.n_heads,
+                                         c.n_groups, c.chunk, h->sm_count, y, h_final, ws + l.ssd);
+            if (rc != SWIMBA_OK) rc = fail(h, rc, "SSD tile kernel launch failed");
+        } else {
+            // per-timestep evaluation, sequence by sequence
+            const size_t es = elt_size(c.dtype);
+            const size_t HP = (size_t)c.n_heads * c.head_dim, S = 2u * c.n_groups * c.d_state;
+            for (int b = 0; b < nseq && rc == SWIMBA_OK; ++b) {
+                const size_t t0 = (size_t)cu_seqlens[b];
+                const int len = cu_seqlens[b + 1] - cu_seqlens[b];
+                float *hf = h_final ? h_final + (size_t)b * PN : nullptr;
+                const float *hin = h0 ? h0 + (size_t)b * PN : nullptr;
+                if (len == 0) {
+                    if (hf) {
+                        const cudaError_t e = hin ? cudaMemcpyAsync(hf, hin, PN * sizeof(float), cudaMemcpyDeviceToDevice, ctx.stream)
+                                                  : cudaMemsetAsync(hf, 0, PN * sizeof(float), ctx.stream);
+                        if (e != cudaSuccess) rc = fail(h, SWIMBA_ERR_CUDA, "copying a state failed");
+                    }
+                    continue;
+                }
+                rc = launch_ssd_sequential(ctx, c.dtype, (const char *)x + t0 * HP * es, (const char *)BC + t0 * S * es,
+                                           false, dt ? dt + t0 * c.n_heads : nullptr, w->A, w->dt_bias, w->D, hin, 1,
+                                           len, c.n_heads, c.head_dim, c.d_state, c.n_groups,
+                                           (char *)y + t0 * HP * es, hf);
+                if (rc != SWIMBA_OK) rc = fail(h, rc, "SSD launch failed");
+            }
+        }
+    }
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
                        const float *dt, float *state, int32_t B, void *y, int32_t *topk_idx,
                        float *topk_w, void *workspace, size_t workspace_bytes, void *cuda_stream)

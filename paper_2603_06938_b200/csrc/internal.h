@@ -69,6 +69,15 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
                      int chunk, int sm_count, void *y, float *h_final, void *workspace,
                      bool scalars_done);
 
+// The same over a packed batch: nseq sequences back to back in [T, ...] arrays, sequence b holding
+// tokens cu[b] .. cu[b+1]-1 (cu is a HOST array of nseq + 1 entries, read before the call returns).
+// h0 / h_final are [nseq, H, P, N].  The step sizes are produced inside the call.
+size_t ssd_packed_workspace_bytes(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count);
+int ssd_packed_segments(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count);
+int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                            const float *dt_bias, const float *D, const float *h0, const int32_t *cu, int nseq,
+                            int H, int G, int chunk, int sm_count, void *y, float *h_final, void *workspace);
+
 // One warp waiting on a barrier nobody signals, with the given limit (see swimba_selftest_wait).
 // out_dev: three 64-bit words on the device.
 int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev);

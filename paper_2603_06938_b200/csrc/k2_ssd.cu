@@ -30,6 +30,8 @@
 // Long sequences with few (sequence, head) pairs are cut into segments: a first pass of this
 // kernel computes every segment's local end state (MMA 4 only), segment_scan_kernel (K3) chains
 // them, and a second pass evaluates each segment from its true incoming state.
+#include <vector>
+
 #include "internal.h"
 #include "ssd_scalars.cuh"
 #include "tc05.cuh"
@@ -62,6 +64,11 @@ constexpr uint32_t TM_Y = 128, TM_DH = 256, TM_M = 384;
 
 enum { MODE_FULL = 0, MODE_STATE_ONLY = 1 };
 
+struct SeqDesc {            // one sequence of a packed batch
+    int tok0, len;          // first token in the packed arrays, tokens
+    int tile0, seg0;        // first 128-token tile / first segment of the sequence in the batch-wide lists
+};
+
 struct SsdParams {
     const float *l2;        // [B,H,Lpad] log2-decay accumulated inside the 128-token tile
     const TileScalars *rec; // [B,H,Lpad/128] per-tile weights and block ends
@@ -74,6 +81,16 @@ struct SsdParams {
     int split_tiles;        // > 0 (MODE_FULL, nseg == 1): every (sequence, head pair) is worked by two
                             // CTAs, see ssd_tiles_kernel
     int *d_status;
+    // Packed batch (sequences of different lengths back to back in one [T, ...] array): seqs has one
+    // entry per sequence plus a closing one, items lists the (sequence, segment) pairs of this launch
+    // (grid.x), the scalar arrays are laid out [H, tiles of the batch], and the per-segment state
+    // arrays are indexed by seqs[b].seg0 + segment.  seg_states: h_in / state-only h_out are those
+    // per-segment arrays (else h_in is [sequences, H, P, N]).  y: base of the output (ragged last
+    // tiles are stored row by row).  Null seqs: dense [B, L].
+    const SeqDesc *seqs;
+    const int2 *items;
+    int ntile_total, seg_states;
+    void *y;
 };
 
 struct __align__(8) HeadBars {
@@ -222,8 +239,23 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     // those first tiles.  No CTA waits for another.
     constexpr bool split = SPLIT;                                // (prm.split_tiles > 0)
     const bool head_part = split && blockIdx.z == 1;             // y of the leading tiles only
-    const int seg = split ? 0 : blockIdx.x, b = split ? blockIdx.x : blockIdx.z;
-    const int L = prm.L, H = prm.H;
+    const bool packed = !SPLIT && prm.seqs != nullptr;
+    int seg = split ? 0 : blockIdx.x, b = split ? blockIdx.x : blockIdx.z;
+    int L = prm.L, nseg = prm.nseg, tok0 = 0, bco = b;
+    const int H = prm.H;
+    int seg_base = b * prm.nseg;                     // index of the sequence's first segment
+    int64_t rec_base = (int64_t)b * H * (prm.Lpad / ST);   // tile record of head 0, tile 0: + h * rec_hstride
+    int rec_hstride = prm.Lpad / ST;
+    if (packed) {
+        const int2 it = prm.items[blockIdx.x];
+        b = it.x; seg = it.y;
+        const SeqDesc sd = prm.seqs[b];
+        L = sd.len; tok0 = sd.tok0; bco = 0;
+        seg_base = sd.seg0;
+        nseg = prm.seqs[b + 1].seg0 - sd.seg0;
+        rec_base = sd.tile0;
+        rec_hstride = prm.ntile_total;
+    }
     const int HG = H / prm.G, ppg = pairs_per_group(H, prm.G);
     const int g = blockIdx.y / ppg, pr = blockIdx.y % ppg;
     const int head0 = g * HG + pr * NHD;
@@ -284,33 +316,32 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         // ------------------------------------------------------------------ TMA producer
         // (the whole warp runs the loop; one elected lane issues the copies)
         const bool leader = tc::elect_one();
-        const int ntile_seq = prm.Lpad / ST;
         // record of tile t_begin / ST + j of head head0 + hd
         auto scal_rec = [&](int hd, int j) {
-            return prm.rec + ((int64_t)b * H + head0 + hd) * ntile_seq + t_begin / ST + j;
+            return prm.rec + rec_base + (int64_t)(head0 + hd) * rec_hstride + t_begin / ST + j;
         };
-        if (leader) {
+        if (leader && ntiles > 0) {
             for (int hd = 0; hd < nh; ++hd) {               // X and scalars of tile 0
                 HeadBars *hb = &bars->hd[hd];
                 tc::mbar_arrive_expect_tx(&hb->x_full[0], SLAB);
                 tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES, &tmap_x, &hb->x_full[0], 0,
-                                head0 + hd, t_begin, b);
+                                head0 + hd, tok0 + t_begin, bco);
                 tc::mbar_arrive_expect_tx(&hb->sc_full, (uint32_t)sizeof(TileScalars));
                 tc::bulk_load(&sm->sc[hd], scal_rec(hd, 0), (uint32_t)sizeof(TileScalars), &hb->sc_full);
             }
         }
         for (int j = 0; j < ntiles; ++j) {
-            const int t0 = t_begin + j * ST;
+            const int t0 = tok0 + t_begin + j * ST;
             const bool full = SPLIT ? (kfull && j >= n_pre) : kfull;
             tc::mbar_wait(&bars->cb_empty, (j & 1) ^ 1, abort_flag, d_status);
             if (leader) {
                 tc::mbar_arrive_expect_tx(&bars->cb_full, full ? 4 * SLAB : 2 * SLAB);
                 if (full) {
-                    tc::tma_load_3d(smem + SM_CB + 0 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN, t0, b);
-                    tc::tma_load_3d(smem + SM_CB + 1 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN + 64, t0, b);
+                    tc::tma_load_3d(smem + SM_CB + 0 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN, t0, bco);
+                    tc::tma_load_3d(smem + SM_CB + 1 * SLAB, &tmap_bc, &bars->cb_full, (prm.G + g) * SN + 64, t0, bco);
                 }
-                tc::tma_load_3d(smem + SM_CB + 2 * SLAB, &tmap_bc, &bars->cb_full, g * SN, t0, b);
-                tc::tma_load_3d(smem + SM_CB + 3 * SLAB, &tmap_bc, &bars->cb_full, g * SN + 64, t0, b);
+                tc::tma_load_3d(smem + SM_CB + 2 * SLAB, &tmap_bc, &bars->cb_full, g * SN, t0, bco);
+                tc::tma_load_3d(smem + SM_CB + 3 * SLAB, &tmap_bc, &bars->cb_full, g * SN + 64, t0, bco);
             }
             if (j + 1 < ntiles) {                            // X one tile ahead
                 const int jn = j + 1, sx = jn & 1;
@@ -320,7 +351,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                     if (leader) {
                         tc::mbar_arrive_expect_tx(&hb->x_full[sx], SLAB);
                         tc::tma_load_4d(smem + SM_HEAD + hd * SM_HEAD_BYTES + sx * SLAB, &tmap_x,
-                                        &hb->x_full[sx], 0, head0 + hd, t0 + ST, b);
+                                        &hb->x_full[sx], 0, head0 + hd, t0 + ST, bco);
                     }
                 }
                 // scalars of the next tile: the record buffer is single; its last readers are the
@@ -447,9 +478,11 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                 if (full) {
                     // the staged y tile goes out as one TMA store (rows past the end of the
                     // sequence are clipped by the tensor map)
+                    // (packed batch: a tile that runs past the end of its sequence is stored row by row
+                    // by the compute warps, the rows behind it belong to the next sequence)
                     tc::mbar_wait(&hb->y_staged, jf & 1, abort_flag, d_status);
-                    if (leader) {
-                        tc::tma_store_4d(&tmap_y, s_y, 0, head0 + hd, t_begin + j * ST, b);
+                    if (leader && !(packed && t_begin + (j + 1) * ST > L)) {
+                        tc::tma_store_4d(&tmap_y, s_y, 0, head0 + hd, tok0 + t_begin + j * ST, bco);
                         tc::bulk_commit_group();
                     }
                     __syncwarp();
@@ -476,8 +509,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         {
             const float *h_in = prm.h_in;
             if (h_in && kfull) {
-                const int64_t base = prm.nseg > 1
-                    ? ((((int64_t)b * prm.nseg + seg) * H + h) * SP) * SN
+                const int64_t base = prm.seg_states
+                    ? ((((int64_t)seg_base + seg) * H + h) * SP) * SN
                     : (((int64_t)b * H + h) * SP) * SN;
 #pragma unroll
                 for (int q = 0; q < 32; ++q) Hst[q] = h_in[base + (int64_t)(p0 + q) * SN + i];
@@ -508,8 +541,9 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
             }
         }
         float seg_l2 = 0.f;      // log2 of the product of a_t over the tiles done so far
-        const float *l2p = prm.l2 + ((int64_t)b * H + h) * prm.Lpad + t_begin;
-        float l2_next = l2p[i];
+        const int64_t rec_row = rec_base + (int64_t)h * rec_hstride;     // tile 0 of this (sequence, head)
+        const float *l2p = prm.l2 + rec_row * ST + t_begin;
+        float l2_next = ntiles > 0 ? l2p[i] : 0.f;
         // A run of state-only tiles (a whole segment in the state-only pass, the lead of a split
         // launch) is one long contraction: with every token weighted by its decay up to the END OF
         // THE RUN (exponent <= 0), Btilde^T (w . X) accumulates over all tiles of the run in tensor
@@ -518,7 +552,7 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         const int run_end = kfull ? n_pre : ntiles;
         float run_total = 0.f;   // log2 decay over the whole run
         {
-            const TileScalars *rec0 = prm.rec + ((int64_t)b * H + h) * (prm.Lpad / ST) + t_begin / ST;
+            const TileScalars *rec0 = prm.rec + rec_row + t_begin / ST;
             for (int jr = 0; jr < run_end; ++jr) run_total += rec0[jr].ends[3];
         }
         float run_done = 0.f;    // ... over the tiles of the run up to and including the current one
@@ -695,6 +729,11 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
                                                    fmaf(Dh, x1, __uint_as_float(yd[e0 + 1])));
                         }
                         *reinterpret_cast<uint4 *>(s_y + off) = make_uint4(o[0], o[1], o[2], o[3]);
+                        if (packed && t_begin + (j + 1) * ST > L && t_begin + j * ST + i < L) {
+                            __nv_bfloat16 *yrow = reinterpret_cast<__nv_bfloat16 *>(prm.y) +
+                                ((int64_t)(tok0 + t_begin + j * ST + i) * H + h) * SP;
+                            *reinterpret_cast<uint4 *>(yrow + p0 + 16 * hh + 8 * c2) = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
                     }
                 }
                 tc::tc_fence_before();
@@ -709,16 +748,16 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 
         // ---- final state of the segment
         if (kfull) {
-            if (prm.h_out && seg == prm.nseg - 1 && !head_part) {
+            if (prm.h_out && seg == nseg - 1 && !head_part) {
                 float *dst = prm.h_out + (((int64_t)b * H + h) * SP) * SN;
 #pragma unroll
                 for (int q = 0; q < 32; ++q) dst[(int64_t)(p0 + q) * SN + i] = Hst[q];
             }
         } else {
-            float *dst = prm.h_out + ((((int64_t)b * prm.nseg + seg) * H + h) * SP) * SN;
+            float *dst = prm.h_out + ((((int64_t)seg_base + seg) * H + h) * SP) * SN;
 #pragma unroll
             for (int q = 0; q < 32; ++q) dst[(int64_t)(p0 + q) * SN + i] = Hst[q];
-            if (i == 0 && hf == 0) prm.seg_decay[((int64_t)b * prm.nseg + seg) * H + h] = tc::ex2_approx(seg_l2);
+            if (i == 0 && hf == 0) prm.seg_decay[((int64_t)seg_base + seg) * H + h] = tc::ex2_approx(seg_l2);
         }
     }
     tc::tc_fence_before();
@@ -730,13 +769,19 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 // zero initial state) on entry and the state ENTERING segment s on exit:
 //   H_in(0) = h0,   H_in(s+1) = decay(s) H_in(s) + S(s).
 // One thread per 4 consecutive state entries; segments are walked in order.
+// (packed batch: sequence b owns segments seqs[b].seg0 .. seqs[b+1].seg0 - 1 of the batch-wide list)
 __global__ void __launch_bounds__(256)
 segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_decay,
-                    const float *__restrict__ h0, int nseg, int H, int PN4)
+                    const float *__restrict__ h0, int nseg, int H, int PN4, const SeqDesc *__restrict__ seqs)
 {
     const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // float4 index inside [P*N/4]
     const int h = blockIdx.y, b = blockIdx.z;
     if (v >= PN4) return;
+    int64_t sb = (int64_t)b * nseg;
+    if (seqs) {
+        sb = seqs[b].seg0;
+        nseg = seqs[b + 1].seg0 - seqs[b].seg0;
+    }
     float4 run = h0 ? reinterpret_cast<const float4 *>(h0)[((int64_t)b * H + h) * PN4 + v]
                     : make_float4(0.f, 0.f, 0.f, 0.f);
     // the loads do not depend on the running state: four segments are fetched at a time
@@ -748,15 +793,15 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
         for (int q = 0; q < U; ++q) {
             const int s = s0 + q;
             if (s < nseg) {
-                loc[q] = reinterpret_cast<const float4 *>(states)[(((int64_t)b * nseg + s) * H + h) * PN4 + v];
-                d[q] = seg_decay[((int64_t)b * nseg + s) * H + h];
+                loc[q] = reinterpret_cast<const float4 *>(states)[((sb + s) * H + h) * PN4 + v];
+                d[q] = seg_decay[(sb + s) * H + h];
             }
         }
 #pragma unroll
         for (int q = 0; q < U; ++q) {
             const int s = s0 + q;
             if (s < nseg) {
-                reinterpret_cast<float4 *>(states)[(((int64_t)b * nseg + s) * H + h) * PN4 + v] = run;
+                reinterpret_cast<float4 *>(states)[((sb + s) * H + h) * PN4 + v] = run;
                 run.x = fmaf(d[q], run.x, loc[q].x);
                 run.y = fmaf(d[q], run.y, loc[q].y);
                 run.z = fmaf(d[q], run.z, loc[q].z);
@@ -896,6 +941,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
     p.D = D;
     p.L = L; p.Lpad = Lpad; p.H = H; p.G = G; p.nseg = nseg; p.seg_len = seg_len;
     p.d_status = ctx.d_status;
+    p.seqs = nullptr; p.items = nullptr; p.ntile_total = 0; p.seg_states = nseg > 1; p.y = y;
     dim3 grid((unsigned)nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
     p.split_tiles = 0;
     if (nseg == 1) {
@@ -918,11 +964,179 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
         segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
-            states, decay, h0, nseg, H, PN4);
+            states, decay, h0, nseg, H, PN4, nullptr);
         ctx.end();
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
         launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        ctx.end();
+    }
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Packed batches: nseq sequences of different lengths back to back in [T, ...] arrays, sequence b
+// holding tokens cu[b] .. cu[b+1]-1.  Tiles start at sequence starts.  A sequence longer than the
+// segment length is cut into segments (state-only pass, segment scan, full pass, as in the dense
+// case); the segment length is the per-SM share of the batch's tiles, so that one long sequence
+// among short ones does not serialise the launch.
+namespace {
+struct PackedPlan {
+    std::vector<SeqDesc> seqs;        // nseq + 1
+    std::vector<int2> tiles;          // (first token, valid tokens) per tile
+    std::vector<int2> items, pre;     // (sequence, segment): all of them / those whose end state the scan needs
+    int total_tiles = 0, total_segs = 0, seg_len = 0;
+    bool segmented = false;
+};
+
+PackedPlan packed_plan(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count)
+{
+    PackedPlan pl;
+    int64_t tiles = 0;
+    for (int b = 0; b < nseq; ++b) tiles += ceil_div(cu[b + 1] - cu[b], ST);
+    const int64_t pairs = (int64_t)G * pairs_per_group(H, G);
+    const int q_tiles = chunk >= ST ? chunk / ST : 1;
+    int64_t seg_tiles = ceil_div64(tiles * pairs, sm_count);
+    if (seg_tiles < 4) seg_tiles = 4;
+    seg_tiles = ceil_div64(seg_tiles, q_tiles) * q_tiles;
+    if (seg_tiles > (1 << 22)) seg_tiles = 1 << 22;
+    pl.seg_len = (int)seg_tiles * ST;
+    pl.seqs.resize((size_t)nseq + 1);
+    int tile0 = 0, seg0 = 0;
+    for (int b = 0; b < nseq; ++b) {
+        const int len = cu[b + 1] - cu[b];
+        const int nt = ceil_div(len, ST);
+        const int ns = len > 0 ? ceil_div(len, pl.seg_len) : 1;
+        pl.seqs[b] = SeqDesc{cu[b], len, tile0, seg0};
+        for (int t = 0; t < nt; ++t)
+            pl.tiles.push_back(make_int2(cu[b] + t * ST, len - t * ST < ST ? len - t * ST : ST));
+        for (int sgi = 0; sgi < ns; ++sgi) {
+            pl.items.push_back(make_int2(b, sgi));
+            if (sgi + 1 < ns) pl.pre.push_back(make_int2(b, sgi));
+        }
+        if (ns > 1) pl.segmented = true;
+        tile0 += nt;
+        seg0 += ns;
+    }
+    pl.seqs[nseq] = SeqDesc{cu[nseq], 0, tile0, seg0};
+    pl.total_tiles = tile0;
+    pl.total_segs = seg0;
+    return pl;
+}
+
+struct PackedLayout {
+    size_t seqs, tiles, items, pre, l2, rec, states, decay, total;
+};
+PackedLayout packed_layout(const PackedPlan &pl, int nseq, int H)
+{
+    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+    PackedLayout l;
+    size_t off = 0;
+    l.seqs = off;  off += up(((size_t)nseq + 1) * sizeof(SeqDesc));
+    l.tiles = off; off += up((size_t)pl.total_tiles * sizeof(int2));
+    l.items = off; off += up(pl.items.size() * sizeof(int2));
+    l.pre = off;   off += up(pl.pre.size() * sizeof(int2));
+    l.l2 = off;    off += up((size_t)H * pl.total_tiles * ST * sizeof(float));
+    l.rec = off;   off += up((size_t)H * pl.total_tiles * sizeof(TileScalars));
+    l.states = off;
+    if (pl.segmented) off += up((size_t)pl.total_segs * H * SP * SN * sizeof(float));
+    l.decay = off;
+    if (pl.segmented) off += up((size_t)pl.total_segs * H * sizeof(float));
+    l.total = off;
+    return l;
+}
+}  // namespace
+
+size_t ssd_packed_workspace_bytes(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count)
+{
+    const PackedPlan pl = packed_plan(cu, nseq, H, G, chunk, sm_count);
+    return packed_layout(pl, nseq, H).total;
+}
+
+int ssd_packed_segments(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count)
+{
+    return packed_plan(cu, nseq, H, G, chunk, sm_count).total_segs;
+}
+
+int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                            const float *dt_bias, const float *D, const float *h0, const int32_t *cu, int nseq,
+                            int H, int G, int chunk, int sm_count, void *y, float *h_final, void *workspace)
+{
+    const int64_t T = cu[nseq];
+    if (nseq <= 0 || T <= 0) return SWIMBA_OK;
+    const PackedPlan pl = packed_plan(cu, nseq, H, G, chunk, sm_count);
+    const PackedLayout lay = packed_layout(pl, nseq, H);
+    char *ws = (char *)workspace;
+    // the tables go to the device in stream order (the copies read host memory before returning)
+    if (cudaMemcpyAsync(ws + lay.seqs, pl.seqs.data(), pl.seqs.size() * sizeof(SeqDesc), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess ||
+        cudaMemcpyAsync(ws + lay.tiles, pl.tiles.data(), pl.tiles.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess ||
+        cudaMemcpyAsync(ws + lay.items, pl.items.data(), pl.items.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess ||
+        (!pl.pre.empty() &&
+         cudaMemcpyAsync(ws + lay.pre, pl.pre.data(), pl.pre.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess))
+        return SWIMBA_ERR_CUDA;
+
+    const int S = 2 * G * SN;
+    CUtensorMap tm_bc, tm_x, tm_y;
+    {
+        const uint64_t dims[3] = {(uint64_t)S, (uint64_t)T, 1};
+        const uint64_t str[2] = {(uint64_t)S * 2, (uint64_t)T * S * 2};
+        const uint32_t box[3] = {64, ST, 1};
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_bc, BC, 3, dims, str, box)) return SWIMBA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[4] = {(uint64_t)SP, (uint64_t)H, (uint64_t)T, 1};
+        const uint64_t str[3] = {(uint64_t)SP * 2, (uint64_t)H * SP * 2, (uint64_t)T * H * SP * 2};
+        const uint32_t box[4] = {SP, 1, ST, 1};
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_x, x, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_y, y, 4, dims, str, box)) return SWIMBA_ERR_CUDA;
+    }
+    const size_t smem = ssd_smem_bytes();
+    if (!ensure_dynamic_smem((const void *)ssd_tiles_kernel<false>, smem)) return SWIMBA_ERR_CUDA;
+
+    ScalarsArgs sa;
+    sa.dt = dt; sa.A = A; sa.dt_bias = dt_bias;
+    sa.l2 = (float *)(ws + lay.l2);
+    sa.rec = (TileScalars *)(ws + lay.rec);
+    sa.L = (int)T; sa.Lpad = pl.total_tiles * ST; sa.H = H; sa.B = 1;
+    sa.tile_tab = (const int2 *)(ws + lay.tiles);
+    int rc = launch_ssd_scalars(ctx, sa);
+    if (rc != SWIMBA_OK) return rc;
+
+    SsdParams p;
+    p.l2 = sa.l2; p.rec = sa.rec; p.D = D;
+    p.L = 0; p.Lpad = sa.Lpad; p.H = H; p.G = G; p.nseg = 1; p.seg_len = pl.seg_len;
+    p.split_tiles = 0;
+    p.d_status = ctx.d_status;
+    p.seqs = (const SeqDesc *)(ws + lay.seqs);
+    p.ntile_total = pl.total_tiles;
+    p.y = y;
+    const unsigned pairs = (unsigned)(G * pairs_per_group(H, G));
+    if (!pl.segmented) {
+        p.items = (const int2 *)(ws + lay.items);
+        p.h_in = h0; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL; p.seg_states = 0;
+        ctx.begin(STAGE_SSD_TILES);
+        launch_kernel(ssd_tiles_kernel<false>, dim3((unsigned)pl.items.size(), pairs, 1), dim3(SSD_THREADS), smem,
+                      ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        ctx.end();
+    } else {
+        float *states = (float *)(ws + lay.states);
+        float *decay = (float *)(ws + lay.decay);
+        p.items = (const int2 *)(ws + lay.pre);
+        p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY; p.seg_states = 1;
+        ctx.begin(STAGE_SSD_TILES);
+        launch_kernel(ssd_tiles_kernel<false>, dim3((unsigned)pl.pre.size(), pairs, 1), dim3(SSD_THREADS), smem,
+                      ctx.stream, true, tm_bc, tm_x, tm_y, p);
+        ctx.end();
+        const int PN4 = SP * SN / 4;
+        ctx.begin(STAGE_SEGMENT_SCAN);
+        segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)nseq), 256, 0, ctx.stream>>>(
+            states, decay, h0, 0, H, PN4, p.seqs);
+        ctx.end();
+        p.items = (const int2 *)(ws + lay.items);
+        p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
+        ctx.begin(STAGE_SSD_TILES);
+        launch_kernel(ssd_tiles_kernel<false>, dim3((unsigned)pl.items.size(), pairs, 1), dim3(SSD_THREADS), smem,
+                      ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     }
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;

@@ -31,6 +31,10 @@ struct ScalarsArgs {
     float *l2;            // null: nothing to do
     TileScalars *rec;
     int L, Lpad, H, B;
+    // packed batch (sequences of different lengths back to back): per 128-token tile of the batch,
+    // (first token, valid tokens); tiles start at sequence starts.  dt is then [T, H], the arrays
+    // are laid out [H, tiles] and Lpad = 128 * tiles, B = 1.  Null: dense [B, L].
+    const int2 *tile_tab = nullptr;
 };
 
 __host__ __device__ inline int64_t scalars_units(const ScalarsArgs &a)
@@ -49,7 +53,7 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
     const int ntile = a.Lpad / SCALARS_TILE;
     const int64_t nunits = scalars_units(a);
     float raw[NU][4];
-    int hh[NU], tt[NU];
+    int hh[NU], nleft[NU];
     int64_t out[NU];
 #pragma unroll
     for (int q = 0; q < NU; ++q) {
@@ -58,13 +62,20 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
         const int tile = act ? (int)(unit % ntile) : 0;
         const int h = act ? (int)((unit / ntile) % a.H) : 0;
         const int64_t b = act ? unit / ((int64_t)ntile * a.H) : 0;
-        const int t = tile * SCALARS_TILE + lane * 4;
+        // first token of the lane's four in dt, and tokens of the tile that exist from there on
+        int64_t tok = b * a.L + tile * SCALARS_TILE + lane * 4;
+        int left = a.L - (tile * SCALARS_TILE + lane * 4);
+        if (a.tile_tab && act) {
+            const int2 tt2 = a.tile_tab[tile];
+            tok = (int64_t)tt2.x + lane * 4;
+            left = tt2.y - lane * 4;
+        }
         hh[q] = h;
-        tt[q] = t;
+        nleft[q] = left;
         out[q] = act ? (b * a.H + h) * ntile + tile : -1;        // record index
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-            raw[q][i] = (act && a.dt && t + i < a.L) ? a.dt[(b * a.L + t + i) * a.H + h] : 0.f;
+            raw[q][i] = (act && a.dt && i < left) ? a.dt[(tok + i) * a.H + h] : 0.f;
     }
 #pragma unroll
     for (int q = 0; q < NU; ++q) {
@@ -74,7 +85,7 @@ __device__ __forceinline__ void ssd_scalars_warp(const ScalarsArgs &a, int64_t u
         float d[4], p[4], run = 0.f;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            d[i] = tt[q] + i < a.L ? softplus_f(raw[q][i] + bias) : 0.f;
+            d[i] = i < nleft[q] ? softplus_f(raw[q][i] + bias) : 0.f;
             run += d[i] * a2;
             p[i] = run;
         }
