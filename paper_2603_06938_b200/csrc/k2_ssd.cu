@@ -772,7 +772,8 @@ ssd_tiles_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 // (packed batch: sequence b owns segments seqs[b].seg0 .. seqs[b+1].seg0 - 1 of the batch-wide list)
 __global__ void __launch_bounds__(256)
 segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_decay,
-                    const float *__restrict__ h0, int nseg, int H, int PN4, const SeqDesc *__restrict__ seqs)
+                    const float *__restrict__ h0, int nseg, int H, int PN4, const SeqDesc *__restrict__ seqs,
+                    float *__restrict__ end_state, float *__restrict__ end_decay)
 {
     const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // float4 index inside [P*N/4]
     const int h = blockIdx.y, b = blockIdx.z;
@@ -784,6 +785,7 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
     }
     float4 run = h0 ? reinterpret_cast<const float4 *>(h0)[((int64_t)b * H + h) * PN4 + v]
                     : make_float4(0.f, 0.f, 0.f, 0.f);
+    float dtot = 1.f;
     // the loads do not depend on the running state: four segments are fetched at a time
     constexpr int U = 4;
     for (int s0 = 0; s0 < nseg; s0 += U) {
@@ -806,8 +808,49 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
                 run.y = fmaf(d[q], run.y, loc[q].y);
                 run.z = fmaf(d[q], run.z, loc[q].z);
                 run.w = fmaf(d[q], run.w, loc[q].w);
+                dtot *= d[q];
             }
         }
+    }
+    // (dense batches only) the state after the last segment and the decay over all of them
+    if (end_state) reinterpret_cast<float4 *>(end_state)[((int64_t)b * H + h) * PN4 + v] = run;
+    if (end_decay && v == 0) end_decay[(int64_t)b * H + h] = dtot;
+}
+
+// Sequence-sharded evaluation, second half.  Rank r of R holds tokens [r L, (r+1) L) of every
+// sequence; all ranks' summaries (end state from a zero entry state, decay over the shard) have been
+// gathered: gs [R, B, H, P*N], gd [R, B, H].  The state entering this rank's shard is
+//   H_in = scan over ranks r' < rank of  H <- gd[r'] H + gs[r'],  from h0,
+// and the states entering its local segments, computed from a zero entry state by the local scan,
+// gain the entry state decayed up to the segment's start: states[b,s] += (prod_{s'<s} decay[b,s']) H_in.
+__global__ void __launch_bounds__(256)
+shard_entry_kernel(float *__restrict__ states, const float *__restrict__ seg_decay, const float *__restrict__ h0,
+                   const float *__restrict__ gs, const float *__restrict__ gd, int rank, int B, int nseg, int H,
+                   int PN4)
+{
+    const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int h = blockIdx.y, b = blockIdx.z;
+    if (v >= PN4) return;
+    float4 run = h0 ? reinterpret_cast<const float4 *>(h0)[((int64_t)b * H + h) * PN4 + v]
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int r = 0; r < rank; ++r) {
+        const float d = gd[((int64_t)r * B + b) * H + h];
+        const float4 loc = reinterpret_cast<const float4 *>(gs)[(((int64_t)r * B + b) * H + h) * PN4 + v];
+        run.x = fmaf(d, run.x, loc.x);
+        run.y = fmaf(d, run.y, loc.y);
+        run.z = fmaf(d, run.z, loc.z);
+        run.w = fmaf(d, run.w, loc.w);
+    }
+    float cum = 1.f;
+    for (int sgi = 0; sgi < nseg; ++sgi) {
+        float4 *p = reinterpret_cast<float4 *>(states) + (((int64_t)b * nseg + sgi) * H + h) * PN4 + v;
+        float4 cur = *p;
+        cur.x = fmaf(cum, run.x, cur.x);
+        cur.y = fmaf(cum, run.y, cur.y);
+        cur.z = fmaf(cum, run.z, cur.z);
+        cur.w = fmaf(cum, run.w, cur.w);
+        *p = cur;
+        cum *= seg_decay[((int64_t)b * nseg + sgi) * H + h];
     }
 }
 
@@ -964,7 +1007,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
         segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
-            states, decay, h0, nseg, H, PN4, nullptr);
+            states, decay, h0, nseg, H, PN4, nullptr, nullptr, nullptr);
         ctx.end();
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
         ctx.begin(STAGE_SSD_TILES);
@@ -1130,7 +1173,7 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
         segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)nseq), 256, 0, ctx.stream>>>(
-            states, decay, h0, 0, H, PN4, p.seqs);
+            states, decay, h0, 0, H, PN4, p.seqs, nullptr, nullptr);
         ctx.end();
         p.items = (const int2 *)(ws + lay.items);
         p.h_in = states; p.h_out = h_final; p.seg_decay = nullptr; p.mode = MODE_FULL;
@@ -1139,6 +1182,128 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
                       ctx.stream, true, tm_bc, tm_x, tm_y, p);
         ctx.end();
     }
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Sequence-sharded evaluation: every rank holds L consecutive tokens of each of the B sequences.
+// First half (summary): state-only pass over the shard's segments and the local scan from a zero
+// entry state; leaves the shard's end state and total decay for the exchange, and the zero-entry
+// segment states in the workspace.  Second half (finish), after the ranks' summaries have been
+// gathered: entry state from the ranks in front, segment states corrected, full pass.
+namespace {
+struct ShardLayout {
+    size_t scal, states, decay, total;
+    int seg_len, nseg;
+};
+ShardLayout shard_layout(int B, int L, int H, int G, int chunk, int sm_count)
+{
+    ShardLayout l;
+    l.seg_len = ssd_segment_len(B, L, H, G, chunk, sm_count);
+    l.nseg = ceil_div(L, l.seg_len);
+    size_t off = 0;
+    l.scal = off;   off += ssd_scalars_bytes(B, L, H);
+    l.states = off; off += ((size_t)B * l.nseg * H * SP * SN * sizeof(float) + 255) / 256 * 256;
+    l.decay = off;  off += ((size_t)B * l.nseg * H * sizeof(float) + 255) / 256 * 256;
+    l.total = off;
+    return l;
+}
+
+bool shard_maps(LaunchCtx &ctx, const void *x, const void *BC, const void *y, int B, int L, int H, int G,
+                CUtensorMap *tm_bc, CUtensorMap *tm_x, CUtensorMap *tm_y)
+{
+    const int S = 2 * G * SN;
+    const uint64_t dims3[3] = {(uint64_t)S, (uint64_t)L, (uint64_t)B};
+    const uint64_t str3[2] = {(uint64_t)S * 2, (uint64_t)L * S * 2};
+    const uint32_t box3[3] = {64, ST, 1};
+    if (!encode_tmap_bf16_cached(ctx.tmaps, tm_bc, BC, 3, dims3, str3, box3)) return false;
+    const uint64_t dims[4] = {(uint64_t)SP, (uint64_t)H, (uint64_t)L, (uint64_t)B};
+    const uint64_t str[3] = {(uint64_t)SP * 2, (uint64_t)H * SP * 2, (uint64_t)L * H * SP * 2};
+    const uint32_t box[4] = {SP, 1, ST, 1};
+    if (!encode_tmap_bf16_cached(ctx.tmaps, tm_x, x, 4, dims, str, box)) return false;
+    // (the state-only pass stores no y; its map is a copy of x's)
+    if (!encode_tmap_bf16_cached(ctx.tmaps, tm_y, y ? y : x, 4, dims, str, box)) return false;
+    return ensure_dynamic_smem((const void *)ssd_tiles_kernel<false>, ssd_smem_bytes());
+}
+
+SsdParams shard_params(LaunchCtx &ctx, const ShardLayout &lay, int B, int L, int H, int G, void *workspace)
+{
+    SsdParams p;
+    const ScalarsArgs sa = ssd_scalars_args(nullptr, nullptr, nullptr, B, L, H, (char *)workspace + lay.scal);
+    p.l2 = sa.l2; p.rec = sa.rec;
+    p.D = nullptr;
+    p.L = L; p.Lpad = ceil_div(L, ST) * ST; p.H = H; p.G = G; p.nseg = lay.nseg; p.seg_len = lay.seg_len;
+    p.split_tiles = 0;
+    p.d_status = ctx.d_status;
+    p.seqs = nullptr; p.items = nullptr; p.ntile_total = 0; p.seg_states = 1; p.y = nullptr;
+    return p;
+}
+}  // namespace
+
+size_t ssd_shard_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count)
+{
+    return shard_layout(B, L, H, G, chunk, sm_count).total;
+}
+
+ScalarsArgs ssd_shard_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,
+                                   int G, int chunk, int sm_count, void *workspace)
+{
+    const ShardLayout lay = shard_layout(B, L, H, G, chunk, sm_count);
+    return ssd_scalars_args(dt, A, dt_bias, B, L, H, (char *)workspace + lay.scal);
+}
+
+int launch_ssd_shard_summary(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                             const float *dt_bias, int B, int L, int H, int G, int chunk, int sm_count,
+                             float *sum_state, float *sum_decay, void *workspace, bool scalars_done)
+{
+    if (B <= 0 || L <= 0) return SWIMBA_OK;
+    const ShardLayout lay = shard_layout(B, L, H, G, chunk, sm_count);
+    CUtensorMap tm_bc, tm_x, tm_y;
+    if (!shard_maps(ctx, x, BC, nullptr, B, L, H, G, &tm_bc, &tm_x, &tm_y)) return SWIMBA_ERR_CUDA;
+    if (!scalars_done) {
+        const int rc = launch_ssd_scalars(ctx, ssd_scalars_args(dt, A, dt_bias, B, L, H, (char *)workspace + lay.scal));
+        if (rc != SWIMBA_OK) return rc;
+    }
+    SsdParams p = shard_params(ctx, lay, B, L, H, G, workspace);
+    float *states = (float *)((char *)workspace + lay.states);
+    float *decay = (float *)((char *)workspace + lay.decay);
+    p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
+    const dim3 grid((unsigned)lay.nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
+    ctx.begin(STAGE_SSD_TILES);
+    launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), ssd_smem_bytes(), ctx.stream, true, tm_bc, tm_x,
+                  tm_y, p);
+    ctx.end();
+    const int PN4 = SP * SN / 4;
+    ctx.begin(STAGE_SEGMENT_SCAN);
+    segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
+        states, decay, nullptr, lay.nseg, H, PN4, nullptr, sum_state, sum_decay);
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
+int launch_ssd_shard_finish(LaunchCtx &ctx, const void *x, const void *BC, const float *D, const float *h0,
+                            const float *all_state, const float *all_decay, int rank, int B, int L, int H, int G,
+                            int chunk, int sm_count, void *y, float *h_end, void *workspace)
+{
+    if (B <= 0 || L <= 0) return SWIMBA_OK;
+    const ShardLayout lay = shard_layout(B, L, H, G, chunk, sm_count);
+    CUtensorMap tm_bc, tm_x, tm_y;
+    if (!shard_maps(ctx, x, BC, y, B, L, H, G, &tm_bc, &tm_x, &tm_y)) return SWIMBA_ERR_CUDA;
+    SsdParams p = shard_params(ctx, lay, B, L, H, G, workspace);
+    float *states = (float *)((char *)workspace + lay.states);
+    float *decay = (float *)((char *)workspace + lay.decay);
+    const int PN4 = SP * SN / 4;
+    ctx.begin(STAGE_SEGMENT_SCAN);
+    shard_entry_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
+        states, decay, h0, all_state, all_decay, rank, B, lay.nseg, H, PN4);
+    ctx.end();
+    p.D = D; p.y = y;
+    p.h_in = states; p.h_out = h_end; p.seg_decay = nullptr; p.mode = MODE_FULL;
+    const dim3 grid((unsigned)lay.nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
+    ctx.begin(STAGE_SSD_TILES);
+    launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), ssd_smem_bytes(), ctx.stream, true, tm_bc, tm_x,
+                  tm_y, p);
+    ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
 
