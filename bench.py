@@ -521,6 +521,10 @@ def main():
     if single and not args.no_serving:
         serving = bench_serving(sb)
 
+    shard = None
+    if single and not args.no_serving:
+        shard = bench_shard(sb)
+
     cpu = None
     if single and not args.no_cpu_baseline:
         cpu, _ = time_oracle_sample(cfg, cfg.B)
@@ -538,7 +542,8 @@ def main():
                        "how": "value is the median over rounds of exactly `steps` steps each"},
             "ssd_segments": nseg,
             "kernels": kernels, "comparators": comparators, "workloads": workloads,
-            "decode": decode, "serving": serving, "cpu_baseline": cpu,
+            "decode": decode, "serving": serving, "sequence_sharded": shard,
+            "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     if dist is not None:
@@ -602,6 +607,57 @@ def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
     }
     sb.swimba_destroy(h)
     return out
+
+
+def bench_shard(sb, ranks: int = 8, steps: int = 10, warmup: int = 3):
+    """One rank's compute of the sequence-sharded forward: the long_seq workload cut into `ranks` runs
+    of tokens, the two halves (swimba_shard_summary, swimba_shard_finish) timed on this device for one
+    shard, with the other ranks' summaries standing in as given arrays (the all-gather itself, about
+    1 MB per rank, is not in the figure)."""
+    cfg = synth.CONFIGS["long_seq"]
+    L = cfg.L // ranks
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(12)
+    wts = {n: v.cuda() for n, v in synth.make_weights(cfg, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    dgen = torch.Generator(device="cuda")
+    dgen.manual_seed(13)
+    nsets = 6                         # 6 x 30 MB of inputs + outputs: above L2 together
+    sets = [dict(u=torch.randn(cfg.B, L, cfg.F, generator=dgen, device="cuda").bfloat16(),
+                 x=torch.randn(cfg.B, L, cfg.H, cfg.P, generator=dgen, device="cuda").bfloat16(),
+                 dt=0.5 * torch.randn(cfg.B, L, cfg.H, generator=dgen, device="cuda")) for _ in range(nsets)]
+    ys = [torch.empty_like(s_["x"]) for s_ in sets]
+    ws = torch.empty(sb.swimba_shard_workspace_bytes(h, cfg.B, L), dtype=torch.uint8, device="cuda")
+    st = torch.empty(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
+    dc = torch.empty(cfg.B, cfg.H, device="cuda")
+    all_state = 0.01 * torch.randn(ranks, cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
+    all_decay = torch.rand(ranks, cfg.B, cfg.H, device="cuda")
+    he = torch.empty(cfg.B, cfg.H, cfg.P, cfg.N, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        s_ = sets[i % nsets]
+        sb.swimba_shard_summary(h, w, s_["u"], s_["x"], s_["dt"], cfg.B, L, st, dc, None, None, ws)
+        sb.swimba_shard_finish(h, w, s_["x"], None, all_state, all_decay, ranks - 1, ranks, cfg.B, L,
+                               ys[i % nsets], he, ws)
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    return {"workload": f"long_seq cut into {ranks} shards of {L} tokens; the last rank's shard",
+            "ms_per_shard": ms, "tokens_per_s_per_rank": cfg.B * L / (ms * 1e-3),
+            "exchange_bytes_per_rank": cfg.B * cfg.H * (cfg.P * cfg.N + 1) * 4,
+            "note": "compute of one rank (summary + finish); the all-gather between the halves is not timed"}
 
 
 def bench_serving(sb, steps: int = 10, warmup: int = 3):

@@ -164,6 +164,34 @@ int swimba_forward_packed(swimba_handle *h, const swimba_weights *w, const void 
                           void *y, float *h_final, int32_t *topk_idx, float *topk_w, void *workspace,
                           size_t workspace_bytes, void *cuda_stream);
 
+/* The layer forward with the SEQUENCE dimension sharded over n_ranks devices (one process per
+ * device): rank r holds tokens [r L, (r+1) L) of each of the B sequences, in u [B,L,F], x [B,L,H,P],
+ * dt [B,L,H].  The recurrence of Theorem 1 is linear in the state, so a shard is summarised by its
+ * end state from a ZERO entry state and the product of a_t over the shard (Background, "Mamba-2 and
+ * SSD": a linear recurrence between blocks of tokens; here the blocks are the ranks' shards).
+ *   1. swimba_shard_summary: routing, projection, mix and a state-only pass over the local shard;
+ *      writes summary_state [B,H,P,N] fp32 and summary_decay [B,H] fp32 (and the routing outputs,
+ *      [B,L,k], may be NULL).  The mixed streams and intermediate states stay in the workspace.
+ *   2. The caller gathers all ranks' summaries in rank order (one all-gather; the library holds no
+ *      communicator): all_state [n_ranks,B,H,P,N], all_decay [n_ranks,B,H].  Rank 0 may pass NULL.
+ *   3. swimba_shard_finish, with the SAME workspace, untouched in between, and the same x, B, L:
+ *      chains h0 [B,H,P,N] (the state in front of rank 0's tokens; NULL => zeros; every rank passes
+ *      the same) through the summaries of the ranks in front, produces y [B,L,H,P] of the local
+ *      shard and h_end [B,H,P,N] (may be NULL), the state after the shard's last token (on the last
+ *      rank: the sequence's final state).
+ * bf16, head_dim 64, d_state 128 only (SWIMBA_ERR_UNSUPPORTED_SHAPE otherwise; the workspace query
+ * then returns 0).  Device pointers, caller-owned, 16-byte aligned; everything is enqueued on
+ * cuda_stream; errors as swimba_forward. */
+size_t swimba_shard_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+int swimba_shard_summary(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                         const float *dt, int32_t B, int32_t L, float *summary_state, float *summary_decay,
+                         int32_t *topk_idx, float *topk_w, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream);
+int swimba_shard_finish(swimba_handle *h, const swimba_weights *w, const void *x, const float *h0,
+                        const float *all_state, const float *all_decay, int32_t rank, int32_t n_ranks,
+                        int32_t B, int32_t L, void *y, float *h_end, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream);
+
 /* The general form of the layer, with expert-specific SSM inputs (the state equation of Section
  * "MoE-parameterized SSM" as printed: h_t = A h_{t-1} + sum_{e in K_t} pi_{t,e} B_t^(e) X_t^(e)^T,
  * Y_t = (sum_{e in K_t} pi_{t,e} C_t^(e))^T h_t).  The caller's experts produce X^(e) themselves (in

@@ -31,6 +31,7 @@ FLAG_CHECK_INDICES = 1
 EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_packed_workspace_bytes", "swimba_packed_segments", "swimba_forward_packed",
+    "swimba_shard_workspace_bytes", "swimba_shard_summary", "swimba_shard_finish",
     "swimba_route_project_slots", "swimba_ssd_slots_workspace_bytes", "swimba_ssd_slots",
     "swimba_block_workspace_bytes", "swimba_block_forward",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
@@ -93,6 +94,14 @@ def lib() -> ctypes.CDLL:
         L.swimba_forward_packed.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp,
                                             ctypes.POINTER(i32), i32, vp, vp, vp, vp, vp, sz, vp]
         L.swimba_forward_packed.restype = ctypes.c_int
+        L.swimba_shard_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_shard_workspace_bytes.restype = sz
+        L.swimba_shard_summary.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, i32, i32, vp, vp,
+                                           vp, vp, vp, sz, vp]
+        L.swimba_shard_summary.restype = ctypes.c_int
+        L.swimba_shard_finish.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, i32, i32, i32,
+                                          i32, vp, vp, vp, sz, vp]
+        L.swimba_shard_finish.restype = ctypes.c_int
         L.swimba_route_mix.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, i64, vp, vp, vp, vp,
                                        sz, vp]
         L.swimba_route_mix.restype = ctypes.c_int
@@ -219,6 +228,32 @@ def swimba_forward(h: Handle, w: swimba_weights, u, x, dt, h0, B: int, L: int, y
     rc = lib().swimba_forward(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), B, L,
                               _ptr(y), _ptr(h_final), _ptr(topk_idx), _ptr(topk_w), wp, wb,
                               _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_shard_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_shard_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_shard_summary(h: Handle, w: swimba_weights, u, x, dt, B: int, L: int, summary_state,
+                         summary_decay, topk_idx, topk_w, workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_shard_summary(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), B, L,
+                                    _ptr(summary_state), _ptr(summary_decay), _ptr(topk_idx), _ptr(topk_w),
+                                    wp, wb, _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_shard_finish(h: Handle, w: swimba_weights, x, h0, all_state, all_decay, rank: int, n_ranks: int,
+                        B: int, L: int, y, h_end, workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_shard_finish(h.ptr, ctypes.byref(w), _ptr(x), _ptr(h0), _ptr(all_state),
+                                   _ptr(all_decay), rank, n_ranks, B, L, _ptr(y), _ptr(h_end), wp, wb,
+                                   _stream(stream))
     if check and rc != OK:
         h._raise(rc)
     return rc

@@ -747,6 +747,100 @@ int swimba_forward_packed(swimba_handle *h, const swimba_weights *w, const void 
     return rc;
 }
 
+namespace {
+// Workspace of the sequence-sharded forward: the forward's token regions, then the shard's SSD region.
+FwdLayout shard_fwd_layout(const swimba_config &c, int B, int L, int sm_count)
+{
+    FwdLayout l = fwd_layout(c, B, L, sm_count);
+    l.total = l.ssd + align_up(ssd_shard_workspace_bytes(B, L, c.n_heads, c.n_groups, c.chunk, sm_count));
+    return l;
+}
+}  // namespace
+
+size_t swimba_shard_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    if (!ssd_tiles_supported(h->cfg.dtype, h->cfg.head_dim, h->cfg.d_state)) return 0;
+    return shard_fwd_layout(h->cfg, B, L, h->sm_count).total;
+}
+
+int swimba_shard_summary(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                         const float *dt, int32_t B, int32_t L, float *summary_state, float *summary_decay,
+                         int32_t *topk_idx, float *topk_w, void *workspace, size_t workspace_bytes,
+                         void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    const swimba_config &c = h->cfg;
+    if (B <= 0 || L <= 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "a shard needs B > 0 and L > 0");
+    if ((int64_t)B * L * c.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (B * L * top_k must stay below 2^31)");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
+    if (!ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "the sequence-sharded forward needs bf16, head_dim 64, d_state 128");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (!u || !x || !summary_state || !summary_decay || !workspace)
+        return fail(h, SWIMBA_ERR_NULL_ARG, "u, x, a summary output or the workspace is NULL");
+    if (!aligned16(u) || !aligned16(x) || !aligned16(dt) || !aligned16(summary_state) || !aligned16(summary_decay) ||
+        !aligned16(topk_idx) || !aligned16(topk_w) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const FwdLayout l = shard_fwd_layout(c, B, L, h->sm_count);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.idx);
+    float *wt = topk_w ? topk_w : (float *)(ws + l.w);
+    void *BC = ws + l.bc;
+    const ScalarsArgs sa = ssd_shard_scalars_args(dt, w->A, w->dt_bias, B, L, c.n_heads, c.n_groups, c.chunk,
+                                                  h->sm_count, ws + l.ssd);
+    rc = run_route_mix(h, ctx, w, u, (int64_t)B * L, BC, false, idx, wt, ws + l.gemm, &sa);
+    if (rc == SWIMBA_OK) {
+        rc = launch_ssd_shard_summary(ctx, x, BC, dt, w->A, w->dt_bias, B, L, c.n_heads, c.n_groups, c.chunk,
+                                      h->sm_count, summary_state, summary_decay, ws + l.ssd, true);
+        if (rc != SWIMBA_OK) rc = fail(h, rc, "SSD state-only pass launch failed");
+    }
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
+int swimba_shard_finish(swimba_handle *h, const swimba_weights *w, const void *x, const float *h0,
+                        const float *all_state, const float *all_decay, int32_t rank, int32_t n_ranks,
+                        int32_t B, int32_t L, void *y, float *h_end, void *workspace, size_t workspace_bytes,
+                        void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    const swimba_config &c = h->cfg;
+    if (B <= 0 || L <= 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "a shard needs B > 0 and L > 0");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
+    if (n_ranks <= 0 || rank < 0 || rank >= n_ranks) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "rank outside [0, n_ranks)");
+    if (!ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "the sequence-sharded forward needs bf16, head_dim 64, d_state 128");
+    int rc = check_weights(h, w, false);
+    if (rc != SWIMBA_OK) return rc;
+    if (!x || !y || !workspace || (rank > 0 && (!all_state || !all_decay)))
+        return fail(h, SWIMBA_ERR_NULL_ARG, "x, y, the workspace or the gathered summaries are NULL");
+    if (!aligned16(x) || !aligned16(y) || !aligned16(h0) || !aligned16(all_state) || !aligned16(all_decay) ||
+        !aligned16(h_end) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    const FwdLayout l = shard_fwd_layout(c, B, L, h->sm_count);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    char *ws = (char *)workspace;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    rc = launch_ssd_shard_finish(ctx, x, ws + l.bc, w->D, h0, all_state, all_decay, rank, B, L, c.n_heads, c.n_groups,
+                                 c.chunk, h->sm_count, y, h_end, ws + l.ssd);
+    if (rc != SWIMBA_OK) rc = fail(h, rc, "SSD full pass launch failed");
+    h->last_stream = ctx.stream;
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
                        const float *dt, float *state, int32_t B, void *y, int32_t *topk_idx,
                        float *topk_w, void *workspace, size_t workspace_bytes, void *cuda_stream)

@@ -78,6 +78,24 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
                             const float *dt_bias, const float *D, const float *h0, const int32_t *cu, int nseq,
                             int H, int G, int chunk, int sm_count, void *y, float *h_final, void *workspace);
 
+// Sequence-sharded evaluation (every rank holds L consecutive tokens of each of B sequences), in two
+// halves around the exchange of the ranks' summaries.  summary: state-only pass + local scan from a
+// zero entry state; sum_state [B,H,P,N] and sum_decay [B,H] receive the shard's end state and the
+// product of a_t over the shard; the workspace keeps the step sizes and the zero-entry segment
+// states for the second half.  finish: all_state [R,B,H,P,N] / all_decay [R,B,H] are the gathered
+// summaries in rank order; the state entering this rank's shard is chained from h0 through the
+// ranks in front, y [B,L,H,P] is produced and h_end [B,H,P,N] (may be NULL) is the state after the
+// shard's last token.
+size_t ssd_shard_workspace_bytes(int B, int L, int H, int G, int chunk, int sm_count);
+ScalarsArgs ssd_shard_scalars_args(const float *dt, const float *A, const float *dt_bias, int B, int L, int H,
+                                   int G, int chunk, int sm_count, void *workspace);
+int launch_ssd_shard_summary(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                             const float *dt_bias, int B, int L, int H, int G, int chunk, int sm_count,
+                             float *sum_state, float *sum_decay, void *workspace, bool scalars_done);
+int launch_ssd_shard_finish(LaunchCtx &ctx, const void *x, const void *BC, const float *D, const float *h0,
+                            const float *all_state, const float *all_decay, int rank, int B, int L, int H, int G,
+                            int chunk, int sm_count, void *y, float *h_end, void *workspace);
+
 // One warp waiting on a barrier nobody signals, with the given limit (see swimba_selftest_wait).
 // out_dev: three 64-bit words on the device.
 int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev);
