@@ -232,6 +232,36 @@ def swimba_forward(u, x, dt, W_r, W_e, A, dt_bias, D, k: int, G: int = 1, h0=Non
     return dict(y=y, h_final=hf, idx=idx, w=w, BC=BC)
 
 
+def backward_weights(u, x, dt, W_r, W_e, A, dt_bias, dy, k: int, G: int = 1, h0=None, forced_idx=None):
+    """Gradients of sum(dy * y) with respect to W_r [E,F] and W_e [E,S,F] (the parameters the paper
+    trains), the active sets held fixed: dict(dW_r, dW_e, dBC [B,L,S], dpi [B,L,k])."""
+    u = _d(u)
+    x = _d(x)
+    B, L, F = u.shape
+    _, _, H, P = x.shape
+    W_e = _d(W_e)
+    E, S, _ = W_e.shape
+    N = S // (2 * G)
+    if k > 64:
+        raise ValueError("k <= 64")
+    W_r = _d(W_r, (E, F))
+    dt = _d(dt, (B, L, H)) if dt is not None else None
+    A = _d(A, (H,))
+    dt_bias = _d(dt_bias, (H,))
+    h0 = _d(h0, (B, H, P, N)) if h0 is not None else None
+    dy = _d(dy, (B, L, H, P))
+    fi = _i(forced_idx).reshape(B * L, k) if forced_idx is not None else None
+    dW_r = np.zeros((E, F), np.float64)
+    dW_e = np.zeros((E, S, F), np.float64)
+    dBC = np.zeros((B, L, S), np.float64)
+    dpi = np.zeros((B, L, k), np.float64)
+    _check(_load().oracle_swimba_backward_weights(_p(u), _p(x), _p(dt), _p(h0), _p(W_r), _p(W_e), _p(A),
+                                                  _p(dt_bias), _p(dy), B, L, F, H, P, N, G, E, k, _p(fi),
+                                                  _p(dW_r), _p(dW_e), _p(dBC), _p(dpi)),
+           "oracle_swimba_backward_weights")
+    return dict(dW_r=dW_r, dW_e=dW_e, dBC=dBC, dpi=dpi)
+
+
 def swimba_decode_step(u, x, dt, W_r, W_e, A, dt_bias, D, k: int, state, G: int = 1,
                        forced_idx=None, forced_w=None):
     """One token per sequence; `state`[B,H,P,N] (float64, C-contiguous) is updated in place."""

@@ -394,6 +394,142 @@ int oracle_swimba_forward(const double *u, const double *x, const double *dt, co
 }
 
 /* ---------------------------------------------------------------------------
+ * Gradients of  loss = sum_{b,t,h,p} dy[b,t,h,p] * y[b,t,h,p]  with respect to the router matrix
+ * W_r and the expert matrices W_e (Section "Training": only the router and the expert
+ * parameters that the conversion adds are trained, the rest of the layer is frozen), by
+ * reverse-mode differentiation of oracle_swimba_forward's steps, taken in reverse order:
+ *   recurrence   lambda_t = a_{t+1} lambda_{t+1} + dy_t Ctilde_t^T      (adjoint of the state)
+ *                dCtilde_t[g,n] = sum_{h in g, p} dy_t[h,p] h_t[h,p,n]
+ *                dBtilde_t[g,n] = Delta_t sum_{h in g, p} x_t[h,p] lambda_t[h,p,n]
+ *   mix          dpi_{t,j} = <dBC_t, W_e[e_j] u_t>,   dW_e[e_j] += pi_{t,e_j} dBC_t u_t^T
+ *   softmax      dg_{t,i} = pi_{t,i} ( [i in K_t] dpi_{t,i} - sum_{j in K_t} pi_{t,j} dpi_{t,j} )
+ *   logits       dW_r += dg_t u_t^T
+ * The active sets K_t are constants of the differentiation (the selection itself has no
+ * derivative); the kept weights are the softmax values over all E, not renormalised, and are
+ * differentiated as such.  forced_idx (may be NULL) replaces the router's selection; the
+ * weights are always the softmax values of the selected experts.
+ *   Outputs: dW_r[E,F] (may be NULL when W_r is NULL and E == 1), dW_e[E,S,F]; optional
+ *   dBC[T,S], dpi[T,k].
+ * ------------------------------------------------------------------------- */
+int oracle_swimba_backward_weights(const double *u, const double *x, const double *dt,
+                                   const double *h0, const double *W_r, const double *W_e,
+                                   const double *A, const double *dt_bias, const double *dy,
+                                   int B, int L, int F, int H, int P, int N, int G, int E, int k,
+                                   const int *forced_idx, double *dW_r, double *dW_e,
+                                   double *dBC_out, double *dpi_out)
+{
+    if (!u || !x || !W_e || !W_r || !A || !dt_bias || !dy || !dW_e || !dW_r || B < 0 || L < 0 ||
+        F <= 0 || E <= 0 || k <= 0 || k > E || N <= 0 || G <= 0 || H % G != 0)
+        return ORACLE_BAD_ARG;
+    const long T = (long)B * L;
+    const int S = 2 * G * N, hpg = H / G;
+    const long PN = (long)P * N;
+    int *idx = (int *)malloc(sizeof(int) * (size_t)(T * k + 1));
+    double *w = (double *)malloc(sizeof(double) * (size_t)(T * k + 1));
+    double *pi = (double *)malloc(sizeof(double) * (size_t)(T * E + 1));
+    double *BC = (double *)malloc(sizeof(double) * (size_t)(T * S + 1));
+    double *dBC = (double *)calloc((size_t)(T * S + 1), sizeof(double));
+    double *dg = (double *)calloc((size_t)(T * E + 1), sizeof(double));
+    int rc = ORACLE_OK;
+    if (!idx || !w || !pi || !BC || !dBC || !dg) rc = ORACLE_NO_MEM;
+    if (rc == ORACLE_OK) rc = oracle_router(u, W_r, T, F, E, k, idx, w, pi, NULL, NULL);
+    if (rc == ORACLE_OK && forced_idx) {
+        memcpy(idx, forced_idx, sizeof(int) * (size_t)(T * k));
+        for (long r = 0; r < T * k; ++r) w[r] = pi[(r / k) * E + idx[r]];
+    }
+    if (rc == ORACLE_OK) rc = oracle_mix_topk(u, W_e, T, F, S, E, k, idx, w, BC);
+    int fail = 0;
+    if (rc == ORACLE_OK) {
+        /* the recurrence, one (sequence, head) at a time: forward in time for h_t, then backward
+         * in time for lambda_t */
+#pragma omp parallel for collapse(2) schedule(dynamic)
+        for (int b = 0; b < B; ++b)
+            for (int h = 0; h < H; ++h) {
+                double *st = (double *)malloc(sizeof(double) * (size_t)PN);
+                if (!st) { fail = 1; continue; }
+                const int g = h / hpg;
+                for (long i = 0; i < PN; ++i) st[i] = h0 ? h0[((long)b * H + h) * PN + i] : 0.0;
+                for (int t = 0; t < L; ++t) {
+                    const long bt = (long)b * L + t;
+                    const double *Bt = BC + bt * S + (long)g * N;
+                    const double delta = softplus((dt ? dt[bt * H + h] : 0.0) + dt_bias[h]);
+                    const double a = exp(delta * A[h]);
+                    for (int n = 0; n < N; ++n) {
+                        double acc = 0.0;
+                        for (int p = 0; p < P; ++p) {
+                            double *sp = st + (long)p * N + n;
+                            *sp = a * (*sp) + delta * x[(bt * H + h) * P + p] * Bt[n];
+                            acc += dy[(bt * H + h) * P + p] * (*sp);
+                        }
+#pragma omp atomic
+                        dBC[bt * S + (long)(G + g) * N + n] += acc;
+                    }
+                }
+                for (long i = 0; i < PN; ++i) st[i] = 0.0;          /* lambda past the last token */
+                double a_next = 0.0;
+                for (int t = L - 1; t >= 0; --t) {
+                    const long bt = (long)b * L + t;
+                    const double *Ct = BC + bt * S + (long)(G + g) * N;
+                    const double delta = softplus((dt ? dt[bt * H + h] : 0.0) + dt_bias[h]);
+                    for (int n = 0; n < N; ++n) {
+                        double acc = 0.0;
+                        for (int p = 0; p < P; ++p) {
+                            double *sp = st + (long)p * N + n;
+                            *sp = a_next * (*sp) + dy[(bt * H + h) * P + p] * Ct[n];
+                            acc += x[(bt * H + h) * P + p] * (*sp);
+                        }
+#pragma omp atomic
+                        dBC[bt * S + (long)g * N + n] += delta * acc;
+                    }
+                    a_next = exp(delta * A[h]);
+                }
+                free(st);
+            }
+        if (fail) rc = ORACLE_NO_MEM;
+    }
+    if (rc == ORACLE_OK) {
+        /* mix and softmax, token by token */
+#pragma omp parallel for schedule(static)
+        for (long t = 0; t < T; ++t) {
+            double dpi[64], inner = 0.0;
+            for (int j = 0; j < k && j < 64; ++j) {
+                const int e = idx[t * k + j];
+                double acc = 0.0;
+                for (int srow = 0; srow < S; ++srow) {
+                    double proj = 0.0;
+                    for (int f = 0; f < F; ++f) proj += W_e[((long)e * S + srow) * F + f] * u[t * F + f];
+                    acc += dBC[t * S + srow] * proj;
+                }
+                dpi[j] = acc;
+                inner += w[t * k + j] * acc;
+                if (dpi_out) dpi_out[t * k + j] = acc;
+            }
+            for (int i = 0; i < E; ++i) dg[t * E + i] = -pi[t * E + i] * inner;
+            for (int j = 0; j < k && j < 64; ++j) dg[t * E + idx[t * k + j]] += w[t * k + j] * dpi[j];
+        }
+        /* weight gradients, one expert at a time (no two threads touch the same rows) */
+#pragma omp parallel for schedule(dynamic)
+        for (int e = 0; e < E; ++e) {
+            for (long i = 0; i < (long)S * F; ++i) dW_e[(long)e * S * F + i] = 0.0;
+            for (int f = 0; f < F; ++f) dW_r[(long)e * F + f] = 0.0;
+            for (long t = 0; t < T; ++t) {
+                for (int f = 0; f < F; ++f) dW_r[(long)e * F + f] += dg[t * E + e] * u[t * F + f];
+                for (int j = 0; j < k; ++j) {
+                    if (idx[t * k + j] != e) continue;
+                    for (int srow = 0; srow < S; ++srow) {
+                        const double c = w[t * k + j] * dBC[t * S + srow];
+                        for (int f = 0; f < F; ++f) dW_e[((long)e * S + srow) * F + f] += c * u[t * F + f];
+                    }
+                }
+            }
+        }
+        if (dBC_out) memcpy(dBC_out, dBC, sizeof(double) * (size_t)(T * S));
+    }
+    free(idx); free(w); free(pi); free(BC); free(dBC); free(dg);
+    return rc;
+}
+
+/* ---------------------------------------------------------------------------
  * One autoregressive step: the layer above with one token per sequence and the
  * carried state updated in place (state[B,H,P,N]).
  * ------------------------------------------------------------------------- */

@@ -462,3 +462,89 @@ def test_block_forward_is_the_composition_of_its_steps_and_reduces_to_a_plain_bl
                               conv_state=r1["conv_state"], h0=r1["h_final"])
     np.testing.assert_allclose(np.concatenate([r1["out"], r2["out"]], 1), r["out"], rtol=1e-9, atol=1e-11)
     np.testing.assert_allclose(r2["h_final"], r["h_final"], rtol=1e-9, atol=1e-12)
+
+
+# ----------------------------------------------------------------- gradients of the trained weights
+def _loss(lay, dy, k, G, idx, W_r=None, W_e=None, h0=None):
+    """sum(dy * y) of the oracle's forward with the active sets held at idx and the weights taken
+    from the softmax of the (possibly perturbed) router matrix."""
+    W_r = lay["W_r"] if W_r is None else W_r
+    W_e = lay["W_e"] if W_e is None else W_e
+    T = idx.shape[0] * idx.shape[1]
+    pi = oracle.router(lay["u"].reshape(T, -1), W_r, k)["pi"]
+    fw = np.take_along_axis(pi, idx.reshape(T, k).astype(np.int64), -1)
+    out = oracle.swimba_forward(lay["u"], lay["x"], lay["dt"], W_r, W_e, lay["A"], lay["dt_bias"], lay["D"],
+                                k=k, G=G, h0=h0, forced_idx=idx, forced_w=fw)
+    return float(np.sum(dy * out["y"]))
+
+
+@pytest.mark.parametrize("G,k", [(1, 2), (2, 1), (1, 3)])
+def test_backward_matches_central_differences_of_the_forward(G, k):
+    lay = rand_layer(31 + k, B=2, L=7, F=5, H=4, P=3, N=4, G=G, E=3)
+    r = rng(77)
+    h0 = 0.3 * r.standard_normal((2, 4, 3, 4))
+    dy = r.standard_normal(lay["x"].shape)
+    fwd = oracle.swimba_forward(lay["u"], lay["x"], lay["dt"], lay["W_r"], lay["W_e"], lay["A"], lay["dt_bias"],
+                                lay["D"], k=k, G=G, h0=h0)
+    idx = fwd["idx"]
+    got = oracle.backward_weights(lay["u"], lay["x"], lay["dt"], lay["W_r"], lay["W_e"], lay["A"], lay["dt_bias"],
+                                  dy, k=k, G=G, h0=h0)
+    eps = 1e-6
+    for name, grad in (("W_e", got["dW_e"]), ("W_r", got["dW_r"])):
+        base = lay[name]
+        flat = r.choice(base.size, size=min(base.size, 24), replace=False)
+        for pos in flat:
+            where = np.unravel_index(pos, base.shape)
+            up, dn = base.copy(), base.copy()
+            up[where] += eps
+            dn[where] -= eps
+            fd = (_loss(lay, dy, k, G, idx, h0=h0, **{name: up}) - _loss(lay, dy, k, G, idx, h0=h0, **{name: dn})) / (2 * eps)
+            assert abs(fd - grad[where]) <= 1e-6 * max(1.0, abs(fd)), (name, where, fd, grad[where])
+
+
+def test_backward_single_token_closed_form():
+    # L = 1, zero initial state: y[h,p] = Delta_h x[h,p] (Ctilde . Btilde) + D_h x[h,p], so with
+    # c = sum_{h,p} dy Delta x:  dBtilde = c Ctilde, dCtilde = c Btilde, dW_e[e] = pi_e [dB; dC] u^T
+    lay = rand_layer(41, B=1, L=1, F=4, H=2, P=3, N=5, G=1, E=3)
+    k = 2
+    dy = rng(5).standard_normal(lay["x"].shape)
+    fwd = oracle.swimba_forward(lay["u"], lay["x"], lay["dt"], lay["W_r"], lay["W_e"], lay["A"], lay["dt_bias"],
+                                lay["D"], k=k)
+    got = oracle.backward_weights(lay["u"], lay["x"], lay["dt"], lay["W_r"], lay["W_e"], lay["A"], lay["dt_bias"],
+                                  dy, k=k)
+    delta = np_softplus(lay["dt"][0, 0] + lay["dt_bias"])
+    c = float(np.sum(dy[0, 0] * delta[:, None] * lay["x"][0, 0]))
+    Bt, Ct = fwd["BC"][0, 0, :5], fwd["BC"][0, 0, 5:]
+    dBC = np.concatenate([c * Ct, c * Bt])
+    np.testing.assert_allclose(got["dBC"][0, 0], dBC, rtol=1e-12, atol=1e-14)
+    want = np.zeros_like(lay["W_e"])
+    for j in range(k):
+        e = fwd["idx"][0, 0, j]
+        want[e] += fwd["w"][0, 0, j] * np.outer(dBC, lay["u"][0, 0])
+    np.testing.assert_allclose(got["dW_e"], want, rtol=1e-12, atol=1e-14)
+
+
+def test_backward_invariants():
+    lay = rand_layer(43, B=2, L=8, F=6, H=4, P=3, N=4, G=2, E=4)
+    r = rng(9)
+    dy1, dy2 = r.standard_normal(lay["x"].shape), r.standard_normal(lay["x"].shape)
+    args = (lay["u"], lay["x"], lay["dt"], lay["W_r"], lay["W_e"], lay["A"], lay["dt_bias"])
+    g1 = oracle.backward_weights(*args, dy1, k=2, G=2)
+    g2 = oracle.backward_weights(*args, dy2, k=2, G=2)
+    g12 = oracle.backward_weights(*args, 2.0 * dy1 - 3.0 * dy2, k=2, G=2)
+    # linear in dy
+    np.testing.assert_allclose(g12["dW_e"], 2.0 * g1["dW_e"] - 3.0 * g2["dW_e"], rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(g12["dW_r"], 2.0 * g1["dW_r"] - 3.0 * g2["dW_r"], rtol=1e-10, atol=1e-12)
+    # the softmax values sum to one: the logit gradients of a token sum to zero, hence the columns of dW_r
+    np.testing.assert_allclose(g1["dW_r"].sum(axis=0), 0.0, atol=1e-12 * np.abs(g1["dW_r"]).max())
+    # experts outside every active set receive no gradient; k == E (dense) reaches all of them
+    idx = oracle.swimba_forward(*args, lay["D"], k=2, G=2)["idx"]
+    unused = [e for e in range(4) if not np.any(idx == e)]
+    for e in unused:
+        assert not np.any(g1["dW_e"][e])
+    # one expert: the softmax is constant, the router receives nothing
+    one = rand_layer(44, E=1)
+    g = oracle.backward_weights(one["u"], one["x"], one["dt"], one["W_r"], one["W_e"], one["A"], one["dt_bias"],
+                                r.standard_normal(one["x"].shape), k=1)
+    assert not np.any(g["dW_r"])
+    assert np.any(g["dW_e"])
