@@ -525,6 +525,10 @@ def main():
     if single and not args.no_serving:
         shard = bench_shard(sb)
 
+    backward = None
+    if single and not args.no_serving:
+        backward = {name: bench_backward(sb, synth.CONFIGS[name]) for name in ("small_lm", "mid")}
+
     cpu = None
     if single and not args.no_cpu_baseline:
         cpu, _ = time_oracle_sample(cfg, cfg.B)
@@ -542,7 +546,7 @@ def main():
                        "how": "value is the median over rounds of exactly `steps` steps each"},
             "ssd_segments": nseg,
             "kernels": kernels, "comparators": comparators, "workloads": workloads,
-            "decode": decode, "serving": serving, "sequence_sharded": shard,
+            "decode": decode, "serving": serving, "sequence_sharded": shard, "backward_weights": backward,
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
@@ -607,6 +611,52 @@ def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
     }
     sb.swimba_destroy(h)
     return out
+
+
+def bench_backward(sb, cfg, steps: int = 5, warmup: int = 2):
+    """The gradients of the router and expert matrices (swimba_backward_weights) for one batch of the
+    workload: ms per call and per kernel.  These kernels run on the CUDA cores and are not tuned."""
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(21)
+    wts = {n: v.cuda() for n, v in synth.make_weights(cfg, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    dgen = torch.Generator(device="cuda")
+    dgen.manual_seed(22)
+    B, L = cfg.B, cfg.L
+    u = torch.randn(B, L, cfg.F, generator=dgen, device="cuda").bfloat16()
+    x = torch.randn(B, L, cfg.H, cfg.P, generator=dgen, device="cuda").bfloat16()
+    dy = torch.randn(B, L, cfg.H, cfg.P, generator=dgen, device="cuda").bfloat16()
+    dt = 0.5 * torch.randn(B, L, cfg.H, generator=dgen, device="cuda")
+    dWr = torch.empty(cfg.E, cfg.F, device="cuda")
+    dWe = torch.empty(cfg.E, cfg.S, cfg.F, device="cuda")
+    ws = torch.empty(sb.swimba_backward_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        sb.swimba_backward_weights(h, w, u, x, dt, None, dy, B, L, dWr, dWe, None, ws)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    sb.swimba_profile(h, True)
+    step()
+    torch.cuda.synchronize()
+    per = {}
+    for name, t in sb.swimba_profile_read(h):
+        per[name] = per.get(name, 0.0) + t
+    sb.swimba_profile(h, False)
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    return {"workload": config_dict(cfg)["workload"], "ms": ms, "tokens_per_s": cfg.tokens / (ms * 1e-3),
+            "kernel_ms": per}
 
 
 def bench_shard(sb, ranks: int = 8, steps: int = 10, warmup: int = 3):

@@ -192,6 +192,26 @@ int swimba_shard_finish(swimba_handle *h, const swimba_weights *w, const void *x
                         int32_t B, int32_t L, void *y, float *h_end, void *workspace, size_t workspace_bytes,
                         void *cuda_stream);
 
+/* Backward pass for the weights the paper trains (Section "Training": the router and the expert
+ * parameters; everything else in the layer is frozen): given dy [B,L,H,P] dtype, the gradient of a
+ * scalar loss with respect to y, writes
+ *   dW_router [E, F] fp32   and   dW_expert [E, 2*G*N, F] fp32
+ * (overwritten; dW_router may be NULL when E == 1).  The forward's routing and mixed streams are
+ * recomputed from u; the active sets K_t are constants of the differentiation and the kept weights
+ * are differentiated as softmax values over all E (router equation, no renormalisation).  The
+ * recurrence's adjoint (Theorem 1's state equation run backwards) gives dBtilde, dCtilde; the
+ * mix, the softmax and the logits follow.  The final state does not enter the loss.  topk_idx
+ * [B,L,k] (may be NULL) receives the active sets the gradients were taken with.  u, x, dt, h0 as
+ * in swimba_forward; device pointers, caller-owned, 16-byte aligned; workspace of
+ * swimba_backward_workspace_bytes(h, B, L) bytes.  Sums over tokens are accumulated with fp32
+ * atomics: results are reproducible to rounding, not bit for bit.  Errors as swimba_forward;
+ * SWIMBA_ERR_UNSUPPORTED_SHAPE when d_state * ceil(head_dim / 16) exceeds 1024 threads. */
+size_t swimba_backward_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L);
+int swimba_backward_weights(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                            const float *dt, const float *h0, const void *dy, int32_t B, int32_t L,
+                            float *dW_router, float *dW_expert, int32_t *topk_idx, void *workspace,
+                            size_t workspace_bytes, void *cuda_stream);
+
 /* The general form of the layer, with expert-specific SSM inputs (the state equation of Section
  * "MoE-parameterized SSM" as printed: h_t = A h_{t-1} + sum_{e in K_t} pi_{t,e} B_t^(e) X_t^(e)^T,
  * Y_t = (sum_{e in K_t} pi_{t,e} C_t^(e))^T h_t).  The caller's experts produce X^(e) themselves (in
@@ -303,9 +323,9 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..17 (1 router + grouping by
+ * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..22 (1 router + grouping by
  * expert (for fewer than about 28000 tokens the launch also computes the SSD step sizes), 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
- * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection, 15 convolution + SiLU, 16 gated norm, 17 step-size columns; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
+ * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection, 15 convolution + SiLU, 16 gated norm, 17 step-size columns, 18 adjoint recurrence pass, 19 router softmax over all experts, 20 weight / logit adjoints, 21 router-matrix gradient, 22 expert-matrix gradient; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);

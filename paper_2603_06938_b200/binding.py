@@ -32,6 +32,7 @@ EXPORTS = [
     "swimba_create", "swimba_workspace_bytes", "swimba_ssd_segments", "swimba_forward", "swimba_route_mix", "swimba_ssd",
     "swimba_packed_workspace_bytes", "swimba_packed_segments", "swimba_forward_packed",
     "swimba_shard_workspace_bytes", "swimba_shard_summary", "swimba_shard_finish",
+    "swimba_backward_workspace_bytes", "swimba_backward_weights",
     "swimba_route_project_slots", "swimba_ssd_slots_workspace_bytes", "swimba_ssd_slots",
     "swimba_block_workspace_bytes", "swimba_block_forward",
     "swimba_decode_workspace_bytes", "swimba_decode_step", "swimba_host_workspace_bytes",
@@ -94,6 +95,11 @@ def lib() -> ctypes.CDLL:
         L.swimba_forward_packed.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp,
                                             ctypes.POINTER(i32), i32, vp, vp, vp, vp, vp, sz, vp]
         L.swimba_forward_packed.restype = ctypes.c_int
+        L.swimba_backward_workspace_bytes.argtypes = [vp, i32, i32]
+        L.swimba_backward_workspace_bytes.restype = sz
+        L.swimba_backward_weights.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, vp, vp, i32, i32,
+                                              vp, vp, vp, vp, sz, vp]
+        L.swimba_backward_weights.restype = ctypes.c_int
         L.swimba_shard_workspace_bytes.argtypes = [vp, i32, i32]
         L.swimba_shard_workspace_bytes.restype = sz
         L.swimba_shard_summary.argtypes = [vp, ctypes.POINTER(swimba_weights), vp, vp, vp, i32, i32, vp, vp,
@@ -228,6 +234,21 @@ def swimba_forward(h: Handle, w: swimba_weights, u, x, dt, h0, B: int, L: int, y
     rc = lib().swimba_forward(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), B, L,
                               _ptr(y), _ptr(h_final), _ptr(topk_idx), _ptr(topk_w), wp, wb,
                               _stream(stream))
+    if check and rc != OK:
+        h._raise(rc)
+    return rc
+
+
+def swimba_backward_workspace_bytes(h: Handle, B: int, L: int) -> int:
+    return int(lib().swimba_backward_workspace_bytes(h.ptr, B, L))
+
+
+def swimba_backward_weights(h: Handle, w: swimba_weights, u, x, dt, h0, dy, B: int, L: int, dW_router,
+                            dW_expert, topk_idx, workspace, stream=None, check: bool = True) -> int:
+    wp, wb = _ws(workspace)
+    rc = lib().swimba_backward_weights(h.ptr, ctypes.byref(w), _ptr(u), _ptr(x), _ptr(dt), _ptr(h0), _ptr(dy),
+                                       B, L, _ptr(dW_router), _ptr(dW_expert), _ptr(topk_idx), wp, wb,
+                                       _stream(stream))
     if check and rc != OK:
         h._raise(rc)
     return rc
@@ -396,7 +417,8 @@ KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 5: "mix_slots", 6: "project_mix_simt", 7: "ssd_sequential", 8: "decode_update",
                 9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars", 12: "slot_streams",
                 13: "slot_sum", 14: "project_small", 15: "conv_silu", 16: "gated_rmsnorm",
-                17: "dt_columns"}
+                17: "dt_columns", 18: "ssd_adjoint", 19: "router_softmax", 20: "dpi_dg", 21: "dw_router",
+                22: "dw_expert"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

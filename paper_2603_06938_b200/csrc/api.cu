@@ -841,6 +841,108 @@ int swimba_shard_finish(swimba_handle *h, const swimba_weights *w, const void *x
     return rc;
 }
 
+namespace {
+// Workspace of the backward: the forward's token regions, then [ones | slot projections | dBC | pi | dg].
+struct BwdLayout {
+    FwdLayout f;
+    size_t ones, slots, dbc, pi, dg, total;
+};
+BwdLayout bwd_layout(const swimba_config &c, int B, int L, int sm_count)
+{
+    BwdLayout l;
+    l.f = fwd_layout(c, B, L, sm_count);
+    const size_t T = (size_t)B * L, S = 2u * c.n_groups * c.d_state;
+    size_t off = l.f.ssd;
+    l.ones = off;  off += align_up(T * c.top_k * sizeof(float));
+    l.slots = off; off += align_up(T * c.top_k * S * elt_size(c.dtype));
+    l.dbc = off;   off += align_up(T * S * sizeof(float));
+    l.pi = off;    off += align_up(T * c.n_experts * sizeof(float));
+    l.dg = off;    off += align_up(T * c.n_experts * sizeof(float));
+    l.total = off;
+    return l;
+}
+}  // namespace
+
+size_t swimba_backward_workspace_bytes(const swimba_handle *h, int32_t B, int32_t L)
+{
+    if (!h || B <= 0 || L <= 0) return 0;
+    return bwd_layout(h->cfg, B, L, h->sm_count).total;
+}
+
+int swimba_backward_weights(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
+                            const float *dt, const float *h0, const void *dy, int32_t B, int32_t L,
+                            float *dW_router, float *dW_expert, int32_t *topk_idx, void *workspace,
+                            size_t workspace_bytes, void *cuda_stream)
+{
+    if (!h) return SWIMBA_ERR_NULL_ARG;
+    h->err[0] = 0;
+    const swimba_config &c = h->cfg;
+    if (B < 0 || L < 0) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "negative B or L");
+    const int64_t T = (int64_t)B * L;
+    if (T * c.top_k >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (B * L * top_k must stay below 2^31)");
+    if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
+    if (!ssd_adjoint_supported(c.head_dim, c.d_state) || (int64_t)c.n_experts * ((T + 2047) / 2048) > 65535 ||
+        (int64_t)B * c.n_heads >= (int64_t)1 << 31)
+        return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "shape outside what the backward kernels take");
+    int rc = check_weights(h, w, true);
+    if (rc != SWIMBA_OK) return rc;
+    if (!dW_expert || (!dW_router && c.n_experts > 1))
+        return fail(h, SWIMBA_ERR_NULL_ARG, "a gradient output is NULL");
+    if (!aligned16(u) || !aligned16(x) || !aligned16(dy) || !aligned16(dt) || !aligned16(h0) || !aligned16(dW_router) ||
+        !aligned16(dW_expert) || !aligned16(topk_idx) || !aligned16(workspace))
+        return fail(h, SWIMBA_ERR_MISALIGNED, "tensors must be 16-byte aligned");
+    if ((rc = set_device(h)) != SWIMBA_OK) return rc;
+    LaunchCtx ctx{(cudaStream_t)cuda_stream, h->d_status, 0, &h->prof, (c.flags & SWIMBA_FLAG_CHECK_INDICES) != 0, &h->tmaps};
+    h->prof.n = 0;
+    const size_t S = 2u * c.n_groups * c.d_state;
+    // the gradients of an empty batch are zero
+    if (cudaMemsetAsync(dW_expert, 0, (size_t)c.n_experts * S * c.d_model * sizeof(float), ctx.stream) != cudaSuccess ||
+        (dW_router &&
+         cudaMemsetAsync(dW_router, 0, (size_t)c.n_experts * c.d_model * sizeof(float), ctx.stream) != cudaSuccess))
+        return fail(h, SWIMBA_ERR_CUDA, "clearing the gradients failed");
+    h->last_stream = ctx.stream;
+    if (T == 0) { h->last_launches = 0; return SWIMBA_OK; }
+    if (!u || !x || !dy || !workspace) return fail(h, SWIMBA_ERR_NULL_ARG, "u, x, dy or workspace is NULL");
+    const BwdLayout l = bwd_layout(c, B, L, h->sm_count);
+    if (workspace_bytes < l.total) return fail(h, SWIMBA_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    char *ws = (char *)workspace;
+    int32_t *idx = topk_idx ? topk_idx : (int32_t *)(ws + l.f.idx);
+    float *wt = (float *)(ws + l.f.w);
+    void *BC = ws + l.f.bc;
+    float *ones = (float *)(ws + l.ones);
+    void *slots = ws + l.slots;
+    float *dBC = (float *)(ws + l.dbc);
+    // forward quantities again: routing, mixed streams, and the unscaled projection of every kept slot
+    rc = run_route_mix(h, ctx, w, u, T, BC, false, idx, wt, ws + l.f.gemm);
+    if (rc == SWIMBA_OK) rc = launch_fill(ctx, ones, T * c.top_k, 1.f);
+    if (rc == SWIMBA_OK) {
+        if (use_tensor_k1(c))
+            rc = launch_expert_gemm(ctx, u, w->W_expert, ones, T, c.d_model, (int)S, c.n_experts, c.top_k, h->sm_count,
+                                    BC, ws + l.f.gemm, slots);
+        else
+            rc = launch_project_slots_simt(ctx, c.dtype, u, w->W_expert, idx, ones, T, c.d_model, (int)S, c.n_experts,
+                                           c.top_k, slots);
+        if (rc != SWIMBA_OK) rc = fail(h, rc, "slot projection launch failed");
+    }
+    if (rc == SWIMBA_OK && cudaMemsetAsync(dBC, 0, (size_t)T * S * sizeof(float), ctx.stream) != cudaSuccess)
+        rc = fail(h, SWIMBA_ERR_CUDA, "clearing dBC failed");
+    if (rc == SWIMBA_OK) {
+        rc = launch_ssd_adjoint(ctx, c.dtype, x, dy, BC, dt, w->A, w->dt_bias, h0, B, L, c.n_heads, c.head_dim,
+                                c.d_state, c.n_groups, dBC);
+        if (rc != SWIMBA_OK) rc = fail(h, rc, "adjoint recurrence launch failed");
+    }
+    if (rc == SWIMBA_OK) {
+        const void *Wr = w->W_router ? w->W_router : w->W_expert;
+        rc = launch_weight_grads(ctx, c.dtype, u, Wr, slots, idx, wt, dBC, T, c.d_model, (int)S, c.n_experts, c.top_k,
+                                 (float *)(ws + l.pi), (float *)(ws + l.dg),
+                                 dW_router, dW_expert);
+        if (rc != SWIMBA_OK) rc = fail(h, rc, "weight gradient launch failed");
+    }
+    h->last_launches = ctx.launches;
+    return rc;
+}
+
 int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u, const void *x,
                        const float *dt, float *state, int32_t B, void *y, int32_t *topk_idx,
                        float *topk_w, void *workspace, size_t workspace_bytes, void *cuda_stream)

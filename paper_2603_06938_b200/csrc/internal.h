@@ -96,6 +96,20 @@ int launch_ssd_shard_finish(LaunchCtx &ctx, const void *x, const void *BC, const
                             const float *all_state, const float *all_decay, int rank, int B, int L, int H, int G,
                             int chunk, int sm_count, void *y, float *h_end, void *workspace);
 
+// Backward for the trained weights (router and expert matrices), plain CUDA-core kernels.
+// adjoint: both passes of the recurrence's adjoint; dBC [T,S] fp32 (zeroed by the caller) receives
+// dBtilde | dCtilde.  weight_grads: softmax over all E (pi [T,E] scratch), dpi / dg (dg [T,E]
+// scratch) from the unscaled slot projections slots [T*k,S] (dtype), then dW_r [E,F] and dW_e
+// [E,S,F] (fp32, zeroed by the caller, accumulated with atomics).
+bool ssd_adjoint_supported(int P, int N);
+int launch_fill(LaunchCtx &ctx, float *p, int64_t n, float v);
+int launch_ssd_adjoint(LaunchCtx &ctx, int dtype, const void *x, const void *dy, const void *BC, const float *dt,
+                       const float *A, const float *dt_bias, const float *h0, int B, int L, int H, int P, int N,
+                       int G, float *dBC);
+int launch_weight_grads(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, const void *slots,
+                        const int32_t *idx, const float *w, const float *dBC, int64_t Tn, int F, int S, int E,
+                        int k, float *pi, float *dg, float *dW_r, float *dW_e);
+
 // One warp waiting on a barrier nobody signals, with the given limit (see swimba_selftest_wait).
 // out_dev: three 64-bit words on the device.
 int launch_wait_selftest(LaunchCtx &ctx, long long limit_cycles, long long *out_dev);
