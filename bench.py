@@ -47,14 +47,14 @@ TIMED_SECONDS = 1.5   # the K-step timed region is repeated until it has covered
 # writes can still sit in L2 when it ends.
 NCU_TRAFFIC_BYTES = {
     # profiles/forward_small_lm_kernels.md (the router launch includes the SSD step sizes)
-    "small_lm": {"router_topk": 26.790e6, "expert_gemm": 36.988e6, "ssd_tiles": 83.644e6},
+    "small_lm": {"router_topk": 26.790e6, "expert_gemm": 36.989e6, "ssd_tiles": 83.015e6},
     # profiles/forward_mid_kernels.md
-    "mid": {"ssd_scalars": 8.415e6, "router_topk": 147.477e6, "expert_gemm": 258.521e6, "ssd_tiles": 586.430e6},
+    "mid": {"ssd_scalars": 8.413e6, "router_topk": 147.366e6, "expert_gemm": 258.593e6, "ssd_tiles": 580.232e6},
     # profiles/ssd_segmented_long_seq.md; ssd_tiles is launched twice per step (state-only pass
-    # 347.9 MB + full pass 621.7 MB) and rated per step, so the figure is the sum of the two launches
-    "long_seq": {"ssd_tiles": 969.591e6, "segment_scan": 18.882e6},
+    # 348.0 MB + full pass 620.2 MB) and rated per step, so the figure is the sum of the two launches
+    "long_seq": {"ssd_tiles": 968.194e6, "segment_scan": 18.883e6},
     # profiles/decode_step_kernels.md
-    "decode": {"router_topk": 0.593e6, "project_small": 9.070e6, "decode_update": 479.797e6},
+    "decode": {"router_topk": 0.593e6, "project_small": 9.071e6, "decode_update": 479.881e6},
 }
 
 
