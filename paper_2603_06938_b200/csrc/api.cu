@@ -845,7 +845,7 @@ namespace {
 // Workspace of the backward: the forward's token regions, then [ones | slot projections | dBC | pi | dg].
 struct BwdLayout {
     FwdLayout f;
-    size_t ones, slots, dbc, pi, dg, total;
+    size_t ones, slots, dbc, pi, dg, adj, total;
 };
 BwdLayout bwd_layout(const swimba_config &c, int B, int L, int sm_count)
 {
@@ -858,6 +858,9 @@ BwdLayout bwd_layout(const swimba_config &c, int B, int L, int sm_count)
     l.dbc = off;   off += align_up(T * S * sizeof(float));
     l.pi = off;    off += align_up(T * c.n_experts * sizeof(float));
     l.dg = off;    off += align_up(T * c.n_experts * sizeof(float));
+    l.adj = off;
+    if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+        off += align_up(ssd_adjoint_tiles_workspace_bytes(B, L, c.n_heads, c.chunk, sm_count));
     l.total = off;
     return l;
 }
@@ -928,8 +931,14 @@ int swimba_backward_weights(swimba_handle *h, const swimba_weights *w, const voi
     if (rc == SWIMBA_OK && cudaMemsetAsync(dBC, 0, (size_t)T * S * sizeof(float), ctx.stream) != cudaSuccess)
         rc = fail(h, SWIMBA_ERR_CUDA, "clearing dBC failed");
     if (rc == SWIMBA_OK) {
-        rc = launch_ssd_adjoint(ctx, c.dtype, x, dy, BC, dt, w->A, w->dt_bias, h0, B, L, c.n_heads, c.head_dim,
-                                c.d_state, c.n_groups, dBC);
+        // shapes of the forward's tile kernel: the adjoint is two more evaluations of that kernel on
+        // re-arranged operands; everything else: per-timestep passes
+        if (ssd_tiles_supported(c.dtype, c.head_dim, c.d_state))
+            rc = launch_ssd_adjoint_tiles(ctx, x, dy, BC, dt, w->A, w->dt_bias, h0, B, L, c.n_heads, c.n_groups,
+                                          c.chunk, h->sm_count, dBC, ws + l.adj);
+        else
+            rc = launch_ssd_adjoint(ctx, c.dtype, x, dy, BC, dt, w->A, w->dt_bias, h0, B, L, c.n_heads, c.head_dim,
+                                    c.d_state, c.n_groups, dBC);
         if (rc != SWIMBA_OK) rc = fail(h, rc, "adjoint recurrence launch failed");
     }
     if (rc == SWIMBA_OK) {

@@ -106,6 +106,12 @@ int launch_fill(LaunchCtx &ctx, float *p, int64_t n, float v);
 int launch_ssd_adjoint(LaunchCtx &ctx, int dtype, const void *x, const void *dy, const void *BC, const float *dt,
                        const float *A, const float *dt_bias, const float *h0, int B, int L, int H, int P, int N,
                        int G, float *dBC);
+// The same adjoint through the forward's tile kernel (bf16, P = 64, N = 128): both passes are
+// evaluations of a virtual layer of 2H heads in H groups; dBC is overwritten, not accumulated.
+size_t ssd_adjoint_tiles_workspace_bytes(int B, int L, int H, int chunk, int sm_count);
+int launch_ssd_adjoint_tiles(LaunchCtx &ctx, const void *x, const void *dy, const void *BC, const float *dt,
+                             const float *A, const float *dt_bias, const float *h0, int B, int L, int H, int G,
+                             int chunk, int sm_count, float *dBC, void *workspace);
 int launch_weight_grads(LaunchCtx &ctx, int dtype, const void *u, const void *W_r, const void *slots,
                         const int32_t *idx, const float *w, const float *dBC, int64_t Tn, int F, int S, int E,
                         int k, float *pi, float *dg, float *dW_r, float *dW_e);

@@ -62,6 +62,9 @@ CASES = [
     cfg_of("bf16", L=33, B=3, P=32, N=64, H=3, F=40),
     cfg_of("bf16", L=2100, B=1, H=2, F=256, E=16, k=2),        # several token runs per expert
     cfg_of("bf16", L=260, k=1, E=1),                           # one expert: nothing reaches the router
+    cfg_of("bf16", L=2100, B=1, H=2),                          # the tile-kernel adjoint cut into segments
+    cfg_of("bf16", L=390, B=2, H=3),                           # odd head count
+    cfg_of("bf16", L=1, B=3),                                  # single token
 ]
 
 
