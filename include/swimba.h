@@ -285,9 +285,11 @@ int swimba_decode_step(swimba_handle *h, const swimba_weights *w, const void *u,
 /* End-to-end variant of swimba_forward for callers whose activations live in HOST memory
  * (pinned memory makes the copies asynchronous): copies u_host, x_host, dt_host (may be NULL)
  * to device staging, runs the forward of Theorem 1, copies y (and h_final / topk outputs when
- * given) back; the batch goes through in up to eight slices of whole sequences so that the copies
- * in, the kernels and the copies out of successive slices overlap (two copy streams owned by the
- * handle, the kernels on the given stream).  The given stream ends after the last copy out: the
+ * given) back; the batch goes through in slices so that the copies in, the kernels and the copies
+ * out of successive slices overlap (two copy streams owned by the handle, the kernels on the given
+ * stream): up to eight slices of whole sequences, or, with fewer than eight sequences, runs of
+ * consecutive tokens (multiples of 256) of one sequence at a time, the state carried from run to
+ * run (Theorem 1: the recurrence needs nothing else from the past), about sixteen slices in all.  The given stream ends after the last copy out: the
  * caller synchronises it before reading.
  * Weights stay device pointers.  The workspace holds the staging buffers as well and is sized
  * by swimba_host_workspace_bytes. */

@@ -19,7 +19,7 @@ struct swimba_handle {
     TmapCache tmaps;        // tensor maps encoded so far (same buffers call after call: encoded once)
     // host-buffer entry point: copy streams and events of its batch-slice pipeline
     cudaStream_t s_in, s_out;
-    cudaEvent_t ev_start, ev_out, ev_in[8], ev_done[8];
+    cudaEvent_t ev_start, ev_out, ev_in[32], ev_done[32];
     char err[256];
 };
 
@@ -82,12 +82,17 @@ DecLayout dec_layout(const swimba_config &c, int B)
 
 // Host-variant staging: [u | x | dt | y | h_final | idx | w] in front of the forward workspace.
 struct HostLayout {
-    size_t u, x, dt, y, hf, idx, w, fwd, total;
+    size_t u, x, dt, y, hf, hf2, idx, w, fwd, total;
 };
-constexpr int kHostSlices = 8;     // batch slices of the host-buffer pipeline (at most)
-// Sequences per slice.  Slices start at whole sequences inside the staged tensors, so every
-// per-sequence size has to keep the 16-byte alignment; otherwise the batch goes as one slice.
-inline int host_slice_seqs(const swimba_config &c, int B, int L)
+constexpr int kHostSlices = 8;     // batch slices of the host-buffer pipeline when there are that many sequences
+constexpr int kHostPieces = 16;    // slices aimed at when sequences have to be cut along time instead
+// A slice is `seqs` whole sequences, or (seqs == 1) a run of `piece` tokens of one sequence (a
+// multiple of 256 tokens; the state is carried from run to run).  Slices start at byte offsets
+// that keep the 16-byte alignment; where a per-sequence size does not, the batch goes as one slice.
+struct HostPlan {
+    int seqs, piece, pieces;      // sequences per slice, tokens per piece, pieces per sequence
+};
+inline HostPlan host_plan(const swimba_config &c, int B, int L)
 {
     const size_t es = elt_size(c.dtype);
     const size_t per_seq[5] = {(size_t)L * c.d_model * es, (size_t)L * c.n_heads * c.head_dim * es,
@@ -95,8 +100,12 @@ inline int host_slice_seqs(const swimba_config &c, int B, int L)
                                (size_t)L * c.top_k * sizeof(int32_t),
                                (size_t)c.n_heads * c.head_dim * c.d_state * sizeof(float)};
     for (size_t v : per_seq)
-        if (v % 16 != 0) return B;
-    return (B + kHostSlices - 1) / kHostSlices;
+        if (v % 16 != 0) return HostPlan{B, L, 1};
+    if (B >= kHostSlices) return HostPlan{(B + kHostSlices - 1) / kHostSlices, L, 1};
+    int want = (kHostPieces + B - 1) / B;
+    int piece = ((L + want - 1) / want + 255) / 256 * 256;
+    if (piece >= L) return HostPlan{1, L, 1};
+    return HostPlan{1, piece, (L + piece - 1) / piece};
 }
 
 HostLayout host_layout(const swimba_config &c, int B, int L, int sm_count)
@@ -110,10 +119,12 @@ HostLayout host_layout(const swimba_config &c, int B, int L, int sm_count)
     l.dt = off;  off += align_up(T * c.n_heads * sizeof(float));
     l.y = off;   off += align_up(T * HP * es);
     l.hf = off;  off += align_up((size_t)B * HP * c.d_state * sizeof(float));
+    l.hf2 = off; off += align_up((size_t)B * HP * c.d_state * sizeof(float));   // (carried states alternate)
     l.idx = off; off += align_up(T * c.top_k * sizeof(int32_t));
     l.w = off;   off += align_up(T * c.top_k * sizeof(float));
     // the forward runs slice by slice on the same scratch
-    l.fwd = off; off += fwd_layout(c, host_slice_seqs(c, B, L), L, sm_count).total;
+    const HostPlan hp = host_plan(c, B, L);
+    l.fwd = off; off += fwd_layout(c, hp.seqs, hp.piece, sm_count).total;
     l.total = off;
     return l;
 }
@@ -140,7 +151,7 @@ bool create_host_pipeline(swimba_handle *h)
               cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) == cudaSuccess &&
               cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
               cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; ok && i < 8; ++i)
+    for (int i = 0; ok && i < 32; ++i)
         ok = cudaEventCreateWithFlags(&h->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&h->ev_done[i], cudaEventDisableTiming) == cudaSuccess;
     return ok;
@@ -152,7 +163,7 @@ void destroy_host_pipeline(swimba_handle *h)
     if (h->s_out) cudaStreamDestroy(h->s_out);
     if (h->ev_start) cudaEventDestroy(h->ev_start);
     if (h->ev_out) cudaEventDestroy(h->ev_out);
-    for (int i = 0; i < 8; ++i) {
+    for (int i = 0; i < 32; ++i) {
         if (h->ev_in[i]) cudaEventDestroy(h->ev_in[i]);
         if (h->ev_done[i]) cudaEventDestroy(h->ev_done[i]);
     }
@@ -1029,45 +1040,55 @@ int swimba_forward_host(swimba_handle *h, const swimba_weights *w, const void *u
     const size_t tok_u = (size_t)c.d_model * es, tok_x = HP * es, tok_dt = c.n_heads * sizeof(float);
     const size_t seq_hf = HP * c.d_state * sizeof(float);
     const size_t tok_k = (size_t)c.top_k * sizeof(int32_t);
-    const int bs = host_slice_seqs(c, B, L);
+    const HostPlan plan = host_plan(c, B, L);
     bool ok = cudaEventRecord(h->ev_start, st) == cudaSuccess &&
               cudaStreamWaitEvent(h->s_in, h->ev_start, 0) == cudaSuccess &&
               cudaStreamWaitEvent(h->s_out, h->ev_start, 0) == cudaSuccess;
     int launches = 0, slice = 0;
-    for (int b0 = 0; ok && b0 < B; b0 += bs, ++slice) {
-        const int nb = (B - b0 < bs) ? B - b0 : bs;
-        const size_t t0 = (size_t)b0 * L, nt = (size_t)nb * L;
-        ok = cudaMemcpyAsync(ws + l.u + t0 * tok_u, (const char *)u_host + t0 * tok_u, nt * tok_u,
-                             cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
-             cudaMemcpyAsync(ws + l.x + t0 * tok_x, (const char *)x_host + t0 * tok_x, nt * tok_x,
-                             cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
-        if (ok && dt_host)
-            ok = cudaMemcpyAsync(ws + l.dt + t0 * tok_dt, (const char *)dt_host + t0 * tok_dt, nt * tok_dt,
+    for (int b0 = 0; ok && rc == SWIMBA_OK && b0 < B; b0 += plan.seqs) {
+        const int nb = (B - b0 < plan.seqs) ? B - b0 : plan.seqs;
+        for (int pc = 0; ok && pc < plan.pieces; ++pc, ++slice) {
+            const int l0 = pc * plan.piece;
+            const int len = plan.pieces == 1 ? L : (L - l0 < plan.piece ? L - l0 : plan.piece);
+            const size_t t0 = (size_t)b0 * L + l0, nt = (size_t)nb * len;
+            ok = cudaMemcpyAsync(ws + l.u + t0 * tok_u, (const char *)u_host + t0 * tok_u, nt * tok_u,
+                                 cudaMemcpyHostToDevice, h->s_in) == cudaSuccess &&
+                 cudaMemcpyAsync(ws + l.x + t0 * tok_x, (const char *)x_host + t0 * tok_x, nt * tok_x,
                                  cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
-        ok = ok && cudaEventRecord(h->ev_in[slice], h->s_in) == cudaSuccess &&
-             cudaStreamWaitEvent(st, h->ev_in[slice], 0) == cudaSuccess;
-        if (!ok) break;
-        rc = swimba_forward(h, w, ws + l.u + t0 * tok_u, ws + l.x + t0 * tok_x,
-                            dt_host ? (const float *)(ws + l.dt + t0 * tok_dt) : nullptr, nullptr, nb, L,
-                            ws + l.y + t0 * tok_x,
-                            h_final_host ? (float *)(ws + l.hf + (size_t)b0 * seq_hf) : nullptr,
-                            (int32_t *)(ws + l.idx + t0 * tok_k), (float *)(ws + l.w + t0 * tok_k),
-                            ws + l.fwd, workspace_bytes - l.fwd, cuda_stream);
-        if (rc != SWIMBA_OK) break;
-        launches += h->last_launches;
-        ok = cudaEventRecord(h->ev_done[slice], st) == cudaSuccess &&
-             cudaStreamWaitEvent(h->s_out, h->ev_done[slice], 0) == cudaSuccess &&
-             cudaMemcpyAsync((char *)y_host + t0 * tok_x, ws + l.y + t0 * tok_x, nt * tok_x,
-                             cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
-        if (ok && h_final_host)
-            ok = cudaMemcpyAsync((char *)h_final_host + (size_t)b0 * seq_hf, ws + l.hf + (size_t)b0 * seq_hf,
-                                 (size_t)nb * seq_hf, cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
-        if (ok && topk_idx_host)
-            ok = cudaMemcpyAsync((char *)topk_idx_host + t0 * tok_k, ws + l.idx + t0 * tok_k, nt * tok_k,
+            if (ok && dt_host)
+                ok = cudaMemcpyAsync(ws + l.dt + t0 * tok_dt, (const char *)dt_host + t0 * tok_dt, nt * tok_dt,
+                                     cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+            ok = ok && cudaEventRecord(h->ev_in[slice], h->s_in) == cudaSuccess &&
+                 cudaStreamWaitEvent(st, h->ev_in[slice], 0) == cudaSuccess;
+            if (!ok) break;
+            // the state after a piece enters the next piece of the same sequence; the two buffers
+            // alternate, since a call may still read its initial state while it writes its final one
+            const size_t hf_cur = (pc & 1) ? l.hf2 : l.hf, hf_prev = (pc & 1) ? l.hf : l.hf2;
+            const bool last_piece = pc == plan.pieces - 1;
+            const bool want_state = !last_piece || h_final_host != nullptr;
+            rc = swimba_forward(h, w, ws + l.u + t0 * tok_u, ws + l.x + t0 * tok_x,
+                                dt_host ? (const float *)(ws + l.dt + t0 * tok_dt) : nullptr,
+                                pc > 0 ? (const float *)(ws + hf_prev + (size_t)b0 * seq_hf) : nullptr, nb, len,
+                                ws + l.y + t0 * tok_x,
+                                want_state ? (float *)(ws + hf_cur + (size_t)b0 * seq_hf) : nullptr,
+                                (int32_t *)(ws + l.idx + t0 * tok_k), (float *)(ws + l.w + t0 * tok_k),
+                                ws + l.fwd, workspace_bytes - l.fwd, cuda_stream);
+            if (rc != SWIMBA_OK) break;
+            launches += h->last_launches;
+            ok = cudaEventRecord(h->ev_done[slice], st) == cudaSuccess &&
+                 cudaStreamWaitEvent(h->s_out, h->ev_done[slice], 0) == cudaSuccess &&
+                 cudaMemcpyAsync((char *)y_host + t0 * tok_x, ws + l.y + t0 * tok_x, nt * tok_x,
                                  cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
-        if (ok && topk_w_host)
-            ok = cudaMemcpyAsync((char *)topk_w_host + t0 * tok_k, ws + l.w + t0 * tok_k, nt * tok_k,
-                                 cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+            if (ok && h_final_host && last_piece)
+                ok = cudaMemcpyAsync((char *)h_final_host + (size_t)b0 * seq_hf, ws + hf_cur + (size_t)b0 * seq_hf,
+                                     (size_t)nb * seq_hf, cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+            if (ok && topk_idx_host)
+                ok = cudaMemcpyAsync((char *)topk_idx_host + t0 * tok_k, ws + l.idx + t0 * tok_k, nt * tok_k,
+                                     cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+            if (ok && topk_w_host)
+                ok = cudaMemcpyAsync((char *)topk_w_host + t0 * tok_k, ws + l.w + t0 * tok_k, nt * tok_k,
+                                     cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+        }
     }
     // The caller's stream ends after the last copy in and the last copy out, on the error paths
     // too (copies of earlier slices may still be in flight): synchronising it is enough before the
