@@ -325,9 +325,9 @@ int swimba_route_mix_static(swimba_handle *h, const swimba_weights *w, const voi
 /* Optional per-kernel timing (no counterpart in the paper; measurement aid).  While enabled,
  * every kernel a call enqueues is bracketed by CUDA events on the call's stream.
  * swimba_profile_read synchronises that stream and returns how many kernels the most recent call
- * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..23 (1 router + grouping by
+ * (for swimba_forward_host: its last batch slice) launched (at most max_entries), with kernel_ids[i] in 1..24 (1 router + grouping by
  * expert (for fewer than about 28000 tokens the launch also computes the SSD step sizes), 4 expert GEMM, 5 slot mix, 6 SIMT projection, 7 per-timestep SSM, 8 decode update, 9 SSD
- * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection, 15 convolution + SiLU, 16 gated norm, 17 step-size columns, 18 adjoint recurrence pass, 19 router softmax over all experts, 20 weight / logit adjoints, 21 router-matrix gradient, 22 expert-matrix gradient, 23 operand re-arrangement / head sum of the tile-kernel adjoint; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
+ * tile kernel, 10 segment scan, 11 SSD step sizes and decays, 12 slot stream assembly, 13 slot sum, 14 small-batch projection, 15 convolution + SiLU, 16 gated norm, 17 step-size columns, 18 adjoint recurrence pass, 19 router softmax over all experts, 20 weight / logit adjoints, 21 router-matrix gradient, 22 expert-matrix gradient, 23 operand re-arrangement / head sum of the tile-kernel adjoint, 24 state-only SSD pass; 2 and 3 are not in use) and ms[i] its duration in milliseconds.
  * Both arrays are HOST arrays. */
 int swimba_profile(swimba_handle *h, int enable);
 int swimba_profile_read(swimba_handle *h, int32_t *kernel_ids, float *ms, int32_t max_entries);

@@ -418,7 +418,7 @@ KERNEL_NAMES = {1: "router_topk", 4: "expert_gemm",
                 9: "ssd_tiles", 10: "segment_scan", 11: "ssd_scalars", 12: "slot_streams",
                 13: "slot_sum", 14: "project_small", 15: "conv_silu", 16: "gated_rmsnorm",
                 17: "dt_columns", 18: "ssd_adjoint", 19: "router_softmax", 20: "dpi_dg", 21: "dw_router",
-                22: "dw_expert", 23: "adjoint_pack"}
+                22: "dw_expert", 23: "adjoint_pack", 24: "ssd_state"}
 
 
 def swimba_profile(h: Handle, enable: bool) -> None:

@@ -18,7 +18,7 @@ enum Stage {
     STAGE_SSD_TILES = 9, STAGE_SEGMENT_SCAN = 10, STAGE_SSD_SCALARS = 11, STAGE_SLOT_STREAMS = 12,
     STAGE_SLOT_SUM = 13, STAGE_PROJECT_SMALL = 14, STAGE_CONV = 15, STAGE_GATED_NORM = 16,
     STAGE_DT_COLUMNS = 17, STAGE_SSD_ADJOINT = 18, STAGE_ROUTER_SOFTMAX = 19, STAGE_DPI_DG = 20,
-    STAGE_DW_ROUTER = 21, STAGE_DW_EXPERT = 22, STAGE_ADJOINT_PACK = 23,
+    STAGE_DW_ROUTER = 21, STAGE_DW_EXPERT = 22, STAGE_ADJOINT_PACK = 23, STAGE_SSD_STATE = 24,
 };
 
 constexpr int PROF_MAX = 64;

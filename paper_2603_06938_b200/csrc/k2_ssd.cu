@@ -854,6 +854,219 @@ shard_entry_kernel(float *__restrict__ states, const float *__restrict__ seg_dec
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// State-only pass on its own: the local end state of a segment from a zero entry state,
+//   H_end^T[n,p] = sum_s Btilde_s[n] (w'_s x_s[p]),   w'_s = Delta_s 2^(l(end of segment) - l(s)),
+// one long contraction over the segment's tokens accumulated in tensor memory (see the run
+// accumulation in ssd_tiles_kernel).  Nothing but Btilde, x and the tile records is read, so one
+// CTA takes FOUR heads of a group (the Btilde tile is fetched once for all of them: half the
+// shared-operand traffic of a head pair) and the tiles flow through a two-stage ring in which the
+// x slabs are scaled IN PLACE: TMA fills a stage, 16 warps (one token row of one head per thread)
+// scale, one thread issues a single 128 x 256 x 128 product per tile, its completion frees the
+// stage.  The state is read from tensor memory once, at the end.
+namespace {
+constexpr int NQ = 4;                                   // heads per CTA
+constexpr int ST_STAGES = 2;
+constexpr uint32_t ST_STAGE_BYTES = (2 + NQ) * SLAB;    // B0 B1 X0 X1 X2 X3
+constexpr uint32_t ST_SMALL = ST_STAGES * ST_STAGE_BYTES;
+constexpr int ST_THREADS = 32 * (4 * NQ + 2);
+constexpr uint32_t ST_TM_COLS = 256;
+
+struct __align__(16) StateSmall {
+    TileScalars sc[ST_STAGES][NQ];
+    uint64_t full[ST_STAGES], scaled[ST_STAGES], empty[ST_STAGES], done;
+    uint32_t tmem_slot;
+    int abort_flag;
+};
+
+__host__ __device__ inline int quads_per_group(int H, int G) { return (H / G + NQ - 1) / NQ; }
+}  // namespace
+
+__global__ void __launch_bounds__(ST_THREADS, 1)
+ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_constant__ CUtensorMap tmap_x,
+                 const SsdParams prm)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    StateSmall *sm = (StateSmall *)(smem + ST_SMALL);
+    int *abort_flag = &sm->abort_flag;
+    int *d_status = prm.d_status;
+    if ((tc::smem_u32(smem) & 1023u) != 0) {
+        if (threadIdx.x == 0) atomicCAS(d_status, 0, SWIMBA_ERR_DEVICE_BOUNDS);
+        return;
+    }
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const bool packed = prm.seqs != nullptr;
+    int seg = blockIdx.x, b = blockIdx.z;
+    int L = prm.L, tok0 = 0, bco = b;
+    const int H = prm.H;
+    int seg_base = b * prm.nseg;
+    int64_t rec_base = (int64_t)b * H * (prm.Lpad / ST);
+    int rec_hstride = prm.Lpad / ST;
+    if (packed) {
+        const int2 it = prm.items[blockIdx.x];
+        b = it.x; seg = it.y;
+        const SeqDesc sd = prm.seqs[b];
+        L = sd.len; tok0 = sd.tok0; bco = 0;
+        seg_base = sd.seg0;
+        rec_base = sd.tile0;
+        rec_hstride = prm.ntile_total;
+    }
+    const int HG = H / prm.G, qpg = quads_per_group(H, prm.G);
+    const int g = blockIdx.y / qpg, qd = blockIdx.y % qpg;
+    const int head0 = g * HG + qd * NQ;
+    const int nh = min(NQ, HG - qd * NQ);
+    const int t_begin = seg * prm.seg_len;
+    const int t_end = min(L, t_begin + prm.seg_len);
+    const int ntiles = (t_end - t_begin + ST - 1) / ST;
+
+    if (tid == 0) {
+        for (int s = 0; s < ST_STAGES; ++s) {
+            tc::mbar_init(&sm->full[s], 1);
+            tc::mbar_init(&sm->scaled[s], 128 * nh);
+            tc::mbar_init(&sm->empty[s], 1);
+        }
+        tc::mbar_init(&sm->done, 1);
+        *abort_flag = 0;
+        tc::fence_mbar_init();
+    }
+    if (warp == 4 * NQ + 1) {
+        tc::tmem_alloc(&sm->tmem_slot, ST_TM_COLS);
+        tc::tmem_relinquish();
+    }
+    if (warp == 4 * NQ && lane == 0) {
+        tc::prefetch_tmap(&tmap_bc);
+        tc::prefetch_tmap(&tmap_x);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem = sm->tmem_slot;
+    grid_dep_launch();
+    grid_dep_wait();
+
+    const int uwarp = __shfl_sync(0xffffffffu, warp, 0);
+    if (uwarp == 4 * NQ) {
+        // ------------------------------------------------------------------ TMA producer
+        const bool leader = tc::elect_one();
+        for (int j = 0; j < ntiles; ++j) {
+            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+            tc::mbar_wait(&sm->empty[s], ph ^ 1, abort_flag, d_status);
+            if (leader) {
+                uint8_t *stg = smem + s * ST_STAGE_BYTES;
+                const int t0 = tok0 + t_begin + j * ST;
+                tc::mbar_arrive_expect_tx(&sm->full[s], (2 + nh) * SLAB + nh * (uint32_t)sizeof(TileScalars));
+                tc::tma_load_3d(stg, &tmap_bc, &sm->full[s], g * SN, t0, bco);
+                tc::tma_load_3d(stg + SLAB, &tmap_bc, &sm->full[s], g * SN + 64, t0, bco);
+                for (int hd = 0; hd < nh; ++hd) {
+                    tc::tma_load_4d(stg + (2 + hd) * SLAB, &tmap_x, &sm->full[s], 0, head0 + hd, t0, bco);
+                    tc::bulk_load(&sm->sc[s][hd],
+                                  prm.rec + rec_base + (int64_t)(head0 + hd) * rec_hstride + t_begin / ST + j,
+                                  (uint32_t)sizeof(TileScalars), &sm->full[s]);
+                }
+            }
+            __syncwarp();
+        }
+    } else if (uwarp == 4 * NQ + 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        const bool leader = tc::elect_one();
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+        const uint32_t id_h = tc::idesc_bf16(128, 64 * nh, 1, 1);        // both operands MN-major
+        for (int j = 0; j < ntiles; ++j) {
+            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+            tc::mbar_wait(&sm->scaled[s], ph, abort_flag, d_status);
+            tc::tc_fence_after();
+            if (leader) {
+                const uint32_t base = tc::smem_u32(smem + s * ST_STAGE_BYTES);
+                const uint64_t dBt = tc::smem_desc_sw128(base, SLAB, 1024);
+                const uint64_t dXp = tc::smem_desc_sw128(base + 2 * SLAB, SLAB, 1024);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    tc::mma_ss(tmem_u, tc::smem_desc_advance(dBt, kk * 2048), tc::smem_desc_advance(dXp, kk * 2048),
+                               id_h, (j > 0) || (kk > 0));
+                tc::mma_commit(&sm->empty[s]);
+                if (j == ntiles - 1) tc::mma_commit(&sm->done);
+            }
+            __syncwarp();
+        }
+    } else if ((uwarp >> 2) < nh) {
+        // ------------------------------------------------------------------ compute warps
+        const int hd = warp >> 2, wq = warp & 3;
+        const int h = head0 + hd;
+        const int i = wq * 32 + lane;                    // token row in the tile == state index n
+        const int64_t rec_row = rec_base + (int64_t)h * rec_hstride + t_begin / ST;
+        float run_total = 0.f;                            // log2 decay over the whole segment
+        for (int jr = 0; jr < ntiles; ++jr) run_total += prm.rec[rec_row + jr].ends[3];
+        float run_done = 0.f;
+        for (int j = 0; j < ntiles; ++j) {
+            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+            tc::mbar_wait(&sm->full[s], ph, abort_flag, d_status);
+            const TileScalars *sc = &sm->sc[s][hd];
+            run_done += sc->ends[3];
+            const uint32_t wp = sc->wp[i];
+            const float w = (__uint_as_float(wp << 16) + __uint_as_float(wp & 0xffff0000u)) *
+                            tc::ex2_approx(run_total - run_done);
+            const __nv_bfloat16 w_hi = __float2bfloat16_rn(w);
+            const __nv_bfloat16 w_lo = __float2bfloat16_rn(w - __bfloat162float(w_hi));
+            const __nv_bfloat162 w_hi2 = __halves2bfloat162(w_hi, w_hi), w_lo2 = __halves2bfloat162(w_lo, w_lo);
+            uint8_t *s_x = smem + s * ST_STAGE_BYTES + (2 + hd) * SLAB;
+            uint4 xr[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) xr[c] = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(i, c));
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint32_t wv[4] = {xr[c].x, xr[c].y, xr[c].z, xr[c].w};
+                uint32_t o[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
+                    const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
+                    o[q] = *reinterpret_cast<const uint32_t *>(&pr);
+                }
+                *reinterpret_cast<uint4 *>(s_x + tc::sw128_offset(i, c)) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            tc::fence_proxy_async_smem();
+            tc::mbar_arrive(&sm->scaled[s]);
+        }
+        // ---- the segment's end state (entry state zero) and its total decay
+        float *dst = prm.h_out + ((((int64_t)seg_base + seg) * H + h) * SP) * SN;
+        if (ntiles > 0) {
+            tc::mbar_wait(&sm->done, 0, abort_flag, d_status);
+            tc::tc_fence_after();
+            const uint32_t tm = tmem + ((uint32_t)(wq * 32) << 16) + 64 * hd;
+#pragma unroll
+            for (int hh = 0; hh < 4; ++hh) {
+                uint32_t dh[16];
+                tc::tmem_ld16(tm + 16 * hh, dh);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int q = 0; q < 16; ++q) dst[(int64_t)(16 * hh + q) * SN + i] = __uint_as_float(dh[q]);
+            }
+        } else {
+#pragma unroll 8
+            for (int q = 0; q < SP; ++q) dst[(int64_t)q * SN + i] = 0.f;
+        }
+        if (i == 0) prm.seg_decay[((int64_t)seg_base + seg) * H + h] = tc::ex2_approx(run_total);
+    }
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 4 * NQ + 1) tc::tmem_dealloc(tmem, ST_TM_COLS);
+}
+
+static size_t ssd_state_smem_bytes() { return ST_SMALL + sizeof(StateSmall); }
+
+// The state-only launch behind both the dense and the packed segment passes.
+static int launch_state_pass(LaunchCtx &ctx, const CUtensorMap &tm_bc, const CUtensorMap &tm_x, const SsdParams &p,
+                             unsigned grid_x, int H, int G, unsigned grid_z)
+{
+    const size_t smem = ssd_state_smem_bytes();
+    if (!ensure_dynamic_smem((const void *)ssd_state_kernel, smem)) return SWIMBA_ERR_CUDA;
+    ctx.begin(STAGE_SSD_STATE);
+    launch_kernel(ssd_state_kernel, dim3(grid_x, (unsigned)(G * quads_per_group(H, G)), grid_z), dim3(ST_THREADS), smem,
+                  ctx.stream, true, tm_bc, tm_x, p);
+    ctx.end();
+    return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
+}
+
 bool ssd_tiles_supported(int dtype, int P, int N)
 {
     return dtype == SWIMBA_DTYPE_BF16 && P == SP && N == SN;
@@ -1001,9 +1214,10 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         float *states = (float *)seg_ws;
         float *decay = states + (size_t)B * nseg * H * SP * SN;
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
-        ctx.begin(STAGE_SSD_TILES);
-        launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), smem, ctx.stream, true, tm_bc, tm_x, tm_y, p);
-        ctx.end();
+        {
+            const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)nseg, H, G, (unsigned)B);
+            if (rc != SWIMBA_OK) return rc;
+        }
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
         segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
@@ -1166,10 +1380,8 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
         float *decay = (float *)(ws + lay.decay);
         p.items = (const int2 *)(ws + lay.pre);
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY; p.seg_states = 1;
-        ctx.begin(STAGE_SSD_TILES);
-        launch_kernel(ssd_tiles_kernel<false>, dim3((unsigned)pl.pre.size(), pairs, 1), dim3(SSD_THREADS), smem,
-                      ctx.stream, true, tm_bc, tm_x, tm_y, p);
-        ctx.end();
+        rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)pl.pre.size(), H, G, 1u);
+        if (rc != SWIMBA_OK) return rc;
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
         segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)nseq), 256, 0, ctx.stream>>>(
@@ -1268,11 +1480,10 @@ int launch_ssd_shard_summary(LaunchCtx &ctx, const void *x, const void *BC, cons
     float *states = (float *)((char *)workspace + lay.states);
     float *decay = (float *)((char *)workspace + lay.decay);
     p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
-    const dim3 grid((unsigned)lay.nseg, (unsigned)(G * pairs_per_group(H, G)), (unsigned)B);
-    ctx.begin(STAGE_SSD_TILES);
-    launch_kernel(ssd_tiles_kernel<false>, grid, dim3(SSD_THREADS), ssd_smem_bytes(), ctx.stream, true, tm_bc, tm_x,
-                  tm_y, p);
-    ctx.end();
+    {
+        const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)lay.nseg, H, G, (unsigned)B);
+        if (rc != SWIMBA_OK) return rc;
+    }
     const int PN4 = SP * SN / 4;
     ctx.begin(STAGE_SEGMENT_SCAN);
     segment_scan_kernel<<<dim3((unsigned)ceil_div(PN4, 256), (unsigned)H, (unsigned)B), 256, 0, ctx.stream>>>(
