@@ -870,7 +870,7 @@ constexpr int ST_STAGES = 2;
 constexpr uint32_t ST_STAGE_BYTES = (2 + NQ) * SLAB;    // B0 B1 X0 X1 X2 X3
 constexpr uint32_t ST_SMALL = ST_STAGES * ST_STAGE_BYTES;
 constexpr int ST_THREADS = 32 * (4 * NQ + 2);
-constexpr uint32_t ST_TM_COLS = 256;
+constexpr uint32_t ST_TM_COLS = NQ * 64 < 32 ? 32 : NQ * 64;
 
 struct __align__(16) StateSmall {
     TileScalars sc[ST_STAGES][NQ];
