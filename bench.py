@@ -150,10 +150,13 @@ def algorithmic_work(cfg: synth.LayerConfig, nseg: int = 1, sm_count: int = 148)
     ssd_bytes = T * (2 * H * P * es + S * es + H * 4) + cfg.B * H * P * N * 4
     w["ssd_tiles"] = dict(bound="tensor", work=ssd_flops, bytes=ssd_bytes)
     # the state-only pass of segmented sequences: x, Btilde and the step sizes in, segment states out
-    w["ssd_state"] = dict(bound="hbm", work=T * (H * P * es + G * N * es + H * 4) + nseg * cfg.B * H * P * N * 4)
+    # (every segment but a sequence's last one)
+    part = (nseg - 1) / nseg if nseg > 1 else 0.0
+    w["ssd_state"] = dict(bound="hbm", work=part * T * (H * P * es + G * N * es + H * 4)
+                          + (nseg - 1) * cfg.B * H * P * N * 4)
     w["ssd_sequential"] = dict(bound="alu", work=4.0 * T * H * P * N, bytes=ssd_bytes)
     # the scan reads every segment's local end state and writes the state entering it
-    w["segment_scan"] = dict(bound="hbm", work=2 * nseg * cfg.B * H * P * N * 4)
+    w["segment_scan"] = dict(bound="hbm", work=(2 * nseg - 1) * cfg.B * H * P * N * 4)
     w["ssd_scalars"] = dict(bound="hbm", work=T * H * 12)
     return w
 

@@ -786,6 +786,9 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
     float4 run = h0 ? reinterpret_cast<const float4 *>(h0)[((int64_t)b * H + h) * PN4 + v]
                     : make_float4(0.f, 0.f, 0.f, 0.f);
     float dtot = 1.f;
+    // Local end states exist for all segments but a sequence's last one, unless the caller wants the
+    // state after the last segment (a sequence shard's summary): that one was computed too.
+    const int nlocal = (end_state || end_decay) ? nseg : nseg - 1;
     // the loads do not depend on the running state: four segments are fetched at a time
     constexpr int U = 4;
     for (int s0 = 0; s0 < nseg; s0 += U) {
@@ -794,7 +797,7 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
 #pragma unroll
         for (int q = 0; q < U; ++q) {
             const int s = s0 + q;
-            if (s < nseg) {
+            if (s < nlocal) {
                 loc[q] = reinterpret_cast<const float4 *>(states)[((sb + s) * H + h) * PN4 + v];
                 d[q] = seg_decay[(sb + s) * H + h];
             }
@@ -804,6 +807,7 @@ segment_scan_kernel(float *__restrict__ states, const float *__restrict__ seg_de
             const int s = s0 + q;
             if (s < nseg) {
                 reinterpret_cast<float4 *>(states)[((sb + s) * H + h) * PN4 + v] = run;
+                if (s >= nlocal) continue;
                 run.x = fmaf(d[q], run.x, loc[q].x);
                 run.y = fmaf(d[q], run.y, loc[q].y);
                 run.z = fmaf(d[q], run.z, loc[q].z);
@@ -1215,7 +1219,8 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         float *decay = states + (size_t)B * nseg * H * SP * SN;
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
         {
-            const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)nseg, H, G, (unsigned)B);
+            // (the last segment's end state is nobody's entry state: the full pass produces it)
+            const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)(nseg - 1), H, G, (unsigned)B);
             if (rc != SWIMBA_OK) return rc;
         }
         const int PN4 = SP * SN / 4;
