@@ -753,7 +753,9 @@ def bench_serving(sb, steps: int = 10, warmup: int = 3):
     while sum(mixed) > Tmax:
         mixed.pop()
     mixes.append(("%d sequences, lengths log-uniform in [16, 4096]" % len(mixed), mixed))
+    mixes.append(("one 16384-token prompt", [16384]))
     mixes.append(("one 16384-token prompt among 64 single-token sequences", [16384] + [1] * 64))
+    mixes.append(("64 single-token sequences", [1] * 64))
     for name, lens in mixes:
         cu = [0]
         for v in lens:

@@ -135,6 +135,13 @@ int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *
                           const float *h0, int B, int L, int H, int P, int N, int G, void *y,
                           float *h_final);
 
+// The per-timestep evaluation over n listed sequences of a packed batch (bf16 streams): seq_tab[i] =
+// (first token, tokens, sequence index, 0), a device array; x, BC, dt, y are the packed arrays, h0 /
+// h_final are indexed by the sequence.
+int launch_ssd_sequential_listed(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                                 const float *dt_bias, const float *D, const float *h0, const int4 *seq_tab, int n,
+                                 int H, int P, int N, int G, void *y, float *h_final);
+
 // K4: one-token state update, state[B,H,P,N] in place.
 // BC [B,S] is fp32 when bc_fp32, else bf16.
 int launch_decode_update(LaunchCtx &ctx, int dtype, const void *x, const void *BC, bool bc_fp32,

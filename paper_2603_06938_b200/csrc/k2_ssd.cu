@@ -1247,6 +1247,7 @@ struct PackedPlan {
     std::vector<SeqDesc> seqs;        // nseq + 1
     std::vector<int2> tiles;          // (first token, valid tokens) per tile
     std::vector<int2> items, pre;     // (sequence, segment): all of them / those whose end state the scan needs
+    std::vector<int4> shorts;         // (first token, tokens, sequence, 0) of the sequences stepped token by token
     int total_tiles = 0, total_segs = 0, seg_len = 0;
     bool segmented = false;
 };
@@ -1254,8 +1255,13 @@ struct PackedPlan {
 PackedPlan packed_plan(const int32_t *cu, int nseq, int H, int G, int chunk, int sm_count)
 {
     PackedPlan pl;
+    // Sequences of a few tokens (decode tokens riding in a prefill batch) do not take a 128-token
+    // tile and a CTA per head pair each: they are stepped token by token, one block per head.
+    constexpr int SHORT_MAX = 4;
+    auto is_short = [&](int b) { const int len = cu[b + 1] - cu[b]; return len >= 1 && len <= SHORT_MAX; };
     int64_t tiles = 0;
-    for (int b = 0; b < nseq; ++b) tiles += ceil_div(cu[b + 1] - cu[b], ST);
+    for (int b = 0; b < nseq; ++b)
+        if (!is_short(b)) tiles += ceil_div(cu[b + 1] - cu[b], ST);
     const int64_t pairs = (int64_t)G * pairs_per_group(H, G);
     const int q_tiles = chunk >= ST ? chunk / ST : 1;
     int64_t seg_tiles = ceil_div64(tiles * pairs, sm_count);
@@ -1267,6 +1273,12 @@ PackedPlan packed_plan(const int32_t *cu, int nseq, int H, int G, int chunk, int
     int tile0 = 0, seg0 = 0;
     for (int b = 0; b < nseq; ++b) {
         const int len = cu[b + 1] - cu[b];
+        if (is_short(b)) {
+            pl.seqs[b] = SeqDesc{cu[b], len, tile0, seg0};
+            pl.shorts.push_back(make_int4(cu[b], len, b, 0));
+            seg0 += 1;                                   // (keeps one segment slot, unused)
+            continue;
+        }
         const int nt = ceil_div(len, ST);
         const int ns = len > 0 ? ceil_div(len, pl.seg_len) : 1;
         pl.seqs[b] = SeqDesc{cu[b], len, tile0, seg0};
@@ -1287,7 +1299,7 @@ PackedPlan packed_plan(const int32_t *cu, int nseq, int H, int G, int chunk, int
 }
 
 struct PackedLayout {
-    size_t seqs, tiles, items, pre, l2, rec, states, decay, total;
+    size_t seqs, tiles, items, pre, shorts, l2, rec, states, decay, total;
 };
 PackedLayout packed_layout(const PackedPlan &pl, int nseq, int H)
 {
@@ -1298,6 +1310,7 @@ PackedLayout packed_layout(const PackedPlan &pl, int nseq, int H)
     l.tiles = off; off += up((size_t)pl.total_tiles * sizeof(int2));
     l.items = off; off += up(pl.items.size() * sizeof(int2));
     l.pre = off;   off += up(pl.pre.size() * sizeof(int2));
+    l.shorts = off; off += up(pl.shorts.size() * sizeof(int4));
     l.l2 = off;    off += up((size_t)H * pl.total_tiles * ST * sizeof(float));
     l.rec = off;   off += up((size_t)H * pl.total_tiles * sizeof(TileScalars));
     l.states = off;
@@ -1334,8 +1347,16 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
         cudaMemcpyAsync(ws + lay.tiles, pl.tiles.data(), pl.tiles.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess ||
         cudaMemcpyAsync(ws + lay.items, pl.items.data(), pl.items.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess ||
         (!pl.pre.empty() &&
-         cudaMemcpyAsync(ws + lay.pre, pl.pre.data(), pl.pre.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess))
+         cudaMemcpyAsync(ws + lay.pre, pl.pre.data(), pl.pre.size() * sizeof(int2), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess) ||
+        (!pl.shorts.empty() &&
+         cudaMemcpyAsync(ws + lay.shorts, pl.shorts.data(), pl.shorts.size() * sizeof(int4), cudaMemcpyHostToDevice, ctx.stream) != cudaSuccess))
         return SWIMBA_ERR_CUDA;
+    if (!pl.shorts.empty()) {
+        const int rc = launch_ssd_sequential_listed(ctx, x, BC, dt, A, dt_bias, D, h0, (const int4 *)(ws + lay.shorts),
+                                                    (int)pl.shorts.size(), H, SP, SN, G, y, h_final);
+        if (rc != SWIMBA_OK) return rc;
+    }
+    if (pl.items.empty()) return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 
     const int S = 2 * G * SN;
     CUtensorMap tm_bc, tm_x, tm_y;

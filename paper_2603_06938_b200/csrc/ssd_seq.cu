@@ -16,7 +16,7 @@ ssd_sequential_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
                       const float *__restrict__ dt, const float *__restrict__ A,
                       const float *__restrict__ dt_bias, const float *__restrict__ D,
                       const float *__restrict__ h0, int L, int H, int P, int N, int G, int NS,
-                      T *__restrict__ y, float *__restrict__ h_final)
+                      T *__restrict__ y, float *__restrict__ h_final, const int4 *__restrict__ seq_tab)
 {
     extern __shared__ float smem[];
     float *sB = smem;                    // [TS][N]
@@ -26,7 +26,17 @@ ssd_sequential_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
     float *sdl = sy + SEQ_TS * P;        // [TS] Delta
     float *sa = sdl + SEQ_TS;            // [TS] exp(Delta*A)
 
-    const int b = blockIdx.x / H, h = blockIdx.x % H;
+    int b = blockIdx.x / H;
+    const int h = blockIdx.x % H;
+    // seq_tab (packed batches): entry i = (first token, tokens, sequence index) of the i-th listed
+    // sequence; tokens are rows of the packed arrays, the states are indexed by the sequence
+    int64_t tok_base = (int64_t)b * L;
+    if (seq_tab) {
+        const int4 e = seq_tab[b];
+        tok_base = e.x;
+        L = e.y;
+        b = e.z;
+    }
     const int g = h / (H / G);
     const int S = 2 * G * N;
     const int tid = threadIdx.x, nthr = blockDim.x;
@@ -45,16 +55,16 @@ ssd_sequential_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
         const int nt = min(SEQ_TS, L - t0);
         for (int i = tid; i < nt * N; i += nthr) {
             const int tt = i / N, n = i % N;
-            const TBC *row = BC + ((int64_t)b * L + t0 + tt) * S;
+            const TBC *row = BC + (tok_base + t0 + tt) * S;
             sB[tt * N + n] = to_f32<TBC>(row[g * N + n]);
             sC[tt * N + n] = to_f32<TBC>(row[(G + g) * N + n]);
         }
         for (int i = tid; i < nt * P; i += nthr) {
             const int tt = i / P, pp = i % P;
-            sx[tt * P + pp] = to_f32<T>(x[(((int64_t)b * L + t0 + tt) * H + h) * P + pp]);
+            sx[tt * P + pp] = to_f32<T>(x[((tok_base + t0 + tt) * H + h) * P + pp]);
         }
         for (int i = tid; i < nt; i += nthr) {        // (blocks may have fewer than SEQ_TS threads)
-            const float raw = dt ? dt[((int64_t)b * L + t0 + i) * H + h] : 0.f;
+            const float raw = dt ? dt[(tok_base + t0 + i) * H + h] : 0.f;
             const float delta = softplus_f(raw + bias);
             sdl[i] = delta;
             sa[i] = expf(delta * Ah);
@@ -78,7 +88,7 @@ ssd_sequential_kernel(const T *__restrict__ x, const TBC *__restrict__ BC,
         __syncthreads();
         for (int i = tid; i < nt * P; i += nthr) {
             const int tt = i / P, pp = i % P;
-            y[(((int64_t)b * L + t0 + tt) * H + h) * P + pp] = from_f32<T>(sy[tt * P + pp]);
+            y[((tok_base + t0 + tt) * H + h) * P + pp] = from_f32<T>(sy[tt * P + pp]);
         }
         __syncthreads();
     }
@@ -101,7 +111,8 @@ static int seq_ns(int N)
 template <typename T, typename TBC>
 static int launch_seq_t(LaunchCtx &ctx, const void *x, const void *BC, const float *dt,
                         const float *A, const float *dt_bias, const float *D, const float *h0,
-                        int B, int L, int H, int P, int N, int G, void *y, float *h_final)
+                        int B, int L, int H, int P, int N, int G, void *y, float *h_final,
+                        const int4 *seq_tab = nullptr)
 {
     const int NS = seq_ns(N);
     const size_t smem = sizeof(float) * (size_t)(2 * SEQ_TS * N + 2 * SEQ_TS * P + 2 * SEQ_TS);
@@ -109,7 +120,7 @@ static int launch_seq_t(LaunchCtx &ctx, const void *x, const void *BC, const flo
     if (smem > 48 * 1024 && !ensure_dynamic_smem((const void *)kern, smem)) return SWIMBA_ERR_CUDA;
     ctx.begin(STAGE_SSD_SEQUENTIAL);
     kern<<<B * H, P * NS, smem, ctx.stream>>>((const T *)x, (const TBC *)BC, dt, A, dt_bias, D, h0,
-                                             L, H, P, N, G, NS, (T *)y, h_final);
+                                             L, H, P, N, G, NS, (T *)y, h_final, seq_tab);
     ctx.end();
     return cudaGetLastError() == cudaSuccess ? SWIMBA_OK : SWIMBA_ERR_CUDA;
 }
@@ -125,6 +136,19 @@ int launch_ssd_sequential(LaunchCtx &ctx, int dtype, const void *x, const void *
     if (bc_fp32)
         return launch_seq_t<__nv_bfloat16, float>(ctx, x, BC, dt, A, dt_bias, D, h0, B, L, H, P, N, G, y, h_final);
     return launch_seq_t<__nv_bfloat16, __nv_bfloat16>(ctx, x, BC, dt, A, dt_bias, D, h0, B, L, H, P, N, G, y, h_final);
+}
+
+// The same over a list of sequences of a packed batch (device table of n entries: first token,
+// tokens, sequence index); bf16 streams.  Used for the sequences of a packed batch that are only a
+// few tokens long (decode tokens riding in a prefill batch): one block per (sequence, head) reads
+// the state, steps through the tokens and writes the state, instead of a 128-token tile each.
+int launch_ssd_sequential_listed(LaunchCtx &ctx, const void *x, const void *BC, const float *dt, const float *A,
+                                 const float *dt_bias, const float *D, const float *h0, const int4 *seq_tab, int n,
+                                 int H, int P, int N, int G, void *y, float *h_final)
+{
+    if (n <= 0) return SWIMBA_OK;
+    return launch_seq_t<__nv_bfloat16, __nv_bfloat16>(ctx, x, BC, dt, A, dt_bias, D, h0, n, 0, H, P, N, G, y, h_final,
+                                                      seq_tab);
 }
 
 // ------------------------------------------------------------------------------------------
