@@ -51,7 +51,7 @@ NCU_TRAFFIC_BYTES = {
     # profiles/forward_mid_kernels.md
     "mid": {"ssd_scalars": 8.413e6, "router_topk": 147.366e6, "expert_gemm": 258.593e6, "ssd_tiles": 580.232e6},
     # profiles/ssd_segmented_long_seq.md (the state-only pass is a kernel of its own)
-    "long_seq": {"ssd_state": 308.766e6, "ssd_tiles": 619.744e6, "segment_scan": 18.883e6},
+    "long_seq": {"ssd_state": 306.295e6, "ssd_tiles": 619.417e6, "segment_scan": 17.843e6},
     # profiles/decode_step_kernels.md
     "decode": {"router_topk": 0.593e6, "project_small": 9.071e6, "decode_update": 479.881e6},
 }
