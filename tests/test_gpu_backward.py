@@ -118,3 +118,16 @@ def test_backward_rejects_and_empty_batch():
         assert float(dWr.abs().max()) == 0.0 and float(dWe.abs().max()) == 0.0
     finally:
         sb.swimba_destroy(h)
+
+
+def test_weight_gradients_without_step_sizes_or_initial_state():
+    cfg = cfg_of("bf16", L=200, H=4, G=2)
+    inp = synth.make_inputs(cfg, seed=97, with_dt=False)
+    gen = torch.Generator().manual_seed(5)
+    dy = torch.randn(cfg.B, cfg.L, cfg.H, cfg.P, generator=gen).to(torch.bfloat16)
+    dWr, dWe, idx = gpu_backward(cfg, inp, dy, h0=None)
+    ref = oracle.backward_weights(synth.f64(inp["u"]), synth.f64(inp["x"]), None, synth.f64(inp["W_r"]),
+                                  synth.f64(inp["W_e"]), synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), synth.f64(dy),
+                                  k=cfg.k, G=cfg.G, h0=None, forced_idx=idx.numpy())
+    assert rel_per_expert(dWe, ref["dW_e"]) <= 2e-2
+    assert np.abs(dWr.double().numpy() - ref["dW_r"]).max() <= 2e-2 * np.abs(ref["dW_r"]).max()

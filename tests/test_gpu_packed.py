@@ -179,3 +179,30 @@ def test_packed_rejects_bad_offsets():
         assert float(y.abs().max()) == 0.0
     finally:
         sb.swimba_destroy(h)
+
+
+def test_packed_without_step_sizes_initial_states_or_final_states():
+    # dt == NULL (the literal time-invariant transition), h0 == NULL, h_final == NULL, two B/C groups
+    lens = [140, 2, 391]
+    cfg = cfg_of(H=4, G=2, L=int(sum(lens)))
+    inp = synth.make_inputs(cfg, seed=59, with_dt=False)
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    h = hp.create_handle(cfg)
+    try:
+        w, keep = hp.device_weights(inp)
+        u, x = hp.dev(inp["u"][0]), hp.dev(inp["x"][0])
+        y = torch.full_like(x, float("nan"))
+        idx = torch.full((cfg.L, cfg.k), -1, dtype=torch.int32, device="cuda")
+        wt = torch.full((cfg.L, cfg.k), float("nan"), device="cuda")
+        ws = torch.zeros(sb.swimba_packed_workspace_bytes(h, cu), dtype=torch.uint8, device="cuda")
+        sb.swimba_forward_packed(h, w, u, x, None, None, cu, y, None, idx, wt, ws)
+        assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+        hf = torch.full((len(lens), cfg.H, cfg.P, cfg.N), float("nan"), device="cuda")
+        y2 = torch.full_like(x, float("nan"))
+        sb.swimba_forward_packed(h, w, u, x, None, None, cu, y2, hf, idx, wt, ws)
+        assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+        assert torch.equal(y, y2)
+    finally:
+        sb.swimba_destroy(h)
+    got = dict(y=y.cpu(), h_final=hf.cpu(), idx=idx.cpu(), w=wt.cpu())
+    check_packed(cfg, inp, lens, got)
