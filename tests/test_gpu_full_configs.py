@@ -79,3 +79,53 @@ def test_decode_full_size_every_step_every_sequence(skip_term):
     res = hp.compare_forward(full_cfg, inp, got, 2e-2, 1e-2)
     print(f"decode {'D' if skip_term else 'noD'}: err_y={res['err_y']:.3e} err_h={res['err_h']:.3e} "
           f"elementwise p99.9={res['err_y_elem_p999']:.3e} ambiguous={res['ambiguous']}")
+
+
+def test_packed_full_size_mixed_lengths():
+    """The serving-shaped batch the benchmark times (mid layer shape, sequences of log-uniform
+    lengths, 31 746 tokens in all, a decode token and a long prompt among them): every sequence
+    against the oracle run on its own tokens."""
+    import math
+    import test_gpu_packed as tp
+    base = synth.CONFIGS["mid"]
+    lg = torch.Generator().manual_seed(11)
+    lens = [int(v) for v in torch.exp(torch.rand(48, generator=lg) * (math.log(4096) - math.log(16)) + math.log(16))]
+    while sum(lens) > 32768:
+        lens.pop()
+    lens[3] = 1                                   # a decode token riding in the batch
+    cfg = dataclasses.replace(base, B=1, L=int(sum(lens)))
+    inp = synth.make_inputs(cfg, seed=23)
+    gen = torch.Generator().manual_seed(29)
+    h0 = (0.1 * torch.randn(len(lens), cfg.H, cfg.P, cfg.N, generator=gen)).float()
+    got = tp.packed_forward(cfg, inp, lens, h0=h0)
+    worst = tp.check_packed(cfg, inp, lens, got, h0=h0)
+    print(f"packed mid-shape, {len(lens)} sequences, {cfg.L} tokens: err_y={worst['err_y']:.3e} err_h={worst['err_h']:.3e}")
+
+
+def test_sharded_full_size_long_seq():
+    """long_seq cut into 8 shards of 8192 tokens (the ranks emulated one after the other): the
+    concatenated outputs against the oracle on the whole 65 536-token sequence."""
+    import test_gpu_sharded as ts
+    cfg = synth.CONFIGS["long_seq"]
+    inp = synth.make_inputs(cfg, seed=3)
+    got = ts.sharded_forward(cfg, inp, [cfg.L // 8] * 8)
+    full = dict(y=got["y"], h_final=got["ends"][-1], idx=got["idx"], w=got["w"])
+    res = hp.compare_forward(cfg, inp, full, *hp.tolerances(cfg))
+    print(f"sharded long_seq: err_y={res['err_y']:.3e} err_h={res['err_h']:.3e} ambiguous={res['ambiguous']}")
+
+
+def test_backward_full_size_small_lm():
+    """Weight gradients at the small_lm workload against the oracle's, per expert."""
+    import test_gpu_backward as tb
+    cfg = synth.CONFIGS["small_lm"]
+    inp = synth.make_inputs(cfg, seed=1)
+    gen = torch.Generator().manual_seed(31)
+    dy = torch.randn(cfg.B, cfg.L, cfg.H, cfg.P, generator=gen).to(torch.bfloat16)
+    dWr, dWe, idx = tb.gpu_backward(cfg, inp, dy, h0=None)
+    ref = oracle.backward_weights(synth.f64(inp["u"]), synth.f64(inp["x"]), synth.f64(inp["dt"]), synth.f64(inp["W_r"]),
+                                  synth.f64(inp["W_e"]), synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), synth.f64(dy),
+                                  k=cfg.k, G=cfg.G, h0=None, forced_idx=idx.numpy())
+    err_e = tb.rel_per_expert(dWe, ref["dW_e"])
+    err_r = float(np.abs(dWr.double().numpy() - ref["dW_r"]).max() / np.abs(ref["dW_r"]).max())
+    print(f"backward small_lm: dW_e per-expert err={err_e:.3e} dW_r err={err_r:.3e}")
+    assert err_e <= 2e-2 and err_r <= 2e-2
