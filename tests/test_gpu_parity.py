@@ -395,3 +395,44 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     ref = hp.oracle_forward(cfg, inp)
     hp.check_outputs(cfg, inp, y, hf, ref, 2e-2, 1e-2)
     sb.swimba_destroy(h)
+
+
+def test_decode_steps_replay_from_a_cuda_graph():
+    """The decode step enqueues kernels and nothing else (no allocation, no synchronisation), so a
+    run of steps can be captured once and replayed: the replay must reproduce the eager steps bit
+    for bit (same kernels, same order)."""
+    cfg = cfg_of("bf16", B=16, L=1, F=256, H=4, E=8, k=2)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(6)
+    wts = {n: v.cuda() for n, v in synth.make_weights(cfg, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    toks = [{n: v.cuda() for n, v in synth.make_decode_step_inputs(cfg, gen).items()} for _ in range(4)]
+    state0 = (0.1 * torch.randn(cfg.B, cfg.H, cfg.P, cfg.N, generator=gen)).cuda()
+    state = state0.clone()
+    y = torch.empty(4, *toks[0]["x"].shape, dtype=toks[0]["x"].dtype, device="cuda")
+    h = hp.create_handle(cfg)
+    try:
+        ws = torch.empty(sb.swimba_decode_workspace_bytes(h, cfg.B), dtype=torch.uint8, device="cuda")
+
+        def run(stream=None):
+            for i, t in enumerate(toks):
+                sb.swimba_decode_step(h, w, t["u"], t["x"], t["dt"], state, cfg.B, y[i], None, None, ws, stream=stream)
+
+        run()                                      # eager (also warms the handle's caches)
+        torch.cuda.synchronize()
+        y_eager, s_eager = y.clone(), state.clone()
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                run(side)
+        torch.cuda.synchronize()
+        state.copy_(state0)
+        y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+        assert torch.equal(y, y_eager) and torch.equal(state, s_eager)
+    finally:
+        sb.swimba_destroy(h)
