@@ -1,0 +1,78 @@
+"""GPU parity on seeded random shapes: every case draws batch, length, widths, heads, groups,
+experts, top-k, chunk and which optional arguments are present, runs the forward through the C ABI
+and compares it with the oracle under the same protocol and tolerances as test_gpu_parity.  The
+draws favour the corners the fixed cases visit one at a time (odd head counts per group, one head,
+k == E, lengths around tile and segment boundaries), here in combination."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2603_06938_b200 import synth
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def draw(seed):
+    r = np.random.default_rng(1000 + seed)
+    kind = r.choice(["tile", "tile", "tile", "bf16_other", "fp32"])
+    G = int(r.choice([1, 1, 2, 3]))
+    H = G * int(r.integers(1, 5))
+    if kind == "tile":
+        dtype, P, N = "bf16", 64, 128
+    elif kind == "bf16_other":
+        dtype, P, N = "bf16", int(r.choice([8, 16, 32, 64])), int(r.choice([16, 32, 64]))
+    else:
+        dtype, P, N = "fp32", int(r.choice([8, 16, 64])), int(r.choice([16, 32, 128]))
+    E = int(r.choice([1, 2, 3, 4, 8, 16]))
+    k = int(r.integers(1, min(E, 4) + 1))
+    F = 8 * int(r.integers(1, 66))
+    B = int(r.integers(1, 6))
+    L = int(r.choice([1, int(r.integers(2, 130)), int(r.integers(120, 140)), int(r.integers(250, 700)),
+                      int(r.integers(1000, 3000))]))
+    if kind != "tile":
+        L = min(L, 400)
+    Q = int(r.choice([64, 128, 256]))
+    cfg = synth.LayerConfig("fuzz", dtype, B, L, F, H, P, N, G, E, k, Q, h0_std=float(r.choice([0.0, 0.1])))
+    return cfg, bool(r.integers(0, 2)), bool(r.integers(0, 4) > 0)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_shapes_match_oracle(seed):
+    cfg, use_D, use_dt = draw(seed)
+    inp = synth.make_inputs(cfg, seed=seed, with_dt=use_dt)
+    if not use_D:
+        inp["D"] = None
+    got = hp.gpu_forward(cfg, inp)
+    res = hp.compare_forward(cfg, inp, got, *hp.tolerances(cfg))
+    print(cfg, "D" if use_D else "noD", "dt" if use_dt else "nodt",
+          f"err_y={res['err_y']:.2e} err_h={res['err_h']:.2e} ambiguous={res['ambiguous']}")
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_packed_batches_match_oracle(seed):
+    import test_gpu_packed as tp
+    r = np.random.default_rng(2000 + seed)
+    nseq = int(r.integers(1, 9))
+    lens = [int(r.choice([0, 1, int(r.integers(2, 6)), int(r.integers(6, 140)), int(r.integers(140, 600)),
+                          int(r.integers(600, 2500))])) for _ in range(nseq)]
+    if sum(lens) == 0:
+        lens[0] = 37
+    tile = bool(r.integers(0, 4) > 0)
+    G = int(r.choice([1, 2]))
+    H = G * int(r.integers(1, 4))
+    E = int(r.choice([1, 4, 8]))
+    k = int(r.integers(1, min(E, 3) + 1))
+    if tile:
+        cfg = synth.LayerConfig("fuzz", "bf16", 1, int(sum(lens)), 8 * int(r.integers(4, 40)), H, 64, 128, G, E, k, 128)
+    else:
+        lens = [min(v, 200) for v in lens]
+        cfg = synth.LayerConfig("fuzz", str(r.choice(["bf16", "fp32"])), 1, int(sum(lens)), 8 * int(r.integers(4, 40)), H,
+                                int(r.choice([16, 32])), int(r.choice([16, 64])), G, E, k, 128)
+    inp = synth.make_inputs(cfg, seed=seed)
+    gen = torch.Generator().manual_seed(seed)
+    h0 = (0.1 * torch.randn(len(lens), cfg.H, cfg.P, cfg.N, generator=gen)).float() if r.integers(0, 2) else None
+    got = tp.packed_forward(cfg, inp, lens, h0=h0)
+    worst = tp.check_packed(cfg, inp, lens, got, h0=h0)
+    print(cfg.dtype, cfg.P, cfg.N, lens, f"err_y={worst['err_y']:.2e} err_h={worst['err_h']:.2e}")
