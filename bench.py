@@ -530,8 +530,12 @@ def main():
         shard = bench_shard(sb)
 
     backward = None
+    general = None
+    block = None
     if single and not args.no_serving:
         backward = {name: bench_backward(sb, synth.CONFIGS[name]) for name in ("small_lm", "mid")}
+        general = {name: bench_general(sb, synth.CONFIGS[name]) for name in ("small_lm", "mid")}
+        block = {name: bench_block(sb, synth.CONFIGS[name]) for name in ("small_lm", "mid")}
 
     cpu = None
     if single and not args.no_cpu_baseline:
@@ -551,6 +555,7 @@ def main():
             "ssd_segments": nseg,
             "kernels": kernels, "comparators": comparators, "workloads": workloads,
             "decode": decode, "serving": serving, "sequence_sharded": shard, "backward_weights": backward,
+            "general_form": general, "block_forward": block,
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
@@ -615,6 +620,109 @@ def bench_decode(sb, pk, steps: int = 512, warmup: int = 8):
     }
     sb.swimba_destroy(h)
     return out
+
+
+def _timed_calls(fn, steps, warmup):
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        fn(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def _kernel_ms(sb, h, fns):
+    """Per-kernel milliseconds of one pass through the given calls (event-bracketed)."""
+    sb.swimba_profile(h, True)
+    per = {}
+    for fn in fns:
+        fn(0)
+        torch.cuda.synchronize()
+        for name, t in sb.swimba_profile_read(h):
+            per[name] = per.get(name, 0.0) + t
+    sb.swimba_profile(h, False)
+    return per
+
+
+def bench_general(sb, cfg, steps: int = 10, warmup: int = 3):
+    """The general form of the layer (expert-specific SSM inputs): swimba_route_project_slots, then
+    swimba_ssd_slots on given per-slot inputs, for one batch of the workload.  Not tuned: the state
+    equation is evaluated as k chunked recurrences."""
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(31)
+    wts = {n: v.cuda() for n, v in synth.make_weights(cfg, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], None)
+    dgen = torch.Generator(device="cuda")
+    dgen.manual_seed(32)
+    B, L, T = cfg.B, cfg.L, cfg.tokens
+    u = torch.randn(B, L, cfg.F, generator=dgen, device="cuda").bfloat16()
+    x_slots = torch.randn(cfg.k, B, L, cfg.H, cfg.P, generator=dgen, device="cuda").bfloat16()
+    dt = 0.5 * torch.randn(B, L, cfg.H, generator=dgen, device="cuda")
+    BCs = torch.empty(T, cfg.k, cfg.S, dtype=torch.bfloat16, device="cuda")
+    y = torch.empty(B, L, cfg.H, cfg.P, dtype=torch.bfloat16, device="cuda")
+    hf = torch.empty(B, cfg.H, cfg.P, cfg.N, device="cuda")
+    ws = torch.empty(sb.swimba_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+    ws2 = torch.empty(sb.swimba_ssd_slots_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+
+    def first(i):
+        sb.swimba_route_project_slots(h, w, u, T, BCs, None, None, ws)
+
+    def second(i):
+        sb.swimba_ssd_slots(h, w, x_slots, BCs, dt, None, B, L, y, hf, ws2)
+
+    def step(i):
+        first(i)
+        second(i)
+
+    ms = _timed_calls(step, steps, warmup)
+    per = _kernel_ms(sb, h, [first, second])
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    return {"workload": config_dict(cfg)["workload"], "ms": ms, "tokens_per_s": cfg.tokens / (ms * 1e-3),
+            "kernel_ms": per}
+
+
+def bench_block(sb, cfg, steps: int = 10, warmup: int = 3, d_conv: int = 4):
+    """The whole block around the mixer (swimba_block_forward: in-projection, convolution + SiLU,
+    routing and projection, the recurrence, gated norm, out-projection) for one batch of the
+    workload.  Not tuned: the linear maps run through the grouped projection with one expert."""
+    h = sb.swimba_create(cfg.F, cfg.H, cfg.P, cfg.N, cfg.G, cfg.E, cfg.k, cfg.Q, sb.DTYPE_BF16)
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(41)
+    wts = {n: v.cuda() for n, v in synth.make_weights(cfg, gen).items()}
+    w = sb.make_weights(wts["W_r"], wts["W_e"], wts["A"], wts["dt_bias"], wts["D"])
+    dgen = torch.Generator(device="cuda")
+    dgen.manual_seed(42)
+    B, L = cfg.B, cfg.L
+    D = cfg.H * cfg.P
+    W_in = (torch.randn(2 * D + cfg.H, cfg.F, generator=dgen, device="cuda") / cfg.F ** 0.5).bfloat16()
+    conv_w = 0.5 * torch.randn(D + cfg.S, d_conv, generator=dgen, device="cuda")
+    conv_b = 0.1 * torch.randn(D + cfg.S, generator=dgen, device="cuda")
+    norm_w = 1.0 + 0.1 * torch.randn(D, generator=dgen, device="cuda")
+    W_out = (torch.randn(cfg.F, D, generator=dgen, device="cuda") / D ** 0.5).bfloat16()
+    bw = sb.make_block_weights(W_in, conv_w, conv_b, norm_w, W_out, d_conv)
+    u = torch.randn(B, L, cfg.F, generator=dgen, device="cuda").bfloat16()
+    out = torch.empty_like(u)
+    cst = torch.empty(B, d_conv - 1, D + cfg.S, dtype=torch.bfloat16, device="cuda")
+    hf = torch.empty(B, cfg.H, cfg.P, cfg.N, device="cuda")
+    ws = torch.empty(sb.swimba_block_workspace_bytes(h, B, L), dtype=torch.uint8, device="cuda")
+
+    def step(i):
+        sb.swimba_block_forward(h, w, bw, u, None, None, B, L, out, cst, hf, None, None, ws)
+
+    ms = _timed_calls(step, steps, warmup)
+    per = _kernel_ms(sb, h, [step])
+    assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    sb.swimba_destroy(h)
+    flops = 2.0 * cfg.tokens * cfg.F * (2 * D + cfg.H) + 2.0 * cfg.tokens * D * cfg.F
+    return {"workload": config_dict(cfg)["workload"], "ms": ms, "tokens_per_s": cfg.tokens / (ms * 1e-3),
+            "kernel_ms": per, "linear_map_flops": flops}
 
 
 def bench_backward(sb, cfg, steps: int = 5, warmup: int = 2):
