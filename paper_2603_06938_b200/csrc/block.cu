@@ -9,7 +9,7 @@ namespace swimba {
 
 namespace {
 constexpr int CV_K = 4;        // widest convolution window
-constexpr int CV_STRIP = 32;   // tokens per thread
+constexpr int CV_STRIP = 8;    // tokens per thread
 
 __device__ __forceinline__ float silu_f(float v) { return v / (1.f + __expf(-v)); }
 
@@ -34,7 +34,7 @@ template <> __device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16 
 // (zeros when null).  A thread owns 8 channels and a strip of CV_STRIP tokens and slides its
 // window along the strip; the thread of a sequence's last strip also writes state_out.
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 conv_silu_kernel(const T *__restrict__ xp, int64_t ldx, const T *__restrict__ bcp, const float *__restrict__ cw,
                  const float *__restrict__ cb, const T *__restrict__ state_in, int B, int L, int D, int S,
                  int K, T *__restrict__ x, T *__restrict__ bc, T *__restrict__ state_out)
@@ -55,13 +55,27 @@ conv_silu_kernel(const T *__restrict__ xp, int64_t ldx, const T *__restrict__ bc
     const int64_t ldd = from_x ? (int64_t)D : (int64_t)S;
     // taps aligned to the end of a window of CV_K: tap j multiplies the token CV_K-1-j steps back
     float wt[CV_K][8], bias[8];
+    if (cb) {
+        load8(cb + c0, bias);
+    } else {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        bias[q] = cb ? cb[c0 + q] : 0.f;
+        for (int q = 0; q < 8; ++q) bias[q] = 0.f;
+    }
+    if (K == CV_K) {
+        // one 16-byte load per channel: its four taps
 #pragma unroll
-        for (int j = 0; j < CV_K; ++j) {
-            const int i = j - (CV_K - K);
-            wt[j][q] = i >= 0 ? cw[(int64_t)(c0 + q) * K + i] : 0.f;
+        for (int q = 0; q < 8; ++q) {
+            const float4 t4 = *reinterpret_cast<const float4 *>(cw + (int64_t)(c0 + q) * CV_K);
+            wt[0][q] = t4.x; wt[1][q] = t4.y; wt[2][q] = t4.z; wt[3][q] = t4.w;
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+#pragma unroll
+            for (int j = 0; j < CV_K; ++j) {
+                const int i = j - (CV_K - K);
+                wt[j][q] = i >= 0 ? cw[(int64_t)(c0 + q) * K + i] : 0.f;
+            }
         }
     }
     const int t0 = strip * CV_STRIP;
@@ -76,25 +90,29 @@ conv_silu_kernel(const T *__restrict__ xp, int64_t ldx, const T *__restrict__ bc
             for (int q = 0; q < 8; ++q) v[q] = 0.f;
         }
     };
+    // all rows of the strip and its history are loaded first (raw, so that they are in flight
+    // together), then widened one by one into the sliding window
+    typename Raw8<T>::type raw[CV_STRIP];
+    const int t1 = min(L, t0 + CV_STRIP);
+#pragma unroll
+    for (int r = 0; r < CV_STRIP; ++r)
+        if (t0 + r < t1) load_raw8(src + ((int64_t)b * L + t0 + r) * lds, raw[r]);
     float win[CV_K][8];
 #pragma unroll
     for (int j = 0; j < CV_K - 1; ++j) fetch(t0 - (CV_K - 1) + j, win[j]);
-    const int t1 = min(L, t0 + CV_STRIP);
-    for (int t = t0; t < t1; ++t) {
-        fetch(t, win[CV_K - 1]);
+#pragma unroll
+    for (int r = 0; r < CV_STRIP; ++r) {
+        if (t0 + r >= t1) break;
+        unpack8(raw[r], win[(r + CV_K - 1) % CV_K]);
         float o[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             float acc = bias[q];
 #pragma unroll
-            for (int j = 0; j < CV_K; ++j) acc = fmaf(wt[j][q], win[j][q], acc);
+            for (int j = 0; j < CV_K; ++j) acc = fmaf(wt[j][q], win[(r + j) % CV_K][q], acc);
             o[q] = silu_f(acc);
         }
-        store8<T>(dst + ((int64_t)b * L + t) * ldd, o);
-#pragma unroll
-        for (int j = 0; j < CV_K - 1; ++j)
-#pragma unroll
-            for (int q = 0; q < 8; ++q) win[j][q] = win[j + 1][q];
+        store8<T>(dst + ((int64_t)b * L + t0 + r) * ldd, o);
     }
     if (state_out && strip == nstrip - 1) {
         for (int i = 0; i < K - 1; ++i) {
