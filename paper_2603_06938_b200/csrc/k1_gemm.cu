@@ -135,13 +135,6 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
     if (uwarp < 4) {
         // ---- gather producers: thread -> 16-byte chunk (lane & 7) of rows 4 i + (lane >> 3)
         // of its warp's 64-row quarter
-        // router weights of the two rows this thread scales in the epilogue (needed much later)
-        float wr2[2];
-#pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-            const int row = hf * 128 + warp * 32 + lane;
-            wr2[hf] = (row < nrows && row_src[row] >= 0) ? w_slot[perm[row0 + row]] : 0.f;
-        }
         int tsrc[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) tsrc[i] = row_src[warp * 64 + i * 4 + (lane >> 3)];
@@ -170,6 +163,14 @@ expert_gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __nv_bfloat
         tc::fence_proxy_async_smem();
         for (int kb = (KB > GM_LAG ? KB - GM_LAG : 0); kb < KB; ++kb)
             tc::mbar_arrive(&full[kb % STAGES]);
+        // router weights of the two rows this thread scales in the epilogue: a dependent pair of
+        // loads, fetched here, under the last products, instead of in front of the first gather
+        float wr2[2];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const int row = hf * 128 + warp * 32 + lane;
+            wr2[hf] = (row < nrows && row_src[row] >= 0) ? w_slot[perm[row0 + row]] : 0.f;
+        }
 
         // ---- epilogue: thread = output row of each half.  All MMAs have completed, so the
         // pipeline buffers are free: the scaled bf16 rows are staged there (row stride padded by
