@@ -870,8 +870,10 @@ shard_entry_kernel(float *__restrict__ states, const float *__restrict__ seg_dec
 // stage.  The state is read from tensor memory once, at the end.
 namespace {
 constexpr int NQ = 4;                                   // heads per CTA
-constexpr int ST_STAGES = 2;
-constexpr uint32_t ST_STAGE_BYTES = (2 + NQ) * SLAB;    // B0 B1 X0 X1 X2 X3
+constexpr int ST_STAGES = 4;
+constexpr int HT = 64;                                  // tokens per ring stage: half a tile
+constexpr uint32_t HSLAB = SLAB / 2;                    // 64 rows x 128 bytes
+constexpr uint32_t ST_STAGE_BYTES = (2 + NQ) * HSLAB;   // B0 B1 X0 X1 X2 X3
 constexpr uint32_t ST_SMALL = ST_STAGES * ST_STAGE_BYTES;
 constexpr int ST_THREADS = 32 * (4 * NQ + 2);
 constexpr uint32_t ST_TM_COLS = NQ * 64 < 32 ? 32 : NQ * 64;
@@ -922,6 +924,7 @@ ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     const int t_begin = seg * prm.seg_len;
     const int t_end = min(L, t_begin + prm.seg_len);
     const int ntiles = (t_end - t_begin + ST - 1) / ST;
+    const int nhalves = (t_end - t_begin + HT - 1) / HT;     // ring stages: half tiles that hold tokens
 
     if (tid == 0) {
         for (int s = 0; s < ST_STAGES; ++s) {
@@ -952,19 +955,19 @@ ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
     if (uwarp == 4 * NQ) {
         // ------------------------------------------------------------------ TMA producer
         const bool leader = tc::elect_one();
-        for (int j = 0; j < ntiles; ++j) {
-            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+        for (int q = 0; q < nhalves; ++q) {
+            const int s = q % ST_STAGES, ph = (q / ST_STAGES) & 1;
             tc::mbar_wait(&sm->empty[s], ph ^ 1, abort_flag, d_status);
             if (leader) {
                 uint8_t *stg = smem + s * ST_STAGE_BYTES;
-                const int t0 = tok0 + t_begin + j * ST;
-                tc::mbar_arrive_expect_tx(&sm->full[s], (2 + nh) * SLAB + nh * (uint32_t)sizeof(TileScalars));
+                const int t0 = tok0 + t_begin + q * HT;
+                tc::mbar_arrive_expect_tx(&sm->full[s], (2 + nh) * HSLAB + nh * (uint32_t)sizeof(TileScalars));
                 tc::tma_load_3d(stg, &tmap_bc, &sm->full[s], g * SN, t0, bco);
-                tc::tma_load_3d(stg + SLAB, &tmap_bc, &sm->full[s], g * SN + 64, t0, bco);
+                tc::tma_load_3d(stg + HSLAB, &tmap_bc, &sm->full[s], g * SN + 64, t0, bco);
                 for (int hd = 0; hd < nh; ++hd) {
-                    tc::tma_load_4d(stg + (2 + hd) * SLAB, &tmap_x, &sm->full[s], 0, head0 + hd, t0, bco);
+                    tc::tma_load_4d(stg + (2 + hd) * HSLAB, &tmap_x, &sm->full[s], 0, head0 + hd, t0, bco);
                     tc::bulk_load(&sm->sc[s][hd],
-                                  prm.rec + rec_base + (int64_t)(head0 + hd) * rec_hstride + t_begin / ST + j,
+                                  prm.rec + rec_base + (int64_t)(head0 + hd) * rec_hstride + t_begin / ST + (q >> 1),
                                   (uint32_t)sizeof(TileScalars), &sm->full[s]);
                 }
             }
@@ -975,20 +978,20 @@ ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         const bool leader = tc::elect_one();
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
         const uint32_t id_h = tc::idesc_bf16(128, 64 * nh, 1, 1);        // both operands MN-major
-        for (int j = 0; j < ntiles; ++j) {
-            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+        for (int q = 0; q < nhalves; ++q) {
+            const int s = q % ST_STAGES, ph = (q / ST_STAGES) & 1;
             tc::mbar_wait(&sm->scaled[s], ph, abort_flag, d_status);
             tc::tc_fence_after();
             if (leader) {
                 const uint32_t base = tc::smem_u32(smem + s * ST_STAGE_BYTES);
-                const uint64_t dBt = tc::smem_desc_sw128(base, SLAB, 1024);
-                const uint64_t dXp = tc::smem_desc_sw128(base + 2 * SLAB, SLAB, 1024);
+                const uint64_t dBt = tc::smem_desc_sw128(base, HSLAB, 1024);
+                const uint64_t dXp = tc::smem_desc_sw128(base + 2 * HSLAB, HSLAB, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
+                for (int kk = 0; kk < HT / 16; ++kk)
                     tc::mma_ss(tmem_u, tc::smem_desc_advance(dBt, kk * 2048), tc::smem_desc_advance(dXp, kk * 2048),
-                               id_h, (j > 0) || (kk > 0));
+                               id_h, (q > 0) || (kk > 0));
                 tc::mma_commit(&sm->empty[s]);
-                if (j == ntiles - 1) tc::mma_commit(&sm->done);
+                if (q == nhalves - 1) tc::mma_commit(&sm->done);
             }
             __syncwarp();
         }
@@ -1001,32 +1004,34 @@ ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
         float run_total = 0.f;                            // log2 decay over the whole segment
         for (int jr = 0; jr < ntiles; ++jr) run_total += prm.rec[rec_row + jr].ends[3];
         float run_done = 0.f;
-        for (int j = 0; j < ntiles; ++j) {
-            const int s = j % ST_STAGES, ph = (j / ST_STAGES) & 1;
+        // within a stage: this thread's token row and its half of the row's eight 16-byte chunks
+        const int srow = i >> 1, shalf = i & 1;
+        for (int q = 0; q < nhalves; ++q) {
+            const int s = q % ST_STAGES, ph = (q / ST_STAGES) & 1;
             tc::mbar_wait(&sm->full[s], ph, abort_flag, d_status);
             const TileScalars *sc = &sm->sc[s][hd];
-            run_done += sc->ends[3];
-            const uint32_t wp = sc->wp[i];
+            if ((q & 1) == 0) run_done += sc->ends[3];                 // (both halves of a tile share its record)
+            const uint32_t wp = sc->wp[(q & 1) * HT + srow];
             const float w = (__uint_as_float(wp << 16) + __uint_as_float(wp & 0xffff0000u)) *
                             tc::ex2_approx(run_total - run_done);
             const __nv_bfloat16 w_hi = __float2bfloat16_rn(w);
             const __nv_bfloat16 w_lo = __float2bfloat16_rn(w - __bfloat162float(w_hi));
             const __nv_bfloat162 w_hi2 = __halves2bfloat162(w_hi, w_hi), w_lo2 = __halves2bfloat162(w_lo, w_lo);
-            uint8_t *s_x = smem + s * ST_STAGE_BYTES + (2 + hd) * SLAB;
-            uint4 xr[8];
+            uint8_t *s_x = smem + s * ST_STAGE_BYTES + (2 + hd) * HSLAB;
+            uint4 xr[4];
 #pragma unroll
-            for (int c = 0; c < 8; ++c) xr[c] = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(i, c));
+            for (int c = 0; c < 4; ++c) xr[c] = *reinterpret_cast<const uint4 *>(s_x + tc::sw128_offset(srow, 4 * shalf + c));
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 const uint32_t wv[4] = {xr[c].x, xr[c].y, xr[c].z, xr[c].w};
                 uint32_t o[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[q]);
+                for (int e = 0; e < 4; ++e) {
+                    const __nv_bfloat162 xv = *reinterpret_cast<const __nv_bfloat162 *>(&wv[e]);
                     const __nv_bfloat162 pr = __hfma2(w_hi2, xv, __hmul2(w_lo2, xv));
-                    o[q] = *reinterpret_cast<const uint32_t *>(&pr);
+                    o[e] = *reinterpret_cast<const uint32_t *>(&pr);
                 }
-                *reinterpret_cast<uint4 *>(s_x + tc::sw128_offset(i, c)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4 *>(s_x + tc::sw128_offset(srow, 4 * shalf + c)) = make_uint4(o[0], o[1], o[2], o[3]);
             }
             tc::fence_proxy_async_smem();
             tc::mbar_arrive(&sm->scaled[s]);
@@ -1059,9 +1064,23 @@ ssd_state_kernel(const __grid_constant__ CUtensorMap tmap_bc, const __grid_const
 static size_t ssd_state_smem_bytes() { return ST_SMALL + sizeof(StateSmall); }
 
 // The state-only launch behind both the dense and the packed segment passes.
-static int launch_state_pass(LaunchCtx &ctx, const CUtensorMap &tm_bc, const CUtensorMap &tm_x, const SsdParams &p,
+static int launch_state_pass(LaunchCtx &ctx, const void *x, const void *BC, int64_t rows, int nb, const SsdParams &p,
                              unsigned grid_x, int H, int G, unsigned grid_z)
 {
+    // tensor maps with boxes of half a tile (64 tokens) over x [nb, rows, H, P] and BC [nb, rows, S]
+    CUtensorMap tm_bc, tm_x;
+    {
+        const int S = 2 * G * SN;
+        const uint64_t dims3[3] = {(uint64_t)S, (uint64_t)rows, (uint64_t)nb};
+        const uint64_t str3[2] = {(uint64_t)S * 2, (uint64_t)rows * S * 2};
+        const uint32_t box3[3] = {64, (uint32_t)HT, 1};
+        const uint64_t dims4[4] = {(uint64_t)SP, (uint64_t)H, (uint64_t)rows, (uint64_t)nb};
+        const uint64_t str4[3] = {(uint64_t)SP * 2, (uint64_t)H * SP * 2, (uint64_t)rows * H * SP * 2};
+        const uint32_t box4[4] = {SP, 1, (uint32_t)HT, 1};
+        if (!encode_tmap_bf16_cached(ctx.tmaps, &tm_bc, BC, 3, dims3, str3, box3) ||
+            !encode_tmap_bf16_cached(ctx.tmaps, &tm_x, x, 4, dims4, str4, box4))
+            return SWIMBA_ERR_CUDA;
+    }
     const size_t smem = ssd_state_smem_bytes();
     if (!ensure_dynamic_smem((const void *)ssd_state_kernel, smem)) return SWIMBA_ERR_CUDA;
     ctx.begin(STAGE_SSD_STATE);
@@ -1220,7 +1239,7 @@ int launch_ssd_tiles(LaunchCtx &ctx, const void *x, const void *BC, const float 
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
         {
             // (the last segment's end state is nobody's entry state: the full pass produces it)
-            const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)(nseg - 1), H, G, (unsigned)B);
+            const int rc = launch_state_pass(ctx, x, BC, L, B, p, (unsigned)(nseg - 1), H, G, (unsigned)B);
             if (rc != SWIMBA_OK) return rc;
         }
         const int PN4 = SP * SN / 4;
@@ -1406,7 +1425,7 @@ int launch_ssd_tiles_packed(LaunchCtx &ctx, const void *x, const void *BC, const
         float *decay = (float *)(ws + lay.decay);
         p.items = (const int2 *)(ws + lay.pre);
         p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY; p.seg_states = 1;
-        rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)pl.pre.size(), H, G, 1u);
+        rc = launch_state_pass(ctx, x, BC, T, 1, p, (unsigned)pl.pre.size(), H, G, 1u);
         if (rc != SWIMBA_OK) return rc;
         const int PN4 = SP * SN / 4;
         ctx.begin(STAGE_SEGMENT_SCAN);
@@ -1507,7 +1526,7 @@ int launch_ssd_shard_summary(LaunchCtx &ctx, const void *x, const void *BC, cons
     float *decay = (float *)((char *)workspace + lay.decay);
     p.h_in = nullptr; p.h_out = states; p.seg_decay = decay; p.mode = MODE_STATE_ONLY;
     {
-        const int rc = launch_state_pass(ctx, tm_bc, tm_x, p, (unsigned)lay.nseg, H, G, (unsigned)B);
+        const int rc = launch_state_pass(ctx, x, BC, L, B, p, (unsigned)lay.nseg, H, G, (unsigned)B);
         if (rc != SWIMBA_OK) return rc;
     }
     const int PN4 = SP * SN / 4;
