@@ -47,13 +47,13 @@ TIMED_SECONDS = 1.5   # the K-step timed region is repeated until it has covered
 # writes can still sit in L2 when it ends.
 NCU_TRAFFIC_BYTES = {
     # profiles/forward_small_lm_kernels.md (the router launch includes the SSD step sizes)
-    "small_lm": {"router_topk": 26.790e6, "expert_gemm": 36.989e6, "ssd_tiles": 83.015e6},
+    "small_lm": {"router_topk": 26.790e6, "expert_gemm": 36.989e6, "ssd_tiles": 82.690e6},
     # profiles/forward_mid_kernels.md
-    "mid": {"ssd_scalars": 8.413e6, "router_topk": 147.366e6, "expert_gemm": 258.593e6, "ssd_tiles": 580.232e6},
+    "mid": {"ssd_scalars": 8.413e6, "router_topk": 147.230e6, "expert_gemm": 256.823e6, "ssd_tiles": 584.555e6},
     # profiles/ssd_segmented_long_seq.md (the state-only pass is a kernel of its own)
-    "long_seq": {"ssd_state": 306.295e6, "ssd_tiles": 619.417e6, "segment_scan": 17.843e6},
+    "long_seq": {"ssd_state": 306.343e6, "ssd_tiles": 619.930e6, "segment_scan": 17.834e6},
     # profiles/decode_step_kernels.md
-    "decode": {"router_topk": 0.593e6, "project_small": 9.071e6, "decode_update": 479.881e6},
+    "decode": {"router_topk": 0.593e6, "project_small": 9.070e6, "decode_update": 479.990e6},
 }
 
 
