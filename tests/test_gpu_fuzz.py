@@ -76,3 +76,43 @@ def test_random_packed_batches_match_oracle(seed):
     got = tp.packed_forward(cfg, inp, lens, h0=h0)
     worst = tp.check_packed(cfg, inp, lens, got, h0=h0)
     print(cfg.dtype, cfg.P, cfg.N, lens, f"err_y={worst['err_y']:.2e} err_h={worst['err_h']:.2e}")
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_decode_loops_match_oracle(seed):
+    """A run of decode steps on a drawn shape (both front ends, tile and other state shapes, with
+    and without the skip term) against the oracle's forward over the same tokens."""
+    from paper_2603_06938_b200 import binding as sb
+    r = np.random.default_rng(3000 + seed)
+    dtype = str(r.choice(["bf16", "bf16", "fp32"]))
+    G = int(r.choice([1, 2]))
+    H = G * int(r.integers(1, 4))
+    P, N = (64, 128) if (dtype == "bf16" and r.integers(0, 3) > 0) else (int(r.choice([16, 32, 64])), int(r.choice([16, 32, 64])))
+    E = int(r.choice([1, 2, 4, 8, 16]))
+    k = int(r.integers(1, min(E, 3) + 1))
+    F = int(r.choice([64, 128, 256, 512, 8 * int(r.integers(1, 40))]))
+    B = int(r.choice([1, 2, int(r.integers(3, 40)), int(r.integers(100, 300))]))
+    L = 6 if B > 64 else int(r.integers(2, 20))
+    cfg = synth.LayerConfig("fuzz", dtype, B, L, F, H, P, N, G, E, k, 128, h0_std=0.1)
+    inp = synth.make_inputs(cfg, seed=seed)
+    if r.integers(0, 2):
+        inp["D"] = None
+    h = hp.create_handle(cfg)
+    try:
+        w, keep = hp.device_weights(inp)
+        state = hp.dev(inp["h0"]).clone()
+        ws = torch.empty(max(sb.swimba_decode_workspace_bytes(h, B), 16), dtype=torch.uint8, device="cuda")
+        ys, idxs, wts = [], [], []
+        for t in range(L):
+            u, x, dt = hp.dev(inp["u"][:, t]), hp.dev(inp["x"][:, t]), hp.dev(inp["dt"][:, t])
+            y = torch.empty_like(x)
+            idx = torch.empty(B, k, dtype=torch.int32, device="cuda")
+            wt = torch.empty(B, k, device="cuda")
+            sb.swimba_decode_step(h, w, u, x, dt, state, B, y, idx, wt, ws)
+            ys.append(y.cpu()); idxs.append(idx.cpu()); wts.append(wt.cpu())
+        assert sb.swimba_status(h) == 0, sb.swimba_last_error(h)
+    finally:
+        sb.swimba_destroy(h)
+    got = dict(y=torch.stack(ys, 1), h_final=state.cpu(), idx=torch.stack(idxs, 1), w=torch.stack(wts, 1))
+    res = hp.compare_forward(cfg, inp, got, *hp.tolerances(cfg))
+    print(cfg, f"err_y={res['err_y']:.2e} err_h={res['err_h']:.2e} ambiguous={res['ambiguous']}")
