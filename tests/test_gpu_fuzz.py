@@ -116,3 +116,40 @@ def test_random_decode_loops_match_oracle(seed):
     got = dict(y=torch.stack(ys, 1), h_final=state.cpu(), idx=torch.stack(idxs, 1), w=torch.stack(wts, 1))
     res = hp.compare_forward(cfg, inp, got, *hp.tolerances(cfg))
     print(cfg, f"err_y={res['err_y']:.2e} err_h={res['err_h']:.2e} ambiguous={res['ambiguous']}")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_weight_gradients_match_oracle(seed):
+    import oracle
+    import test_gpu_backward as tb
+    r = np.random.default_rng(4000 + seed)
+    tile = bool(r.integers(0, 3) > 0)
+    G = int(r.choice([1, 2]))
+    H = G * int(r.integers(1, 4))
+    E = int(r.choice([1, 2, 4, 8]))
+    k = int(r.integers(1, min(E, 3) + 1))
+    F = 8 * int(r.integers(2, 40))
+    B = int(r.integers(1, 4))
+    if tile:
+        dtype, P, N = "bf16", 64, 128
+        L = int(r.choice([1, int(r.integers(2, 200)), int(r.integers(200, 900)), int(r.integers(1500, 2600))]))
+    else:
+        dtype, P, N = str(r.choice(["bf16", "fp32"])), int(r.choice([16, 32, 64])), int(r.choice([16, 32, 64]))
+        L = int(r.integers(1, 200))
+    cfg = synth.LayerConfig("fuzz", dtype, B, L, F, H, P, N, G, E, k, 128)
+    inp = synth.make_inputs(cfg, seed=seed, with_dt=bool(r.integers(0, 4) > 0))
+    gen = torch.Generator().manual_seed(seed)
+    dy = torch.randn(B, L, H, P, generator=gen).to(synth.torch_dtype(dtype))
+    h0 = (0.1 * torch.randn(B, H, P, N, generator=gen)).float() if r.integers(0, 2) else None
+    dWr, dWe, idx = tb.gpu_backward(cfg, inp, dy, h0=h0)
+    W_r = inp["W_r"] if E > 1 else torch.zeros(1, F)
+    ref = oracle.backward_weights(synth.f64(inp["u"]), synth.f64(inp["x"]), synth.f64(inp["dt"]), synth.f64(W_r),
+                                  synth.f64(inp["W_e"]), synth.f64(inp["A"]), synth.f64(inp["dt_bias"]), synth.f64(dy),
+                                  k=k, G=G, h0=synth.f64(h0), forced_idx=idx.numpy())
+    tol = 2e-4 if dtype == "fp32" else 2e-2
+    err_e = tb.rel_per_expert(dWe, ref["dW_e"])
+    assert err_e <= tol, err_e
+    if E > 1:
+        den = np.abs(ref["dW_r"]).max()
+        assert np.abs(dWr.double().numpy() - ref["dW_r"]).max() <= tol * den
+    print(cfg, f"dW_e err={err_e:.2e}")
