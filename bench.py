@@ -407,6 +407,10 @@ def main():
                     help="skip the batch x input-length sweep of packed prefill and decode")
     ap.add_argument("--no-e2e", action="store_true",
                     help="skip the host-buffer leg (for profiler launch lists of the device-resident steps)")
+    ap.add_argument("--only", default=None,
+                    choices=["backward", "general", "block", "serving", "sharded"],
+                    help="run one of the side records alone on --config's workload and print it (the line is "
+                         "not a bench line; for profiler captures of those kernels)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = synth.CONFIGS[args.config]
@@ -423,6 +427,14 @@ def main():
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if args.only:
+        side = {"backward": lambda: bench_backward(sb, cfg, steps=max(1, min(args.steps, 5)), warmup=2),
+                "general": lambda: bench_general(sb, cfg, steps=max(1, min(args.steps, 10)), warmup=2),
+                "block": lambda: bench_block(sb, cfg, steps=max(1, min(args.steps, 10)), warmup=2),
+                "serving": lambda: bench_serving(sb, steps=max(1, min(args.steps, 10)), warmup=2),
+                "sharded": lambda: bench_shard(sb, steps=max(1, min(args.steps, 10)), warmup=2)}
+        print(json.dumps({"only": args.only, "record": side[args.only]()}))
+        return
     pk = peaks()
     sm_count = torch.cuda.get_device_properties(local).multi_processor_count
     stream = torch.cuda.current_stream()

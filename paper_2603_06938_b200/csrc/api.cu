@@ -897,6 +897,7 @@ int swimba_backward_weights(swimba_handle *h, const swimba_weights *w, const voi
         return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "too many tokens (B * L * top_k must stay below 2^31)");
     if (B > 65535) return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "more than 65535 sequences per call");
     if (!ssd_adjoint_supported(c.head_dim, c.d_state) || (int64_t)c.n_experts * ((T + 2047) / 2048) > 65535 ||
+        c.n_heads > 1024 ||
         (int64_t)B * c.n_heads >= (int64_t)1 << 31)
         return fail(h, SWIMBA_ERR_UNSUPPORTED_SHAPE, "shape outside what the backward kernels take");
     int rc = check_weights(h, w, true);

@@ -115,7 +115,8 @@ ssd_adjoint_kernel(const T *__restrict__ x, const T *__restrict__ dy, const T *_
     }
 }
 
-// Softmax over all E of the router logits, one warp per token: pi[T,E].
+// Softmax over all E of the router logits, one warp per token: pi[T,E].  A lane takes 8 consecutive
+// features at a time (one 16- or 32-byte load of u, reused for every expert's row).
 template <typename T>
 __global__ void __launch_bounds__(256)
 router_softmax_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_t Tn, int F, int E,
@@ -125,13 +126,23 @@ router_softmax_kernel(const T *__restrict__ u, const T *__restrict__ W_r, int64_
     const int64_t t = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (t >= Tn) return;
     float g[SWIMBA_MAX_EXPERTS];
+    for (int e = 0; e < E; ++e) g[e] = 0.f;
+    for (int f0 = lane * 8; f0 < F; f0 += 256) {            // (F is a multiple of 8)
+        float uv[8];
+        load8(u + t * F + f0, uv);
+        for (int e = 0; e < E; ++e) {
+            float wv[8];
+            load8(W_r + (int64_t)e * F + f0, wv);
+            float acc = g[e];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc = fmaf(wv[q], uv[q], acc);
+            g[e] = acc;
+        }
+    }
     float m = -INFINITY;
     for (int e = 0; e < E; ++e) {
-        float acc = 0.f;
-        for (int f = lane; f < F; f += 32) acc = fmaf(to_f32<T>(W_r[(int64_t)e * F + f]), to_f32<T>(u[t * F + f]), acc);
-        acc = warp_sum(acc);
-        g[e] = acc;
-        m = fmaxf(m, acc);
+        g[e] = warp_sum(g[e]);
+        m = fmaxf(m, g[e]);
     }
     float z = 0.f;
     for (int e = 0; e < E; ++e) { g[e] = expf(g[e] - m); z += g[e]; }
@@ -379,12 +390,18 @@ adjoint_reduce_kernel(const __nv_bfloat16 *__restrict__ yv, const float *__restr
     const int64_t ot = REVERSE ? (int64_t)b * L + (L - 1 - t) : bt;
     const int S = 2 * G * VN, HG = H / G;
     const int n = threadIdx.x, c = n >> 6, pp = n & 63;
+    __shared__ float s_delta[1024];                       // the token's step sizes, one per head
+    if (REVERSE) {
+        for (int h = threadIdx.x; h < H; h += blockDim.x)
+            s_delta[h] = softplus_f((dt ? dt[bt * H + h] : 0.f) + dt_bias[h]);
+        __syncthreads();
+    }
     for (int g = 0; g < G; ++g) {
         float acc = 0.f;
         for (int hh = 0; hh < HG; ++hh) {
             const int h = g * HG + hh;
             float v = __bfloat162float(yv[(ot * 2 * H + 2 * h + c) * VP + pp]);
-            if (REVERSE) v *= softplus_f((dt ? dt[bt * H + h] : 0.f) + dt_bias[h]);
+            if (REVERSE) v *= s_delta[h];
             acc += v;
         }
         dBC[bt * S + (int64_t)(REVERSE ? g : G + g) * VN + n] = acc;
